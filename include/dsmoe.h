@@ -1,0 +1,183 @@
+/*
+ * dsmoe -- the DS-MoE feed-forward layer at inference, for NVIDIA B200 (sm_100a).
+ *
+ * One Mixture-of-Experts FFN layer as the paper states it (Section 3.1, Eq. 1):
+ *
+ *     S = softmax(h(X)),      O = sum_{i=1..K} S_{A_i} * e_{A_i}(X)
+ *
+ * with N experts e (MLPs with GeLU, "Model Hyperparameters" paragraph), a router h,
+ * and A the indices of the K highest-scoring experts.  At inference K is either fixed
+ * or set per token by how many experts score above a threshold eps ("Sparse Inference"
+ * paragraph); the threshold is on the normalised probability S*N and must be exceeded
+ * (Section 4.2 and its footnote).  The dense-training forward evaluates every expert
+ * and weights it by its score ("Dense Training" paragraph, the forward behind Eq. 3);
+ * here it is DSMOE_SELECT_ALL.
+ *
+ * Notation: T tokens in the call, d = model width (paper d_h / D_emb), E = number of
+ * experts (paper N, N_ffd), H = hidden width of one expert (paper D_ffd),
+ * k_t = number of experts selected for token t, A = sum_t k_t assignments.
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller, row-major, 16-byte
+ *     aligned.  Nothing is allocated or freed by the library; nothing synchronises
+ *     the host.  Work is enqueued on the caller's stream.
+ *   - `desc` is a HOST pointer, read during the call only.
+ *   - Return value: DSMOE_OK or an error; on error nothing has been enqueued unless the
+ *     code is DSMOE_ERR_CUDA (a launch failed part-way).
+ *   - Limits: 1 <= E <= 64, d % 8 == 0, H % 8 == 0, T >= 0 (T == 0 is a no-op).
+ *     Violations return DSMOE_ERR_INVALID_ARG / DSMOE_ERR_UNSUPPORTED.
+ *   - Inputs must be finite; NaN/Inf give unspecified values, never a fault.
+ *   - dtype selects the storage type of x, W1, W2, xp, yp and out (fp32 or bf16).
+ *     Router weights, scores and gates are always fp32; accumulation is fp32.
+ *   - Amax = T*E for THRESHOLD and ALL, T*min(K,E) for TOPK: the capacity of every
+ *     per-assignment buffer, so the data-dependent A never has to reach the host.
+ *   - W = E for THRESHOLD and ALL, min(K,E) for TOPK: row stride of token_rows.
+ */
+#ifndef DSMOE_H_
+#define DSMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DSMOE_OK = 0,
+    DSMOE_ERR_INVALID_ARG = 1,   /* null pointer, bad shape, bad alignment, bad enum       */
+    DSMOE_ERR_UNSUPPORTED = 2,   /* valid but outside the limits above (e.g. E > 64)       */
+    DSMOE_ERR_WORKSPACE = 3,     /* ws_bytes smaller than dsmoe_workspace_size reports     */
+    DSMOE_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                      */
+    DSMOE_ERR_TIMEOUT = 5        /* written to *dev_status by a kernel whose bounded wait ran out */
+} dsmoe_status;
+
+typedef enum { DSMOE_F32 = 0, DSMOE_BF16 = 1 } dsmoe_dtype;
+
+typedef enum {
+    DSMOE_SELECT_THRESHOLD = 0,  /* expert e active iff score exceeds eps                  */
+    DSMOE_SELECT_TOPK = 1,       /* the K highest scores; ties go to the lower index       */
+    DSMOE_SELECT_ALL = 2         /* every expert: the dense-training forward               */
+} dsmoe_mode;
+
+typedef struct {
+    int32_t T, d, H, E;
+    int32_t dtype;            /* dsmoe_dtype                                               */
+    int32_t mode;             /* dsmoe_mode                                                */
+    float   eps;              /* THRESHOLD only                                            */
+    int32_t eps_normalized;   /* 1: compare S*E > eps (the paper's normalised probability,
+                                 one fp32 multiply); 0: compare S > eps                    */
+    int32_t K;                /* TOPK only; K > E behaves as K = E                         */
+    int32_t min_k;            /* 0: a token may select nothing and then outputs 0;
+                                 1: such a token keeps its lowest-index argmax             */
+    int32_t out_fp32;         /* 1: `out` is fp32 even when dtype is bf16                  */
+} dsmoe_layer_desc;
+
+/* A void* stands for the caller's cudaStream_t so that this header needs no CUDA include. */
+typedef void* dsmoe_stream;
+
+const char* dsmoe_status_string(dsmoe_status s);
+
+/* Bytes of scratch that dsmoe_permute, dsmoe_expert_mlp and dsmoe_layer_forward need for
+ * this desc (one figure, the maximum over the three and over the internal paths). */
+dsmoe_status dsmoe_workspace_size(const dsmoe_layer_desc* desc, size_t* bytes);
+
+/*
+ * Router scores, Eq. 1 (first half): scores[t,:] = softmax(x[t,:].Wr + br) over all E
+ * experts, fp32 with the row maximum subtracted.
+ *   x [T,d] dtype; Wr [d,E] fp32; br [E] fp32 or NULL; scores [T,E] fp32 (written).
+ */
+dsmoe_status dsmoe_router(const dsmoe_layer_desc* desc, const void* x, const float* Wr,
+                          const float* br, float* scores, dsmoe_stream stream);
+
+/*
+ * Expert selection ("Sparse Inference" paragraph; Section 4.2 footnote), decided in fp32
+ * on the given scores, so identical scores give bit-identical results everywhere.
+ *   scores [T,E] fp32 (read); mask [T] uint64, bit e set iff expert e is selected;
+ *   k_t [T] int32 = popcount(mask); counts [E] int32 = tokens per expert;
+ *   offsets [E+1] int32 = exclusive prefix sum of counts, offsets[E] = A.
+ * All four outputs are written in full.  workspace as reported by dsmoe_workspace_size.
+ */
+dsmoe_status dsmoe_select(const dsmoe_layer_desc* desc, const float* scores, uint64_t* mask,
+                          int32_t* k_t, int32_t* counts, int32_t* offsets, void* workspace,
+                          size_t ws_bytes, dsmoe_stream stream);
+
+/*
+ * Grouping of tokens by expert -- the token duplication the "GPU Inference Analysis"
+ * section names.  Row r in [offsets[e], offsets[e+1]) holds the token with the
+ * (r - offsets[e])-th smallest index among those that selected e.
+ *   x [T,d] dtype, scores [T,E], mask [T], offsets [E+1]: read.
+ *   row_token [Amax] int32: token of row r;  row_gate [Amax] fp32: scores[token,e];
+ *   token_rows [T,W] int32: rows of token t in ascending expert order, -1 beyond k_t;
+ *   xp [Amax,d] dtype: xp[r,:] = x[row_token[r],:].  Entries at r >= A are not written.
+ */
+dsmoe_status dsmoe_permute(const dsmoe_layer_desc* desc, const void* x, const float* scores,
+                           const uint64_t* mask, const int32_t* offsets, int32_t* row_token,
+                           float* row_gate, int32_t* token_rows, void* xp, void* workspace,
+                           size_t ws_bytes, dsmoe_stream stream);
+
+/*
+ * The selected experts' MLPs on grouped rows (Eq. 1's e(X); GeLU is the exact erf form):
+ * yp[r,:] = GeLU(xp[r,:].W1[e]).W2[e] for r in [offsets[e], offsets[e+1]).
+ *   xp [Amax,d] dtype; W1 [E,d,H] dtype; W2 [E,H,d] dtype; offsets [E+1]: read.
+ *   yp [Amax,d] dtype (written for r < A).
+ *   packed: NULL, or the buffer dsmoe_pack_weights filled from these W1, W2 (bf16 only);
+ *   with it the tensor-core kernels run, without it a plain fp32-FMA kernel does.
+ */
+dsmoe_status dsmoe_expert_mlp(const dsmoe_layer_desc* desc, const void* xp, const void* W1,
+                              const void* W2, const void* packed, const int32_t* offsets,
+                              void* yp, void* workspace, size_t ws_bytes, int32_t* dev_status,
+                              dsmoe_stream stream);
+
+/*
+ * Aggregation of expert outputs back into token order (Eq. 1's sum; the aggregation the
+ * "GPU Inference Analysis" section names): out[t,:] = sum_i row_gate[r_i] * yp[r_i,:]
+ * over r_i = token_rows[t,i], i < k_t[t], accumulated in fp32 in that order and rounded
+ * once.  A token with k_t = 0 gets zeros.
+ *   yp [Amax,d] dtype; row_gate [Amax]; token_rows [T,W]; k_t [T]: read.
+ *   out [T,d] dtype (fp32 if desc->out_fp32).
+ */
+dsmoe_status dsmoe_combine(const dsmoe_layer_desc* desc, const void* yp, const float* row_gate,
+                           const int32_t* token_rows, const int32_t* k_t, void* out,
+                           dsmoe_stream stream);
+
+/*
+ * Kernel-preferred copy of the (static, post-training) expert weights: W1 transposed to
+ * [E,H,d] followed by W2 transposed to [E,d,H], both bf16, so that every tensor-core
+ * operand is contiguous along the reduction.  dtype must be DSMOE_BF16.
+ * dsmoe_packed_size reports the bytes `packed` must hold.
+ */
+dsmoe_status dsmoe_packed_size(const dsmoe_layer_desc* desc, size_t* bytes);
+dsmoe_status dsmoe_pack_weights(const dsmoe_layer_desc* desc, const void* W1, const void* W2,
+                                void* packed, dsmoe_stream stream);
+
+/*
+ * The whole layer, Eq. 1: router -> selection -> grouping -> experts -> combine, or, for
+ * DSMOE_SELECT_ALL, the dense-training forward  out = sum_e S_e * e_e(x).
+ *   x [T,d]; Wr [d,E]; br [E] or NULL; W1 [E,d,H]; W2 [E,H,d]; packed NULL or from
+ *   dsmoe_pack_weights (W1/W2 may then be NULL); out [T,d] dtype (fp32 if out_fp32).
+ *   mask_out [T] uint64 and counts_out [E] int32: optional copies of the selection.
+ *   dev_status: optional device int32; kernels write a dsmoe_status there if a bounded
+ *   wait runs out or an index check fails (they then exit cleanly); untouched otherwise.
+ */
+dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, const float* Wr,
+                                 const float* br, const void* W1, const void* W2,
+                                 const void* packed, void* out, uint64_t* mask_out,
+                                 int32_t* counts_out, void* workspace, size_t ws_bytes,
+                                 int32_t* dev_status, dsmoe_stream stream);
+
+/*
+ * Same call with HOST buffers for x and out (pinned or pageable): copies x to the device,
+ * runs dsmoe_layer_forward, copies out back and waits for the stream.  x_dev [T,d] and
+ * out_dev [T,d] are device staging buffers supplied by the caller.
+ */
+dsmoe_status dsmoe_layer_forward_host(const dsmoe_layer_desc* desc, const void* x_host,
+                                      void* x_dev, const float* Wr, const float* br,
+                                      const void* W1, const void* W2, const void* packed,
+                                      void* out_dev, void* out_host, void* workspace,
+                                      size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSMOE_H_ */
