@@ -1,0 +1,70 @@
+// Shared declarations of the dsmoe CUDA library: argument checks, the workspace layout and the
+// internal launchers that the C entry points in api.cu call.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "dsmoe.h"
+
+namespace dsmoe {
+
+constexpr int kMaxExperts = 64;
+constexpr int kChunk = 32;   // tokens per ballot chunk in the grouping kernels
+
+#define DSMOE_CUDA_TRY(expr)                                  \
+    do {                                                      \
+        cudaError_t err__ = (expr);                           \
+        if (err__ != cudaSuccess) return DSMOE_ERR_CUDA;      \
+    } while (0)
+
+#define DSMOE_TRY(expr)                                       \
+    do {                                                      \
+        dsmoe_status st__ = (expr);                           \
+        if (st__ != DSMOE_OK) return st__;                    \
+    } while (0)
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+static inline size_t elem_size(int dtype) { return dtype == DSMOE_BF16 ? 2 : 4; }
+static inline int width_of(const dsmoe_layer_desc& p) {
+    return p.mode == DSMOE_SELECT_TOPK ? (p.K < p.E ? p.K : p.E) : p.E;
+}
+static inline size_t amax_of(const dsmoe_layer_desc& p) { return (size_t)p.T * (size_t)width_of(p); }
+
+dsmoe_status check_desc(const dsmoe_layer_desc* desc);
+static inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+// Byte offsets of every internal buffer inside the caller's workspace.
+struct WsLayout {
+    size_t scores, mask, k_t, counts, offsets, chunk_prefix, row_token, row_gate, token_rows;
+    size_t xp, h, yp, partial, total;
+};
+WsLayout ws_layout(const dsmoe_layer_desc& p);
+
+// ---- router.cu
+dsmoe_status launch_router(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
+                           float* scores, uint64_t* mask, int32_t* k_t, cudaStream_t s);
+dsmoe_status launch_select(const dsmoe_layer_desc& p, const float* scores, uint64_t* mask, int32_t* k_t,
+                           cudaStream_t s);
+dsmoe_status launch_finalize(const dsmoe_layer_desc& p, const uint64_t* mask, int32_t* counts,
+                             int32_t* offsets, int32_t* chunk_prefix, int32_t* counts_out, cudaStream_t s);
+
+// ---- permute.cu
+dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const float* scores,
+                            const uint64_t* mask, const int32_t* offsets, const int32_t* chunk_prefix,
+                            int32_t* row_token, float* row_gate, int32_t* token_rows, void* xp,
+                            cudaStream_t s);
+dsmoe_status launch_combine(const dsmoe_layer_desc& p, const void* yp, const float* row_gate,
+                            const int32_t* token_rows, const int32_t* k_t, void* out, cudaStream_t s);
+dsmoe_status launch_pack(const dsmoe_layer_desc& p, const void* W1, const void* W2, void* packed,
+                         cudaStream_t s);
+
+// ---- mlp_generic.cu : plain fp32-FMA grouped GEMMs (any dtype, no packed weights needed)
+dsmoe_status launch_mlp_generic(const dsmoe_layer_desc& p, const void* xp, const void* W1, const void* W2,
+                                const int32_t* offsets, float* h, void* yp, cudaStream_t s);
+
+}  // namespace dsmoe

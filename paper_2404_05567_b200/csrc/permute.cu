@@ -1,0 +1,204 @@
+// Grouping of tokens by expert and the router-weighted aggregation back into token order -- the
+// "duplication of intermediate tokens and the aggregation of outputs" that the paper's GPU
+// Inference Analysis names as the overhead of sparse inference -- plus the one-off weight packer.
+#include "common.cuh"
+
+namespace dsmoe {
+
+// Row indices.  A warp owns a chunk of 32 consecutive tokens; for expert e the ballot of "selected"
+// gives each token its rank inside the chunk, and chunk_prefix gives the number of earlier tokens,
+// so rows inside an expert segment ascend by token without any atomic.
+__global__ void __launch_bounds__(256) permute_index_kernel(const uint64_t* __restrict__ mask,
+                                                            const float* __restrict__ scores,
+                                                            const int32_t* __restrict__ offsets,
+                                                            const int32_t* __restrict__ chunk_prefix,
+                                                            int32_t* __restrict__ row_token, float* __restrict__ row_gate,
+                                                            int32_t* __restrict__ token_rows, int T, int E, int W,
+                                                            int64_t amax) {
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (c * kChunk >= T) return;
+    const int t = c * kChunk + lane;
+    const uint64_t m = t < T ? mask[t] : 0;
+    int slot = 0;
+    for (int e = 0; e < E; ++e) {
+        const bool bit = (m >> e) & 1;
+        const unsigned b = __ballot_sync(0xffffffffu, bit);
+        if (bit) {
+            const int r = offsets[e] + chunk_prefix[(size_t)c * E + e] + __popc(b & ((1u << lane) - 1u));
+            if (r >= 0 && r < amax) {   // inconsistent caller-supplied offsets must not become a wild store
+                row_token[r] = t;
+                row_gate[r] = scores[(size_t)t * E + e];
+            }
+            if (slot < W) token_rows[(size_t)t * W + slot] = r;
+            ++slot;
+        }
+    }
+    if (t < T)
+        for (; slot < W; ++slot) token_rows[(size_t)t * W + slot] = -1;
+}
+
+// xp[r,:] = x[row_token[r],:] for r < A, 16 bytes per lane per step, one warp per row.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ row_token,
+                                                          const int32_t* __restrict__ offsets, uint4* __restrict__ xp,
+                                                          int E, int T, int vec_per_row, int64_t amax) {
+    const int64_t A = min((int64_t)offsets[E], amax);
+    const int lane = threadIdx.x & 31;
+    const int warps = gridDim.x * 8;
+    for (int64_t r = blockIdx.x * 8 + (threadIdx.x >> 5); r < A; r += warps) {
+        const int t = row_token[r];
+        if ((unsigned)t >= (unsigned)T) continue;   // never trust an index blindly
+        const uint4* src = x + (size_t)t * vec_per_row;
+        uint4* dst = xp + (size_t)r * vec_per_row;
+        for (int v = lane; v < vec_per_row; v += 32) dst[v] = __ldg(src + v);
+    }
+}
+
+__device__ __forceinline__ void fma8(float (&acc)[8], const uint4 v, float g) {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(h[i]);
+        acc[2 * i] = fmaf(g, f.x, acc[2 * i]);
+        acc[2 * i + 1] = fmaf(g, f.y, acc[2 * i + 1]);
+    }
+}
+
+// out[t,:] = sum_i gate[r_i] * yp[r_i,:] in ascending expert order, fp32, one rounding.  Block per token.
+template <bool OUT_F32>
+__global__ void __launch_bounds__(128) combine_bf16_kernel(const uint4* __restrict__ yp, const float* __restrict__ row_gate,
+                                                           const int32_t* __restrict__ token_rows,
+                                                           const int32_t* __restrict__ k_t, void* __restrict__ out,
+                                                           int d, int W, int64_t amax) {
+    __shared__ int32_t rows_s[kMaxExperts];
+    __shared__ float gate_s[kMaxExperts];
+    const int t = blockIdx.x;
+    const int k = max(0, min(k_t[t], W));
+    if ((int)threadIdx.x < k) {
+        const int r = token_rows[(size_t)t * W + threadIdx.x];
+        const bool ok = r >= 0 && r < amax;
+        rows_s[threadIdx.x] = ok ? r : 0;
+        gate_s[threadIdx.x] = ok ? row_gate[r] : 0.f;
+    }
+    __syncthreads();
+    const int nvec = d / 8;
+    for (int v = threadIdx.x; v < nvec; v += 128) {
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+        for (int i = 0; i < k; ++i) fma8(acc, __ldg(yp + (size_t)rows_s[i] * nvec + v), gate_s[i]);
+        if (OUT_F32) {
+            float4* o = reinterpret_cast<float4*>(out) + ((size_t)t * nvec + v) * 2;
+            o[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            o[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+        } else {
+            uint4 pk;
+            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+            reinterpret_cast<uint4*>(out)[(size_t)t * nvec + v] = pk;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(128) combine_f32_kernel(const float4* __restrict__ yp, const float* __restrict__ row_gate,
+                                                          const int32_t* __restrict__ token_rows,
+                                                          const int32_t* __restrict__ k_t, float4* __restrict__ out,
+                                                          int d, int W, int64_t amax) {
+    __shared__ int32_t rows_s[kMaxExperts];
+    __shared__ float gate_s[kMaxExperts];
+    const int t = blockIdx.x;
+    const int k = max(0, min(k_t[t], W));
+    if ((int)threadIdx.x < k) {
+        const int r = token_rows[(size_t)t * W + threadIdx.x];
+        const bool ok = r >= 0 && r < amax;
+        rows_s[threadIdx.x] = ok ? r : 0;
+        gate_s[threadIdx.x] = ok ? row_gate[r] : 0.f;
+    }
+    __syncthreads();
+    const int nvec = d / 4;
+    for (int v = threadIdx.x; v < nvec; v += 128) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = 0; i < k; ++i) {
+            const float4 y = __ldg(yp + (size_t)rows_s[i] * nvec + v);
+            const float g = gate_s[i];
+            acc.x = fmaf(g, y.x, acc.x);
+            acc.y = fmaf(g, y.y, acc.y);
+            acc.z = fmaf(g, y.z, acc.z);
+            acc.w = fmaf(g, y.w, acc.w);
+        }
+        out[(size_t)t * nvec + v] = acc;
+    }
+}
+
+// dst[b][c][r] = src[b][r][c] for a batch of [rows, cols] bf16 matrices (32x32 tiles through smem).
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src,
+                                                             __nv_bfloat16* __restrict__ dst, int rows, int cols) {
+    __shared__ __nv_bfloat16 tile[32][33];
+    const size_t base = (size_t)blockIdx.z * rows * cols;
+    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int i = ty; i < 32; i += 8) {
+        const int r = r0 + i, c = c0 + tx;
+        if (r < rows && c < cols) tile[i][tx] = src[base + (size_t)r * cols + c];
+    }
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) {
+        const int c = c0 + i, r = r0 + tx;
+        if (r < rows && c < cols) dst[base + (size_t)c * rows + r] = tile[tx][i];
+    }
+}
+
+dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const float* scores, const uint64_t* mask,
+                            const int32_t* offsets, const int32_t* chunk_prefix, int32_t* row_token, float* row_gate,
+                            int32_t* token_rows, void* xp, cudaStream_t s) {
+    if (p.T == 0) return DSMOE_OK;
+    const int nchunks = ceil_div(p.T, kChunk);
+    const int64_t amax = (int64_t)amax_of(p);
+    permute_index_kernel<<<ceil_div(nchunks, 8), 256, 0, s>>>(mask, scores, offsets, chunk_prefix, row_token, row_gate,
+                                                             token_rows, p.T, p.E, width_of(p), amax);
+    DSMOE_CUDA_TRY(cudaGetLastError());
+    if (xp) {
+        const int vec_per_row = (int)((size_t)p.d * elem_size(p.dtype) / 16);
+        const int grid = (int)(amax / 8 + 1 < 148 * 16 ? amax / 8 + 1 : 148 * 16);
+        gather_rows_kernel<<<grid, 256, 0, s>>>(static_cast<const uint4*>(x), row_token, offsets,
+                                                static_cast<uint4*>(xp), p.E, p.T, vec_per_row, amax);
+        DSMOE_CUDA_TRY(cudaGetLastError());
+    }
+    return DSMOE_OK;
+}
+
+dsmoe_status launch_combine(const dsmoe_layer_desc& p, const void* yp, const float* row_gate, const int32_t* token_rows,
+                            const int32_t* k_t, void* out, cudaStream_t s) {
+    if (p.T == 0) return DSMOE_OK;
+    const int W = width_of(p);
+    const int64_t amax = (int64_t)amax_of(p);
+    if (p.dtype == DSMOE_BF16) {
+        if (p.out_fp32)
+            combine_bf16_kernel<true><<<p.T, 128, 0, s>>>(static_cast<const uint4*>(yp), row_gate, token_rows, k_t, out,
+                                                         p.d, W, amax);
+        else
+            combine_bf16_kernel<false><<<p.T, 128, 0, s>>>(static_cast<const uint4*>(yp), row_gate, token_rows, k_t, out,
+                                                          p.d, W, amax);
+    } else {
+        combine_f32_kernel<<<p.T, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t,
+                                               static_cast<float4*>(out), p.d, W, amax);
+    }
+    DSMOE_CUDA_TRY(cudaGetLastError());
+    return DSMOE_OK;
+}
+
+dsmoe_status launch_pack(const dsmoe_layer_desc& p, const void* W1, const void* W2, void* packed, cudaStream_t s) {
+    const __nv_bfloat16* w1 = static_cast<const __nv_bfloat16*>(W1);
+    const __nv_bfloat16* w2 = static_cast<const __nv_bfloat16*>(W2);
+    __nv_bfloat16* w1t = static_cast<__nv_bfloat16*>(packed);
+    __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
+    // W1[e]: [d,H] -> [H,d];  W2[e]: [H,d] -> [d,H]
+    transpose_bf16_kernel<<<dim3(ceil_div(p.H, 32), ceil_div(p.d, 32), p.E), 256, 0, s>>>(w1, w1t, p.d, p.H);
+    DSMOE_CUDA_TRY(cudaGetLastError());
+    transpose_bf16_kernel<<<dim3(ceil_div(p.d, 32), ceil_div(p.H, 32), p.E), 256, 0, s>>>(w2, w2t, p.H, p.d);
+    DSMOE_CUDA_TRY(cudaGetLastError());
+    return DSMOE_OK;
+}
+
+}  // namespace dsmoe
