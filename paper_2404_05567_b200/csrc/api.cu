@@ -1,0 +1,213 @@
+// C entry points of the dsmoe library: argument validation, workspace carving and the dispatch
+// between the execution paths of one MoE layer call (Eq. 1).
+#include "common.cuh"
+
+namespace dsmoe {
+
+dsmoe_status check_desc(const dsmoe_layer_desc* p) {
+    if (!p) return DSMOE_ERR_INVALID_ARG;
+    if (p->T < 0 || p->d <= 0 || p->H <= 0 || p->E <= 0) return DSMOE_ERR_INVALID_ARG;
+    if (p->dtype != DSMOE_F32 && p->dtype != DSMOE_BF16) return DSMOE_ERR_INVALID_ARG;
+    if (p->mode != DSMOE_SELECT_THRESHOLD && p->mode != DSMOE_SELECT_TOPK && p->mode != DSMOE_SELECT_ALL)
+        return DSMOE_ERR_INVALID_ARG;
+    if (p->mode == DSMOE_SELECT_TOPK && p->K < 1) return DSMOE_ERR_INVALID_ARG;
+    if (p->min_k != 0 && p->min_k != 1) return DSMOE_ERR_INVALID_ARG;
+    if (p->eps_normalized != 0 && p->eps_normalized != 1) return DSMOE_ERR_INVALID_ARG;
+    if (p->out_fp32 != 0 && p->out_fp32 != 1) return DSMOE_ERR_INVALID_ARG;
+    if (p->mode == DSMOE_SELECT_THRESHOLD && !(p->eps == p->eps)) return DSMOE_ERR_INVALID_ARG;   // NaN
+    if ((p->d & 7) || (p->H & 7)) return DSMOE_ERR_INVALID_ARG;
+    if (p->E > kMaxExperts) return DSMOE_ERR_UNSUPPORTED;
+    // every per-assignment index is an int32
+    if ((double)p->T * p->E * (double)(p->d > p->H ? p->d : p->H) > 9.0e15) return DSMOE_ERR_UNSUPPORTED;
+    if ((size_t)p->T * (size_t)p->E > 0x7fffffffull) return DSMOE_ERR_UNSUPPORTED;
+    return DSMOE_OK;
+}
+
+WsLayout ws_layout(const dsmoe_layer_desc& p) {
+    WsLayout L{};
+    const size_t T = (size_t)p.T, E = (size_t)p.E, amax = amax_of(p), es = elem_size(p.dtype);
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t at = off;
+        off = align_up(off + bytes, 256);
+        return at;
+    };
+    L.scores = take(T * E * 4);
+    L.mask = take(T * 8);
+    L.k_t = take(T * 4);
+    L.counts = take(kMaxExperts * 4);
+    L.offsets = take((kMaxExperts + 1) * 4);
+    L.chunk_prefix = take((size_t)ceil_div(p.T, kChunk) * E * 4);
+    L.row_token = take(amax * 4);
+    L.row_gate = take(amax * 4);
+    L.token_rows = take(T * (size_t)width_of(p) * 4);
+    L.xp = take(amax * p.d * es);
+    L.h = take(amax * p.H * 4);          // fp32 in the plain path, bf16 (half of it) in the tensor-core paths
+    L.yp = take(amax * p.d * es);
+    L.partial = take((size_t)4 << 20);   // split-K partial sums of the small-T path
+    L.total = off;
+    return L;
+}
+
+static const char* const kStatusText[] = {
+    "ok", "invalid argument", "unsupported configuration", "workspace too small", "CUDA call failed",
+    "bounded wait expired on the device"};
+
+}  // namespace dsmoe
+
+using namespace dsmoe;
+
+extern "C" {
+
+const char* dsmoe_status_string(dsmoe_status s) {
+    return ((int)s >= 0 && (int)s <= 5) ? kStatusText[(int)s] : "unknown status";
+}
+
+dsmoe_status dsmoe_workspace_size(const dsmoe_layer_desc* desc, size_t* bytes) {
+    DSMOE_TRY(check_desc(desc));
+    if (!bytes) return DSMOE_ERR_INVALID_ARG;
+    *bytes = ws_layout(*desc).total;
+    return DSMOE_OK;
+}
+
+dsmoe_status dsmoe_router(const dsmoe_layer_desc* desc, const void* x, const float* Wr, const float* br,
+                          float* scores, dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    if (desc->T == 0) return DSMOE_OK;
+    if (!x || !Wr || !scores || !aligned16(x) || !aligned16(Wr)) return DSMOE_ERR_INVALID_ARG;
+    return launch_router(*desc, x, Wr, br, scores, nullptr, nullptr, (cudaStream_t)stream);
+}
+
+dsmoe_status dsmoe_select(const dsmoe_layer_desc* desc, const float* scores, uint64_t* mask, int32_t* k_t,
+                          int32_t* counts, int32_t* offsets, void* workspace, size_t ws_bytes,
+                          dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    if (!mask && desc->T > 0) return DSMOE_ERR_INVALID_ARG;
+    if (!counts || !offsets || (!scores && desc->T > 0) || (!k_t && desc->T > 0)) return DSMOE_ERR_INVALID_ARG;
+    const WsLayout L = ws_layout(*desc);
+    if (!workspace || ws_bytes < L.total) return DSMOE_ERR_WORKSPACE;
+    char* ws = static_cast<char*>(workspace);
+    cudaStream_t s = (cudaStream_t)stream;
+    DSMOE_TRY(launch_select(*desc, scores, mask, k_t, s));
+    return launch_finalize(*desc, mask, counts, offsets, reinterpret_cast<int32_t*>(ws + L.chunk_prefix), nullptr, s);
+}
+
+dsmoe_status dsmoe_permute(const dsmoe_layer_desc* desc, const void* x, const float* scores, const uint64_t* mask,
+                           const int32_t* offsets, int32_t* row_token, float* row_gate, int32_t* token_rows,
+                           void* xp, void* workspace, size_t ws_bytes, dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    if (desc->T == 0) return DSMOE_OK;
+    if (!x || !scores || !mask || !offsets || !row_token || !row_gate || !token_rows || !xp) return DSMOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(xp)) return DSMOE_ERR_INVALID_ARG;
+    const WsLayout L = ws_layout(*desc);
+    if (!workspace || ws_bytes < L.total) return DSMOE_ERR_WORKSPACE;
+    char* ws = static_cast<char*>(workspace);
+    cudaStream_t s = (cudaStream_t)stream;
+    // recompute the per-chunk ranks from the mask (the caller's offsets are used as given)
+    int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+    int32_t* offs_scratch = reinterpret_cast<int32_t*>(ws + L.offsets);
+    int32_t* chunk_prefix = reinterpret_cast<int32_t*>(ws + L.chunk_prefix);
+    DSMOE_TRY(launch_finalize(*desc, mask, counts, offs_scratch, chunk_prefix, nullptr, s));
+    return launch_permute(*desc, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, xp, s);
+}
+
+dsmoe_status dsmoe_expert_mlp(const dsmoe_layer_desc* desc, const void* xp, const void* W1, const void* W2,
+                              const void* packed, const int32_t* offsets, void* yp, void* workspace,
+                              size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    if (desc->T == 0) return DSMOE_OK;
+    if (!xp || !offsets || !yp || !aligned16(xp) || !aligned16(yp)) return DSMOE_ERR_INVALID_ARG;
+    if (packed && desc->dtype != DSMOE_BF16) return DSMOE_ERR_INVALID_ARG;
+    if (!packed && (!W1 || !W2 || !aligned16(W1) || !aligned16(W2))) return DSMOE_ERR_INVALID_ARG;
+    const WsLayout L = ws_layout(*desc);
+    if (!workspace || ws_bytes < L.total) return DSMOE_ERR_WORKSPACE;
+    char* ws = static_cast<char*>(workspace);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (packed) return launch_mlp_umma(*desc, xp, packed, offsets, ws + L.h, yp, dev_status, s);
+    return launch_mlp_generic(*desc, xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h), yp, s);
+}
+
+dsmoe_status dsmoe_combine(const dsmoe_layer_desc* desc, const void* yp, const float* row_gate,
+                           const int32_t* token_rows, const int32_t* k_t, void* out, dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    if (desc->T == 0) return DSMOE_OK;
+    if (!yp || !row_gate || !token_rows || !k_t || !out || !aligned16(yp) || !aligned16(out)) return DSMOE_ERR_INVALID_ARG;
+    return launch_combine(*desc, yp, row_gate, token_rows, k_t, out, (cudaStream_t)stream);
+}
+
+dsmoe_status dsmoe_packed_size(const dsmoe_layer_desc* desc, size_t* bytes) {
+    DSMOE_TRY(check_desc(desc));
+    if (!bytes || desc->dtype != DSMOE_BF16) return DSMOE_ERR_INVALID_ARG;
+    *bytes = (size_t)2 * desc->E * desc->H * desc->d * 2;
+    return DSMOE_OK;
+}
+
+dsmoe_status dsmoe_pack_weights(const dsmoe_layer_desc* desc, const void* W1, const void* W2, void* packed,
+                                dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    if (desc->dtype != DSMOE_BF16 || !W1 || !W2 || !packed || !aligned16(packed)) return DSMOE_ERR_INVALID_ARG;
+    return launch_pack(*desc, W1, W2, packed, (cudaStream_t)stream);
+}
+
+dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, const float* Wr, const float* br,
+                                 const void* W1, const void* W2, const void* packed, void* out,
+                                 uint64_t* mask_out, int32_t* counts_out, void* workspace, size_t ws_bytes,
+                                 int32_t* dev_status, dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    const dsmoe_layer_desc& p = *desc;
+    if (p.T == 0) return DSMOE_OK;
+    if (!x || !Wr || !out || !aligned16(x) || !aligned16(Wr) || !aligned16(out)) return DSMOE_ERR_INVALID_ARG;
+    if (packed && p.dtype != DSMOE_BF16) return DSMOE_ERR_INVALID_ARG;
+    if (!packed && (!W1 || !W2 || !aligned16(W1) || !aligned16(W2))) return DSMOE_ERR_INVALID_ARG;
+    const WsLayout L = ws_layout(p);
+    if (!workspace || ws_bytes < L.total || !aligned16(workspace)) return DSMOE_ERR_WORKSPACE;
+    char* ws = static_cast<char*>(workspace);
+    cudaStream_t s = (cudaStream_t)stream;
+
+    float* scores = reinterpret_cast<float*>(ws + L.scores);
+    uint64_t* mask = mask_out ? mask_out : reinterpret_cast<uint64_t*>(ws + L.mask);
+    int32_t* k_t = reinterpret_cast<int32_t*>(ws + L.k_t);
+    int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+    int32_t* offsets = reinterpret_cast<int32_t*>(ws + L.offsets);
+    int32_t* chunk_prefix = reinterpret_cast<int32_t*>(ws + L.chunk_prefix);
+    int32_t* row_token = reinterpret_cast<int32_t*>(ws + L.row_token);
+    float* row_gate = reinterpret_cast<float*>(ws + L.row_gate);
+    int32_t* token_rows = reinterpret_cast<int32_t*>(ws + L.token_rows);
+
+    DSMOE_TRY(launch_router(p, x, Wr, br, scores, mask, k_t, s));
+
+    if (packed) {
+        bool done = false;
+        DSMOE_TRY(launch_layer_umma(p, x, packed, scores, mask, k_t, counts_out, out, ws, L, dev_status, s, &done));
+        if (done) return DSMOE_OK;
+    }
+
+    // grouped path: duplicate tokens per selected expert, run the experts, aggregate
+    DSMOE_TRY(launch_finalize(p, mask, counts, offsets, chunk_prefix, counts_out, s));
+    DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, ws + L.xp, s));
+    if (packed)
+        DSMOE_TRY(launch_mlp_umma(p, ws + L.xp, packed, offsets, ws + L.h, ws + L.yp, dev_status, s));
+    else
+        DSMOE_TRY(launch_mlp_generic(p, ws + L.xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h), ws + L.yp, s));
+    return launch_combine(p, ws + L.yp, row_gate, token_rows, k_t, out, s);
+}
+
+dsmoe_status dsmoe_layer_forward_host(const dsmoe_layer_desc* desc, const void* x_host, void* x_dev,
+                                      const float* Wr, const float* br, const void* W1, const void* W2,
+                                      const void* packed, void* out_dev, void* out_host, void* workspace,
+                                      size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    if (desc->T == 0) return DSMOE_OK;
+    if (!x_host || !x_dev || !out_dev || !out_host) return DSMOE_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t n = (size_t)desc->T * desc->d;
+    const size_t out_es = desc->out_fp32 ? 4 : elem_size(desc->dtype);
+    DSMOE_CUDA_TRY(cudaMemcpyAsync(x_dev, x_host, n * elem_size(desc->dtype), cudaMemcpyHostToDevice, s));
+    DSMOE_TRY(dsmoe_layer_forward(desc, x_dev, Wr, br, W1, W2, packed, out_dev, nullptr, nullptr, workspace, ws_bytes,
+                                  dev_status, stream));
+    DSMOE_CUDA_TRY(cudaMemcpyAsync(out_host, out_dev, n * out_es, cudaMemcpyDeviceToHost, s));
+    DSMOE_CUDA_TRY(cudaStreamSynchronize(s));
+    return DSMOE_OK;
+}
+
+}  // extern "C"

@@ -67,4 +67,15 @@ dsmoe_status launch_pack(const dsmoe_layer_desc& p, const void* W1, const void* 
 dsmoe_status launch_mlp_generic(const dsmoe_layer_desc& p, const void* xp, const void* W1, const void* W2,
                                 const int32_t* offsets, float* h, void* yp, cudaStream_t s);
 
+
+// ---- mlp_umma.cu : tcgen05 / TMEM / TMA kernels on packed bf16 weights
+// Grouped expert MLPs on expert-sorted rows: h = GeLU(xp.W1[e]) (bf16, in `hbuf`), yp = h.W2[e].
+dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,
+                             void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s);
+// Whole-layer paths that need no grouping (all experts selected, or few tokens).  *done = false
+// means "not taken": the caller continues with the grouped path.
+dsmoe_status launch_layer_umma(const dsmoe_layer_desc& p, const void* x, const void* packed, const float* scores,
+                               const uint64_t* mask, const int32_t* k_t, int32_t* counts_out, void* out, char* ws,
+                               const WsLayout& L, int32_t* dev_status, cudaStream_t s, bool* done);
+
 }  // namespace dsmoe

@@ -1,0 +1,134 @@
+"""Shared helpers of the GPU parity tests: move generated inputs to the device, call the C-ABI
+through the binding, fetch results as numpy, and compare with the CPU oracle."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import dsmoe_inputs as gi
+import oracle
+import paper_2404_05567_b200 as dm
+
+TOL_BF16 = 2e-2      # max|gpu - oracle| <= 2e-2 * RMS(oracle)   (bf16 storage, fp32 accumulate)
+TOL_F32 = 1e-4       # max|gpu - oracle| <= 1e-4 * RMS(oracle)   (fp32)
+NEAR = 1e-6          # scores this close to a decision boundary may legitimately flip
+
+
+def to_dev(a: np.ndarray) -> torch.Tensor:
+    """numpy (float32 / uint16 bf16 bits / ints) -> CUDA tensor with the matching torch dtype."""
+    if a is None:
+        return None
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    if a.dtype == np.uint64:
+        return torch.from_numpy(a.view(np.int64)).cuda()
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def to_np(t: torch.Tensor) -> np.ndarray:
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).cpu().numpy().view(np.uint16)
+    return t.cpu().numpy()
+
+
+def np_f32(t: torch.Tensor) -> np.ndarray:
+    return t.float().cpu().numpy()
+
+
+def desc_of(s: gi.LayerSpec) -> dm.LayerDesc:
+    return dm.make_desc(s.T, s.d, s.H, s.E, dm.BF16 if s.dtype == "bf16" else dm.F32, s.mode, s.eps,
+                        s.eps_normalized, s.K, s.min_k, s.out_fp32)
+
+
+def torch_dtype(s: gi.LayerSpec):
+    return torch.bfloat16 if s.dtype == "bf16" else torch.float32
+
+
+class Layer:
+    """One synthetic layer resident on the GPU plus the numpy originals for the oracle."""
+
+    def __init__(self, s: gi.LayerSpec, pack: bool = True, layer: int = 0, batch: str = "x"):
+        self.s = s
+        self.desc = desc_of(s)
+        self.x = gi.tokens(s, batch)
+        self.Wr, self.br = gi.router(s, layer)
+        self.W1, self.W2 = gi.experts(s, layer)
+        self.x_d, self.Wr_d, self.br_d = to_dev(self.x), to_dev(self.Wr), to_dev(self.br)
+        self.W1_d, self.W2_d = to_dev(self.W1), to_dev(self.W2)
+        self.ws = torch.empty(dm.dsmoe_workspace_size(self.desc), dtype=torch.uint8, device="cuda")
+        self.packed = None
+        if pack and s.dtype == "bf16":
+            self.packed = torch.empty(dm.dsmoe_packed_size(self.desc), dtype=torch.uint8, device="cuda")
+            dm.dsmoe_pack_weights(self.desc, self.W1_d, self.W2_d, self.packed)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out_dtype = torch.float32 if (s.out_fp32 or s.dtype == "f32") else torch.bfloat16
+        self.out = torch.empty((s.T, s.d), dtype=out_dtype, device="cuda")
+        self.mask = torch.zeros(max(s.T, 1), dtype=torch.int64, device="cuda")
+        self.counts = torch.zeros(64, dtype=torch.int32, device="cuda")
+
+    def forward(self, want_counts: bool = True):
+        dm.dsmoe_layer_forward(self.desc, self.x_d, self.Wr_d, self.br_d, self.W1_d, self.W2_d, self.packed,
+                               self.out, self.mask, self.counts if want_counts else None, self.ws, self.dev_status)
+        torch.cuda.synchronize()
+        assert int(self.dev_status.item()) == 0, f"device status {int(self.dev_status.item())}"
+        return self.out
+
+    # ---- oracle side
+    def oracle_scores(self):
+        return oracle.router_scores(self.x, self.Wr, self.br)
+
+    def oracle_select(self, S):
+        s = self.s
+        return oracle.select(S, s.mode, s.eps, s.eps_normalized, s.K, s.min_k)
+
+
+def check_mask_against_oracle(s: gi.LayerSpec, S: np.ndarray, mask_gpu: np.ndarray, mask_ref: np.ndarray):
+    """The GPU decided on its own fp32 scores; any decision that differs from the oracle's must sit
+    within NEAR of the boundary.  Returns (#flipped decisions, #scores within NEAR of the threshold)."""
+    diff = mask_gpu ^ mask_ref
+    flips = 0
+    near = 0
+    if s.mode == gi.MODE_THRESHOLD:
+        v = S * np.float32(s.E) if s.eps_normalized else S
+        near = int((np.abs(v.astype(np.float64) - s.eps) <= NEAR).sum())
+    for t in np.nonzero(diff)[0]:
+        for e in range(s.E):
+            if (int(diff[t]) >> e) & 1:
+                flips += 1
+                if s.mode == gi.MODE_THRESHOLD:
+                    v = float(S[t, e]) * (s.E if s.eps_normalized else 1)
+                    assert abs(v - s.eps) <= NEAR * (s.E if s.eps_normalized else 1), (t, e, v, s.eps)
+                elif s.mode == gi.MODE_TOPK:
+                    kth = np.sort(S[t])[::-1][min(s.K, s.E) - 1]
+                    assert abs(float(S[t, e]) - float(kth)) <= NEAR, (t, e)
+                else:
+                    raise AssertionError("select-all cannot differ")
+    return flips, near
+
+
+def rel_err(gpu: np.ndarray, ref: np.ndarray) -> float:
+    rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
+    return float(np.max(np.abs(gpu.astype(np.float64) - ref))) / max(rms, 1e-300)
+
+
+def layer_parity(s: gi.LayerSpec, pack: bool = True, sample: int | None = None):
+    """Runs dsmoe_layer_forward and the oracle on the same inputs; returns a dict of measurements.
+
+    ``sample`` = number of seeded tokens the oracle evaluates (None: all tokens)."""
+    L = Layer(s, pack=pack)
+    out = np_f32(L.forward())
+    mask_gpu = to_np(L.mask)[:s.T].view(np.uint64)
+    S = L.oracle_scores()
+    mask_ref, k_ref = L.oracle_select(S)
+    flips, near = check_mask_against_oracle(s, S, mask_gpu, mask_ref)
+    counts_gpu = to_np(L.counts)[:s.E]
+    counts_from_mask = np.array([int(((mask_gpu >> np.uint64(e)) & np.uint64(1)).sum()) for e in range(s.E)])
+    assert np.array_equal(counts_gpu, counts_from_mask)
+    ids = None if sample is None or sample >= s.T else gi.sample_tokens(s, sample)
+    ref = oracle.layer(L.x, L.W1, L.W2, S, mask_gpu, token_ids=ids)
+    got = out if ids is None else out[ids]
+    # the tolerance is relative to the RMS of the oracle's output over the compared tokens
+    err = rel_err(got, ref) if ref.size else 0.0
+    return dict(err=err, flips=flips, near=near, A=int(counts_gpu.sum()), layer=L, ref=ref, got=got,
+                empty_experts=int((counts_gpu == 0).sum()),
+                zero_tokens=int((mask_gpu == 0).sum()))

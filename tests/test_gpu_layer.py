@@ -1,0 +1,81 @@
+"""End-to-end parity of dsmoe_layer_forward against the CPU oracle (GPU required)."""
+import numpy as np
+import pytest
+import torch
+
+import dsmoe_inputs as gi
+import oracle
+import paper_2404_05567_b200 as dm
+from harness import TOL_BF16, TOL_F32, Layer, layer_parity, np_f32, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def test_c1_tiny_fp32_threshold_layer():
+    s = gi.spec("c1")
+    r = layer_parity(s)
+    assert r["err"] <= TOL_F32
+    frac = r["A"] / (s.T * s.E)
+    assert 0.30 <= frac <= 0.40                       # the recipe's 35 % active experts
+
+
+SMALL = [
+    dict(T=7, d=64, H=64, E=3, mode=gi.MODE_THRESHOLD, eps=0.2),
+    dict(T=129, d=128, H=72, E=33, mode=gi.MODE_TOPK, K=4),
+    dict(T=33, d=256, H=136, E=64, mode=gi.MODE_THRESHOLD, eps=0.01, zipf_s=1.1),
+    dict(T=200, d=128, H=128, E=8, mode=gi.MODE_ALL),
+    dict(T=1, d=64, H=64, E=1, mode=gi.MODE_ALL),
+    dict(T=300, d=64, H=64, E=16, mode=gi.MODE_THRESHOLD, eps=0.5),              # most tokens select nothing
+    dict(T=300, d=64, H=64, E=16, mode=gi.MODE_THRESHOLD, eps=0.5, min_k=1),
+    dict(T=64, d=64, H=64, E=2, mode=gi.MODE_TOPK, K=2, out_fp32=1),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("pack", [False, True], ids=["plain", "packed"])
+@pytest.mark.parametrize("case", SMALL, ids=[str(i) for i in range(len(SMALL))])
+def test_small_layers(case, pack, dtype):
+    if pack and dtype == "f32":
+        pytest.skip("packed weights are bf16 only")
+    s = gi.LayerSpec(f"small{SMALL.index(case)}", dtype=dtype, router_gain=6.0, **case)
+    r = layer_parity(s, pack=pack)
+    tol = TOL_F32 if dtype == "f32" else TOL_BF16
+    if dtype == "bf16" and s.out_fp32:
+        tol = TOL_BF16 / 2
+    assert r["err"] <= tol, r["err"]
+    if case.get("eps") == 0.5 and not case.get("min_k"):
+        assert r["zero_tokens"] > 0
+        out = np_f32(r["layer"].out)
+        mask = to_np(r["layer"].mask)[:s.T]
+        assert np.all(out[mask == 0] == 0.0)          # Eq. 1 with an empty selection is the zero vector
+
+
+def test_all_tokens_to_one_expert_and_empty_experts():
+    s = gi.LayerSpec("onehot", T=150, d=64, H=64, E=8, dtype="bf16", mode=gi.MODE_TOPK, K=1)
+    L = Layer(s)
+    br = np.zeros(s.E, np.float32)
+    br[5] = 50.0
+    L.br, L.br_d = br, torch.from_numpy(br).cuda()
+    out = np_f32(L.forward())
+    counts = to_np(L.counts)[:s.E]
+    assert counts.tolist() == [0, 0, 0, 0, 0, 150, 0, 0]
+    S = L.oracle_scores()
+    mask, _ = L.oracle_select(S)
+    ref = oracle.layer(L.x, L.W1, L.W2, S, mask)
+    from harness import rel_err
+    assert rel_err(out, ref) <= TOL_BF16
+
+
+def test_t0_is_a_noop():
+    desc = dm.make_desc(0, 64, 64, 4, dm.BF16)
+    dm.dsmoe_layer_forward(desc, None, None, None, None, None, None, None, None, None, None)
+
+
+def test_selection_is_reproducible_run_to_run():
+    s = gi.LayerSpec("repro", T=777, d=128, H=64, E=32, dtype="bf16", mode=gi.MODE_THRESHOLD, eps=0.03,
+                     router_gain=4.0)
+    L = Layer(s)
+    a = np_f32(L.forward()).copy()
+    m1 = to_np(L.mask).copy()
+    b = np_f32(L.forward())
+    assert np.array_equal(m1, to_np(L.mask)) and np.array_equal(a, b)
