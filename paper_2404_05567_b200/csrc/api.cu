@@ -123,7 +123,8 @@ dsmoe_status dsmoe_expert_mlp(const dsmoe_layer_desc* desc, const void* xp, cons
     if (!workspace || ws_bytes < L.total) return DSMOE_ERR_WORKSPACE;
     char* ws = static_cast<char*>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
-    if (packed) return launch_mlp_umma(*desc, xp, packed, offsets, ws + L.h, yp, dev_status, s);
+    if (packed && umma_supported(*desc)) return launch_mlp_umma(*desc, xp, packed, offsets, ws + L.h, yp, dev_status, s);
+    if (!W1 || !W2) return DSMOE_ERR_UNSUPPORTED;   // packed weights given, but this shape needs the plain path
     return launch_mlp_generic(*desc, xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h), yp, s);
 }
 
@@ -174,9 +175,11 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     float* row_gate = reinterpret_cast<float*>(ws + L.row_gate);
     int32_t* token_rows = reinterpret_cast<int32_t*>(ws + L.token_rows);
 
-    DSMOE_TRY(launch_router(p, x, Wr, br, scores, mask, k_t, s));
+    const bool fast = packed && umma_supported(p);
+    if (!fast && (!W1 || !W2)) return DSMOE_ERR_UNSUPPORTED;   // this shape needs the unpacked weights
 
-    if (packed) {
+    DSMOE_TRY(launch_router(p, x, Wr, br, scores, mask, k_t, s));
+    if (fast) {
         bool done = false;
         DSMOE_TRY(launch_layer_umma(p, x, packed, scores, mask, k_t, counts_out, out, ws, L, dev_status, s, &done));
         if (done) return DSMOE_OK;
@@ -185,7 +188,7 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     // grouped path: duplicate tokens per selected expert, run the experts, aggregate
     DSMOE_TRY(launch_finalize(p, mask, counts, offsets, chunk_prefix, counts_out, s));
     DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, ws + L.xp, s));
-    if (packed)
+    if (fast)
         DSMOE_TRY(launch_mlp_umma(p, ws + L.xp, packed, offsets, ws + L.h, ws + L.yp, dev_status, s));
     else
         DSMOE_TRY(launch_mlp_generic(p, ws + L.xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h), ws + L.yp, s));

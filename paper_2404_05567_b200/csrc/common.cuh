@@ -69,6 +69,7 @@ dsmoe_status launch_mlp_generic(const dsmoe_layer_desc& p, const void* xp, const
 
 
 // ---- mlp_umma.cu : tcgen05 / TMEM / TMA kernels on packed bf16 weights
+bool umma_supported(const dsmoe_layer_desc& p);   // bf16, d and H multiples of 64
 // Grouped expert MLPs on expert-sorted rows: h = GeLU(xp.W1[e]) (bf16, in `hbuf`), yp = h.W2[e].
 dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,
                              void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s);

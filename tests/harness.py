@@ -111,6 +111,22 @@ def rel_err(gpu: np.ndarray, ref: np.ndarray) -> float:
     return float(np.max(np.abs(gpu.astype(np.float64) - ref))) / max(rms, 1e-300)
 
 
+def rel_err_rows(gpu: np.ndarray, ref: np.ndarray) -> float:
+    """Per-token form of the same bar: max_c |gpu[t,c] - ref[t,c]| / RMS(ref[t,:]), maximised over
+    tokens.  Tokens are independent in Eq. 1, so this is the bar to use when row scales differ a lot
+    (tokens that selected 1 expert next to tokens that selected 40).  Rows whose reference is all
+    zero (no expert selected) must be exactly zero."""
+    ref = ref.astype(np.float64)
+    gpu = gpu.astype(np.float64)
+    rms = np.sqrt(np.mean(ref ** 2, axis=1))
+    zero = rms == 0
+    assert np.all(gpu[zero] == 0.0)
+    if np.all(zero):
+        return 0.0
+    e = np.max(np.abs(gpu[~zero] - ref[~zero]), axis=1) / rms[~zero]
+    return float(e.max())
+
+
 def layer_parity(s: gi.LayerSpec, pack: bool = True, sample: int | None = None):
     """Runs dsmoe_layer_forward and the oracle on the same inputs; returns a dict of measurements.
 
@@ -129,6 +145,6 @@ def layer_parity(s: gi.LayerSpec, pack: bool = True, sample: int | None = None):
     got = out if ids is None else out[ids]
     # the tolerance is relative to the RMS of the oracle's output over the compared tokens
     err = rel_err(got, ref) if ref.size else 0.0
-    return dict(err=err, flips=flips, near=near, A=int(counts_gpu.sum()), layer=L, ref=ref, got=got,
+    return dict(err=err, err_rows=rel_err_rows(got, ref) if ref.size else 0.0, flips=flips, near=near, A=int(counts_gpu.sum()), layer=L, ref=ref, got=got,
                 empty_experts=int((counts_gpu == 0).sum()),
                 zero_tokens=int((mask_gpu == 0).sum()))
