@@ -177,6 +177,17 @@ dsmoe_status dsmoe_layer_forward_host(const dsmoe_layer_desc* desc, const void* 
                                       void* out_dev, void* out_host, void* workspace,
                                       size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream);
 
+/*
+ * Measurement aid (no counterpart in the paper): with timing enabled, every tensor-core expert
+ * GEMM launch of dsmoe_expert_mlp / dsmoe_layer_forward is bracketed by a pair of CUDA events on
+ * the caller's stream.  dsmoe_timing_enable(1) creates the events once (call it outside any timed
+ * region); dsmoe_timing_last waits for the most recent call's launches and writes their durations
+ * in milliseconds, in launch order (up-projection, then down-projection), to the HOST array ms
+ * (at most n_max), setting *n to the number written.  Not thread-safe; off by default.
+ */
+dsmoe_status dsmoe_timing_enable(int on);
+dsmoe_status dsmoe_timing_last(float* ms, int n_max, int* n);
+
 #ifdef __cplusplus
 }
 #endif

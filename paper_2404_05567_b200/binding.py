@@ -22,7 +22,7 @@ SELECT_THRESHOLD, SELECT_TOPK, SELECT_ALL = 0, 1, 2
 EXPORTS = (
     "dsmoe_status_string", "dsmoe_workspace_size", "dsmoe_router", "dsmoe_select", "dsmoe_permute",
     "dsmoe_expert_mlp", "dsmoe_combine", "dsmoe_packed_size", "dsmoe_pack_weights",
-    "dsmoe_layer_forward", "dsmoe_layer_forward_host",
+    "dsmoe_layer_forward", "dsmoe_layer_forward_host", "dsmoe_timing_enable", "dsmoe_timing_last",
 )
 
 
@@ -158,3 +158,15 @@ def dsmoe_layer_forward_host(desc, x_host, x_dev, Wr, br, W1, W2, packed, out_de
                                           _ptr(workspace),
                                           ctypes.c_size_t(workspace.numel() if workspace is not None else 0),
                                           _ptr(dev_status), _stream(stream)), "dsmoe_layer_forward_host")
+
+
+def dsmoe_timing_enable(on: bool):
+    _check(lib().dsmoe_timing_enable(ctypes.c_int(1 if on else 0)), "dsmoe_timing_enable")
+
+
+def dsmoe_timing_last(n_max: int = 8):
+    """Durations (ms) of the expert-GEMM launches of the most recent call, in launch order."""
+    buf = (ctypes.c_float * n_max)()
+    n = ctypes.c_int(0)
+    _check(lib().dsmoe_timing_last(buf, ctypes.c_int(n_max), ctypes.byref(n)), "dsmoe_timing_last")
+    return [float(buf[i]) for i in range(n.value)]

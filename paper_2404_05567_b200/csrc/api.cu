@@ -42,9 +42,14 @@ WsLayout ws_layout(const dsmoe_layer_desc& p) {
     L.row_gate = take(amax * 4);
     L.token_rows = take(T * (size_t)width_of(p) * 4);
     L.xp = take(amax * p.d * es);
-    L.h = take(amax * p.H * 4);          // fp32 in the plain path, bf16 (half of it) in the tensor-core paths
+    // h: fp32 [Amax,H] in the plain path, bf16 [Amax,H] in the grouped tensor-core path, bf16 [T,E*H] in
+    // the dense and small-T paths
+    size_t h_bytes = amax * p.H * 4;
+    if (p.T <= kSmallMaxT && T * E * p.H * 2 > h_bytes) h_bytes = T * E * p.H * 2;
+    L.h = take(h_bytes);
     L.yp = take(amax * p.d * es);
-    L.partial = take((size_t)4 << 20);   // split-K partial sums of the small-T path
+    // fp32 partial sums of the small-T path: (CTA, 2 column ranges, T, 256)
+    L.partial = take(p.T <= kSmallMaxT ? (size_t)kSmallMaxCtas * 2 * T * 256 * 4 : 0);
     L.total = off;
     return L;
 }
@@ -123,6 +128,7 @@ dsmoe_status dsmoe_expert_mlp(const dsmoe_layer_desc* desc, const void* xp, cons
     if (!workspace || ws_bytes < L.total) return DSMOE_ERR_WORKSPACE;
     char* ws = static_cast<char*>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
+    timing_reset();
     if (packed && umma_supported(*desc)) return launch_mlp_umma(*desc, xp, packed, offsets, ws + L.h, yp, dev_status, s);
     if (!W1 || !W2) return DSMOE_ERR_UNSUPPORTED;   // packed weights given, but this shape needs the plain path
     return launch_mlp_generic(*desc, xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h), yp, s);
@@ -177,6 +183,7 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
 
     const bool fast = packed && umma_supported(p);
     if (!fast && (!W1 || !W2)) return DSMOE_ERR_UNSUPPORTED;   // this shape needs the unpacked weights
+    timing_reset();
 
     DSMOE_TRY(launch_router(p, x, Wr, br, scores, mask, k_t, s));
     if (fast) {
@@ -211,6 +218,13 @@ dsmoe_status dsmoe_layer_forward_host(const dsmoe_layer_desc* desc, const void* 
     DSMOE_CUDA_TRY(cudaMemcpyAsync(out_host, out_dev, n * out_es, cudaMemcpyDeviceToHost, s));
     DSMOE_CUDA_TRY(cudaStreamSynchronize(s));
     return DSMOE_OK;
+}
+
+dsmoe_status dsmoe_timing_enable(int on) { return timing_enable(on); }
+
+dsmoe_status dsmoe_timing_last(float* ms, int n_max, int* n) {
+    if (!ms || !n || n_max < 0) return DSMOE_ERR_INVALID_ARG;
+    return timing_last(ms, n_max, n);
 }
 
 }  // extern "C"

@@ -13,6 +13,8 @@ namespace dsmoe {
 
 constexpr int kMaxExperts = 64;
 constexpr int kChunk = 32;   // tokens per ballot chunk in the grouping kernels
+constexpr int kSmallMaxT = 128;      // the small-T (decode) path keeps all tokens in one 128-row MMA tile
+constexpr int kSmallMaxCtas = 192;   // upper bound on that path's grid (sizes its partial-sum buffer)
 
 #define DSMOE_CUDA_TRY(expr)                                  \
     do {                                                      \
@@ -69,6 +71,9 @@ dsmoe_status launch_mlp_generic(const dsmoe_layer_desc& p, const void* xp, const
 
 
 // ---- mlp_umma.cu : tcgen05 / TMEM / TMA kernels on packed bf16 weights
+void timing_reset();
+dsmoe_status timing_enable(int on);
+dsmoe_status timing_last(float* ms, int n_max, int* n);
 bool umma_supported(const dsmoe_layer_desc& p);   // bf16, d and H multiples of 64
 // Grouped expert MLPs on expert-sorted rows: h = GeLU(xp.W1[e]) (bf16, in `hbuf`), yp = h.W2[e].
 dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,

@@ -78,3 +78,40 @@ def test_selection_is_reproducible_run_to_run():
     m1 = to_np(L.mask).copy()
     b = np_f32(L.forward())
     assert np.array_equal(m1, to_np(L.mask)) and np.array_equal(a, b)
+
+
+# ---------------------------------------------------------------- the five benchmark workloads
+
+@pytest.mark.parametrize("T", [1, 8, 32, 128])
+def test_c2_decode_shaped_layer(T):
+    s = gi.spec("c2", T=T)
+    r = layer_parity(s)
+    assert r["err"] <= TOL_BF16, r["err"]
+    if T >= 32:
+        assert 0.25 <= r["A"] / (s.T * s.E) <= 0.45     # the recipe's 30-40 % active experts
+
+
+def test_c3_prefill_shaped_layer_topk():
+    s = gi.spec("c3")
+    r = layer_parity(s, sample=48)
+    assert r["A"] == s.T * s.K                           # top-K: exactly K experts per token
+    assert r["err"] <= TOL_BF16, r["err"]
+
+
+def test_c4_dense_forward_all_experts():
+    s = gi.spec("c4")
+    r = layer_parity(s, sample=24)
+    assert r["A"] == s.T * s.E
+    assert r["err"] <= TOL_BF16, r["err"]
+
+
+@pytest.mark.parametrize("eps", [0.0, 0.01, 0.05, 0.1, 0.2])
+def test_c5_skewed_router_threshold_sweep(eps):
+    s = gi.spec("c5", eps=eps)
+    r = layer_parity(s, sample=24 if eps == 0.0 else 128)
+    if eps == 0.0:
+        assert r["A"] == s.T * s.E                       # no score underflows to 0 in this recipe
+    if eps >= 0.1:
+        assert r["empty_experts"] > 0 or r["zero_tokens"] > 0
+    # rows differ wildly in scale here (1 to 64 experts per token): the bar is applied per token
+    assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
