@@ -103,6 +103,23 @@ dsmoe_status dsmoe_select(const dsmoe_layer_desc* desc, const float* scores, uin
                           size_t ws_bytes, dsmoe_stream stream);
 
 /*
+ * dsmoe_select without a workspace argument, for callers that cannot allocate device memory (code
+ * that runs under a framework's own allocator, plugins given only their input and output buffers,
+ * loops in which an allocation is not allowed).  The paper has no counterpart to this entry point:
+ * it computes exactly what dsmoe_select computes, with the same arguments and results, but keeps
+ * its scratch in a 512 KiB device array built into the library (held by every GPU that loads the
+ * library, until the process exits).
+ *   Limit: ceil(T/32) * E <= 131072 (e.g. T <= 65536 at E = 64, T <= 131072 at E = 32); beyond it
+ *   the call returns DSMOE_ERR_WORKSPACE and nothing is enqueued -- use dsmoe_select.
+ *   The first call on each device looks up the array's device address (with that device current);
+ *   make that first call before starting any stream capture.
+ *   It calls no allocation routine.  All calls on a device share the one array: calls whose kernels
+ *   may overlap on the GPU (different streams) race on it and must be serialised by the caller.
+ */
+dsmoe_status dsmoe_select_static(const dsmoe_layer_desc* desc, const float* scores, uint64_t* mask,
+                                 int32_t* k_t, int32_t* counts, int32_t* offsets, dsmoe_stream stream);
+
+/*
  * Grouping of tokens by expert -- the token duplication the "GPU Inference Analysis"
  * section names.  Row r in [offsets[e], offsets[e+1]) holds the token with the
  * (r - offsets[e])-th smallest index among those that selected e.

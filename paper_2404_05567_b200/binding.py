@@ -23,6 +23,7 @@ EXPORTS = (
     "dsmoe_status_string", "dsmoe_workspace_size", "dsmoe_router", "dsmoe_select", "dsmoe_permute",
     "dsmoe_expert_mlp", "dsmoe_combine", "dsmoe_packed_size", "dsmoe_pack_weights",
     "dsmoe_layer_forward", "dsmoe_layer_forward_host", "dsmoe_timing_enable", "dsmoe_timing_last",
+    "dsmoe_select_static",
 )
 
 
@@ -170,3 +171,10 @@ def dsmoe_timing_last(n_max: int = 8):
     n = ctypes.c_int(0)
     _check(lib().dsmoe_timing_last(buf, ctypes.c_int(n_max), ctypes.byref(n)), "dsmoe_timing_last")
     return [float(buf[i]) for i in range(n.value)]
+
+
+def dsmoe_select_static(desc, scores, mask, k_t, counts, offsets, stream=None):
+    """dsmoe_select for callers that cannot allocate: no workspace argument, the scratch is a fixed
+    array inside the library (limit ceil(T/32)*E <= 131072, else status 3)."""
+    _check(lib().dsmoe_select_static(ctypes.byref(desc), _ptr(scores), _ptr(mask), _ptr(k_t), _ptr(counts),
+                                     _ptr(offsets), _stream(stream)), "dsmoe_select_static")
