@@ -250,30 +250,30 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
         step(i)
         durs.append(dm.dsmoe_timing_last())
     dm.dsmoe_timing_enable(False)
-    durs = np.array(durs)                        # [n_timed, launches per step]
-    launch_ms = float(durs.mean())               # average over all launches of that kernel
+    durs = np.array(durs)                        # [n_timed, timed launches per step]
     per_step_launches = durs.shape[1]
+    launch_ms = float(durs.sum(axis=1).mean())   # time inside the dominant kernel per step
     if decode:
-        # selected experts' weights, each byte once; one launch reads W1 of them, the other W2
-        algo = n_act * s.d * s.H * 2.0
+        # selected experts' weights (W1 and W2), each byte once, all inside one launch of small_layer_kernel
+        algo = 2.0 * n_act * s.d * s.H * 2.0
         roof = dict(bound="hbm", achieved=algo / (launch_ms * 1e-3) / 1e9, peak=P["hbm"], unit="GB/s",
-                    peak_source=P["source"] + " (copy bandwidth)")
+                    peak_source=P["source"] + " (copy bandwidth)", kernel="small_layer_kernel")
     else:
-        algo = 2.0 * A * s.d * s.H           # per launch: one of the two projections
+        algo = 4.0 * A * s.d * s.H             # both projections: two launches of umma_gemm_kernel per step
         roof = dict(bound="tensor", achieved=algo / (launch_ms * 1e-3) / 1e12, peak=P["tf_sustained"],
-                    unit="TFLOP/s", peak_source=P["source"] + " (sustained bf16)")
+                    unit="TFLOP/s", peak_source=P["source"] + " (sustained bf16)", kernel="umma_gemm_kernel")
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = None
-    roof["kernel"] = "umma_gemm_kernel"
-    roof["launch_ms"] = launch_ms
+    roof["launch_ms"] = launch_ms / per_step_launches
+    roof["launch_ms_each"] = [float(v) for v in durs.mean(axis=0)]
     roof["launches_per_step"] = per_step_launches
-    roof["algorithmic_per_launch"] = algo
+    roof["algorithmic_per_launch"] = algo / per_step_launches
     # whole-step figure against the same roofline (what the layer as a whole achieves)
     step_s = ms_total * 1e-3 / steps
-    roof["step_frac"] = ((2 * algo / step_s / 1e9) if decode else (2 * algo / step_s / 1e12)) / roof["peak"]
+    roof["step_frac"] = ((algo / step_s / 1e9) if decode else (algo / step_s / 1e12)) / roof["peak"]
 
     res = dict(value=value, ms_per_step=ms_total / steps, clocks=clocks, roofline=roof, A=A, active_experts=n_act,
-               launches_per_step=(4 if decode else (3 if s.mode == gi.MODE_ALL else 7)), spec=s)
+               launches_per_step=(1 if decode else (3 if s.mode == gi.MODE_ALL else 7)), spec=s)
 
     # ---- end to end through the host-buffer entry point
     if with_e2e:

@@ -50,6 +50,7 @@ WsLayout ws_layout(const dsmoe_layer_desc& p) {
     L.yp = take(amax * p.d * es);
     // fp32 partial sums of the small-T path: (CTA, 2 column ranges, T, 256)
     L.partial = take(p.T <= kSmallMaxT ? (size_t)kSmallMaxCtas * 2 * T * 256 * 4 : 0);
+    L.sync = take(64);                   // grid-barrier counters of the small-T kernel
     L.total = off;
     return L;
 }
@@ -184,6 +185,9 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     const bool fast = packed && umma_supported(p);
     if (!fast && (!W1 || !W2)) return DSMOE_ERR_UNSUPPORTED;   // this shape needs the unpacked weights
     timing_reset();
+
+    if (fast && small_supported(p))
+        return launch_layer_small(p, x, Wr, br, packed, scores, mask, k_t, counts_out, out, ws, L, dev_status, s);
 
     DSMOE_TRY(launch_router(p, x, Wr, br, scores, mask, k_t, s));
     if (fast) {

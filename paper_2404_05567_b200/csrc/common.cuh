@@ -43,7 +43,7 @@ static inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; 
 // Byte offsets of every internal buffer inside the caller's workspace.
 struct WsLayout {
     size_t scores, mask, k_t, counts, offsets, chunk_prefix, row_token, row_gate, token_rows;
-    size_t xp, h, yp, partial, total;
+    size_t xp, h, yp, partial, sync, total;
 };
 WsLayout ws_layout(const dsmoe_layer_desc& p);
 
@@ -80,6 +80,11 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
                              void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s);
 // Whole-layer paths that need no grouping (all experts selected, or few tokens).  *done = false
 // means "not taken": the caller continues with the grouped path.
+// Whole layer for few tokens (T <= 128) in one cooperative launch, router included.
+bool small_supported(const dsmoe_layer_desc& p);
+dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
+                                const void* packed, float* scores, uint64_t* mask, int32_t* k_t, int32_t* counts_out,
+                                void* out, char* ws, const WsLayout& L, int32_t* dev_status, cudaStream_t s);
 dsmoe_status launch_layer_umma(const dsmoe_layer_desc& p, const void* x, const void* packed, const float* scores,
                                const uint64_t* mask, const int32_t* k_t, int32_t* counts_out, void* out, char* ws,
                                const WsLayout& L, int32_t* dev_status, cudaStream_t s, bool* done);

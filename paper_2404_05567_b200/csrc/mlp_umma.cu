@@ -1,5 +1,5 @@
-// Expert MLPs (Eq. 1's e(X) = GeLU(X.W1).W2) on the 5th-generation tensor cores: a persistent,
-// warp-specialised GEMM whose operands arrive by TMA into 128-byte-swizzled shared memory, whose
+// Expert MLPs (Eq. 1's e(X) = GeLU(X.W1).W2) on the 5th-generation tensor cores: persistent,
+// warp-specialised kernels whose operands arrive by TMA into 128-byte-swizzled shared memory, whose
 // products are issued by one thread with tcgen05.mma into TMEM accumulators, and whose epilogue
 // (GeLU, router gate, rounding) reads TMEM back with tcgen05.ld while the next tile's mainloop runs
 // on the other half of TMEM.
@@ -8,33 +8,36 @@
 //   warp 1      MMA issuer           (one lane); owns the TMEM allocation
 //   warps 2..5  epilogue             (warp w reads TMEM lanes 32*(w%4) .. +31)
 //
-// Three tilings share the kernel:
+// umma_gemm_kernel, three tilings:
 //   GROUPED     rows sorted by expert (sparse inference): tile = (expert, 128 rows, <=256 columns)
 //   DENSE_UP    every expert on every token (dense forward): h[t, e*H + j] = S[t,e] * GeLU(x[t].W1[e][:,j])
 //   DENSE_DOWN  out[t,:] = sum over (e,j) of that h times W2[e][j,:] -- the router-weighted sum of
 //               Eq. 1 folded into the reduction dimension, so no grouping and no aggregation pass
-//   SMALL_UP / SMALL_DOWN   the same two products for a handful of tokens (decode), where time is
-//               the reading of the selected experts' weights: only experts that some token selected
-//               are streamed, each weight byte once, in contiguous slabs split evenly over the
-//               CTAs (16 weight rows for the up-projection, one 64-wide reduction block for the
-//               down-projection, whose partial sums a short fix-up kernel adds in a fixed order)
+// small_layer_kernel: the whole layer for a handful of tokens (decode) in one cooperative launch.
 #include "common.cuh"
+#include "router_device.cuh"
 #include "umma.cuh"
 
 namespace dsmoe {
 
 namespace {
 
-constexpr int BM = 128, BK = 64, BN = 256, STAGES = 4;
+constexpr int BM = 128, BK = 64, BN = 256, STAGES = 4, MAX_STAGES = 16;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
-constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024;
+constexpr int RING_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);   // operand ring: 4 x 48 KB, or more, smaller slots
+constexpr int SHARED_BYTES = 3072;                                     // barriers and small tables (struct Shared)
+constexpr int STG_LD = 36;                                             // floats per row of the epilogue staging tile
+constexpr int STG_BYTES = BM * STG_LD * 4;
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)RING_BYTES + SHARED_BYTES + STG_BYTES;
 
-enum { GEMM_GROUPED = 0, GEMM_DENSE_UP = 1, GEMM_DENSE_DOWN = 2, GEMM_SMALL_UP = 3, GEMM_SMALL_DOWN = 4 };
-enum { EPI_GELU = 0, EPI_STORE = 1, EPI_PARTIAL = 2 };
-constexpr int kUpUnit = 16;          // weight rows per work unit of SMALL_UP
+enum { GEMM_GROUPED = 0, GEMM_DENSE_UP = 1, GEMM_DENSE_DOWN = 2 };
+enum { EPI_GELU = 0, EPI_STORE = 1 };
+constexpr int kUpUnit = 16;          // small-T up-projection: weight rows per work unit
+constexpr int kUpTileUnits = 16;     // ... and units per tile (256 rows)
+constexpr int kFixBatch = 24;        // partial tiles a fix-up thread loads at once
 
 struct GemmParams {
     int mode, epi;
@@ -48,50 +51,47 @@ struct GemmParams {
     long long ld_out;        // elements
     int out_f32;
     int32_t* dev_status;
-    const uint64_t* mask;    // small-T modes: selection words of the T tokens
-    int a_box_rows;          // rows per TMA box of A (128, or T rounded up to 8 in the small-T modes)
-    int b_box_rows;          // rows per TMA box of B (256, or 16 in SMALL_UP)
+};
+
+// Tensor maps of one packed weight tensor [E, n, k] with boxes of 16, 32, 64, 128 and 256 rows: a tile of
+// any width (a multiple of 16 rows) is fetched with at most five copies, largest first.
+struct BMaps {
+    CUtensorMap m[5];
 };
 
 struct Tile {
     int row0, rows_valid, e, n0, bn, nk, out_col0;
-    int kstart, seg;         // SMALL_DOWN: first global reduction block, partial-sum slot
 };
 
 struct Shared {
-    uint64_t full[STAGES], empty[STAGES], tfull[2], tempty[2];
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
     int bad_offsets;
+    int n_stages, slot_bytes, a_bytes;   // ring geometry (small_layer_kernel)
     int tile_prefix[kMaxExperts + 1];
     int seg0[kMaxExperts], seg1[kMaxExperts];
-    unsigned long long active_mask;   // small-T modes: experts selected by at least one token
+    unsigned long long active_mask;      // experts selected by at least one token
     int n_act;
     int active[kMaxExperts];
+    float gate_s[BM], gate2_s[BM];
 };
+static_assert(sizeof(Shared) <= SHARED_BYTES, "Shared must fit its slot");
 
-// Walks the tiles of one CTA.  The large-T tilings stride a global tile index over the grid; the
-// small-T tilings cut this CTA's contiguous range of work units into tiles.
-struct TileIter {
-    int id, u0, u1, r_first;
+__device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f)); }
 
-    __device__ __forceinline__ void init(const GemmParams& P, const Shared& sh) {
-        id = blockIdx.x;
-        if (P.mode == GEMM_SMALL_UP || P.mode == GEMM_SMALL_DOWN) {
-            const int kbpe = P.k_per_expert / BK;
-            const int total = P.mode == GEMM_SMALL_UP
-                                  ? sh.n_act * (P.n_per_expert / kUpUnit)
-                                  : ((P.n_per_expert + BN - 1) / BN) * sh.n_act * kbpe;
-            const int per = (total + (int)gridDim.x - 1) / (int)gridDim.x;
-            u0 = min(total, (int)blockIdx.x * per);
-            u1 = min(total, u0 + per);
-            const int U = sh.n_act * kbpe;
-            r_first = (P.mode == GEMM_SMALL_DOWN && U > 0) ? u0 / U : 0;
+// Weight rows [n0, n0 + rows) of expert e, reduction block starting at k: power-of-two boxes, largest first.
+__device__ __forceinline__ void load_weight_rows(const BMaps* maps, uint32_t dst, uint32_t bar, int k, int n0, int rows,
+                                                 int e) {
+    int done = 0;
+#pragma unroll
+    for (int lvl = 4; lvl >= 0; --lvl) {
+        if ((rows - done) >= (16 << lvl)) {
+            ptx::tma_load_3d(dst + done * (BK * 2), &maps->m[lvl], bar, k, n0 + done, e);
+            done += 16 << lvl;
         }
     }
-
-    __device__ __forceinline__ bool next(const GemmParams& P, const Shared& sh, Tile& t);
-};
+}
 
 __device__ __forceinline__ int total_tiles(const GemmParams& P, const Shared& sh) {
     const int ntn = (P.n_per_expert + BN - 1) / BN;
@@ -100,45 +100,9 @@ __device__ __forceinline__ int total_tiles(const GemmParams& P, const Shared& sh
     return P.mode == GEMM_DENSE_UP ? mt * ntn * P.E : mt * ntn;
 }
 
-__device__ __forceinline__ bool TileIter::next(const GemmParams& P, const Shared& sh, Tile& t) {
+__device__ __forceinline__ Tile decode_tile(const GemmParams& P, const Shared& sh, int id) {
+    Tile t;
     const int kbpe = P.k_per_expert / BK;
-    t.kstart = 0;
-    t.seg = 0;
-    if (P.mode == GEMM_SMALL_UP) {
-        // units of 16 weight rows over the selected experts, concatenated; a tile stays inside one expert
-        if (u0 >= u1) return false;
-        const int upe = P.n_per_expert / kUpUnit;
-        const int ei = u0 / upe, in_e = u0 % upe;
-        const int len = min(min(u1 - u0, upe - in_e), BN / kUpUnit);
-        t.e = sh.active[ei];
-        t.row0 = 0;
-        t.rows_valid = P.rows;
-        t.n0 = in_e * kUpUnit;
-        t.bn = len * kUpUnit;
-        t.nk = kbpe;
-        t.out_col0 = t.e * P.n_per_expert + t.n0;
-        u0 += len;
-        return true;
-    }
-    if (P.mode == GEMM_SMALL_DOWN) {
-        // units = (256-column range, selected expert, 64-wide reduction block); a tile stays inside one range
-        if (u0 >= u1) return false;
-        const int U = sh.n_act * kbpe;
-        const int r = u0 / U, start = u0 % U;
-        const int len = min(u1 - u0, U - start);
-        t.e = 0;
-        t.row0 = 0;
-        t.rows_valid = P.rows;
-        t.n0 = r * BN;
-        t.bn = min(BN, P.n_per_expert - t.n0);
-        t.nk = len;
-        t.kstart = start;
-        t.seg = r - r_first;
-        t.out_col0 = 0;
-        u0 += len;
-        return true;
-    }
-    if (id >= total_tiles(P, sh)) return false;
     if (P.mode == GEMM_GROUPED) {
         int e = 0;
         while (e + 1 < P.E && id >= sh.tile_prefix[e + 1]) ++e;
@@ -171,22 +135,18 @@ __device__ __forceinline__ bool TileIter::next(const GemmParams& P, const Shared
         }
     }
     t.bn = min(BN, P.n_per_expert - t.n0);
-    id += gridDim.x;
-    return true;
+    return t;
 }
 
-__device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f)); }
-
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams P) {
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ BMaps tmB, const GemmParams P) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;             // 128-byte swizzle wants 1024-byte aligned tiles
     const uint32_t smA = base, smB = base + STAGES * A_STAGE_BYTES;
-    Shared& sh = *reinterpret_cast<Shared*>(smem_raw + (base - raw) + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+    Shared& sh = *reinterpret_cast<Shared*>(smem_raw + (base - raw) + RING_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool small = P.mode == GEMM_SMALL_UP || P.mode == GEMM_SMALL_DOWN;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -199,10 +159,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         sh.abort_flag = 0;
         sh.bad_offsets = 0;
-        sh.active_mask = 0ull;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&tmA);
-        ptx::prefetch_tensormap(&tmB);
+        for (int i = 2; i < 5; ++i) ptx::prefetch_tensormap(&tmB.m[i]);
     }
     if (P.mode == GEMM_GROUPED && threadIdx.x < P.E) {
         // segments as given, clamped so that a corrupt offsets array cannot send a tile out of range
@@ -216,7 +175,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         sh.seg1[e] = s1;
     }
     __syncthreads();
-    if (small && threadIdx.x < P.rows) atomicOr(&sh.active_mask, (unsigned long long)P.mask[threadIdx.x]);
     if (P.mode == GEMM_GROUPED && threadIdx.x == 0) {
         const int ntn = (P.n_per_expert + BN - 1) / BN;
         int run = 0;
@@ -233,16 +191,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
-    if (small && threadIdx.x == 0) {
-        unsigned long long m = sh.active_mask;
-        if (P.E < 64) m &= (1ull << P.E) - 1ull;
-        int n = 0;
-        for (int e = 0; e < P.E; ++e)
-            if ((m >> e) & 1ull) sh.active[n++] = e;
-        sh.n_act = n;
-    }
-    if (small) __syncthreads();
     const uint32_t tmem_base = sh.tmem_base;
+    const int ntiles = total_tiles(P, sh);
     const int kbpe = P.k_per_expert / BK;
 
     if (warp == 0) {
@@ -251,26 +201,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int s = 0;
             uint32_t ph = 0;
             bool alive = true;
-            const uint32_t a_bytes = (uint32_t)P.a_box_rows * BK * 2;
-            TileIter it;
-            it.init(P, sh);
-            Tile t;
-            while (alive && it.next(P, sh, t)) {
-                const int b_boxes = (t.bn + P.b_box_rows - 1) / P.b_box_rows;
-                const uint32_t b_box_bytes = (uint32_t)P.b_box_rows * BK * 2;
+            for (int id = blockIdx.x; id < ntiles && alive; id += gridDim.x) {
+                const Tile t = decode_tile(P, sh, id);
                 for (int i = 0; i < t.nk; ++i) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
                         alive = false;
                         break;
                     }
                     const uint32_t bar = ptx::smem_u32(&sh.full[s]);
-                    ptx::mbar_expect_tx(bar, a_bytes + b_boxes * b_box_bytes);
+                    ptx::mbar_expect_tx(bar, A_STAGE_BYTES + (uint32_t)t.bn * BK * 2);
                     int a_col, b_e, b_k;
-                    if (P.mode == GEMM_DENSE_DOWN || P.mode == GEMM_SMALL_DOWN) {
-                        const int g = t.kstart + i;
-                        const int ei = g / kbpe;
-                        b_e = P.mode == GEMM_SMALL_DOWN ? sh.active[ei] : ei;
-                        b_k = (g % kbpe) * BK;
+                    if (P.mode == GEMM_DENSE_DOWN) {
+                        b_e = i / kbpe;
+                        b_k = (i % kbpe) * BK;
                         a_col = b_e * P.k_per_expert + b_k;
                     } else {
                         b_e = t.e;
@@ -278,9 +221,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         a_col = b_k;
                     }
                     ptx::tma_load_2d(smA + s * A_STAGE_BYTES, &tmA, bar, a_col, t.row0);
-                    for (int b = 0; b < b_boxes; ++b)
-                        ptx::tma_load_3d(smB + s * B_STAGE_BYTES + b * b_box_bytes, &tmB, bar, b_k,
-                                         t.n0 + b * P.b_box_rows, b_e);
+                    load_weight_rows(&tmB, smB + s * B_STAGE_BYTES, bar, b_k, t.n0, t.bn, b_e);
                     if (++s == STAGES) {
                         s = 0;
                         ph ^= 1u;
@@ -300,10 +241,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int s = 0, acc = 0;
             uint32_t ph = 0, aph = 0;
             bool alive = true;
-            TileIter it;
-            it.init(P, sh);
-            Tile t;
-            while (alive && it.next(P, sh, t)) {
+            for (int id = blockIdx.x; id < ntiles && alive; id += gridDim.x) {
+                const Tile t = decode_tile(P, sh, id);
                 if (!ptx::mbar_wait(ptx::smem_u32(&sh.tempty[acc]), aph ^ 1u, &sh.abort_flag)) break;
                 ptx::tc_fence_after();
                 const uint32_t idesc = ptx::make_idesc_bf16(BM, (uint32_t)t.bn);
@@ -338,31 +277,25 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int q = warp & 3;
         int acc = 0;
         uint32_t aph = 0;
-        TileIter it;
-        it.init(P, sh);
-        Tile t;
-        while (it.next(P, sh, t)) {
-            if (!ptx::mbar_wait(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag)) break;
+        for (int id = blockIdx.x; id < ntiles; id += gridDim.x) {
+            const Tile t = decode_tile(P, sh, id);
+            // the TMEM reads below are warp-collective: the warp leaves as one
+            if (__any_sync(0xffffffffu, !ptx::mbar_wait(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag))) break;
             ptx::tc_fence_after();
             const int row = q * 32 + lane;
             const bool valid = row < t.rows_valid;
             const long long grow = (long long)t.row0 + row;
             float g = 1.f;
-            if (P.gate && valid) {
-                g = P.gate[grow * P.E + t.e];
-                if (small && !((P.mask[grow] >> t.e) & 1ull)) g = 0.f;   // expert not selected by this token
-            }
+            if (P.gate && valid) g = P.gate[grow * P.E + t.e];
             const uint32_t taddr = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
-            // warps whose 32 TMEM lanes hold no valid row skip the read-back altogether
-            const bool warp_has_rows = q * 32 < t.rows_valid;
+            const bool warp_has_rows = q * 32 < t.rows_valid;   // warps without a valid row skip the read-back
             for (int c = 0; warp_has_rows && c < t.bn; c += 32) {
                 uint32_t r[32];
                 ptx::tmem_ld32(taddr + (uint32_t)c, r);
                 ptx::tmem_ld_wait();
                 if (!valid) continue;
-                const int ncol = min(32, t.bn - c);   // 16 or 32 (bn is a multiple of 16)
+                const long long o = grow * P.ld_out + t.out_col0 + c;
                 if (P.epi == EPI_GELU) {
-                    const long long o = grow * P.ld_out + t.out_col0 + c;
                     uint4 pk[4];
                     __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
 #pragma unroll
@@ -371,28 +304,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                                       g * gelu_erf(__uint_as_float(r[2 * j + 1])));
                     uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) + o);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        if (j * 8 < ncol) dst[j] = pk[j];
-                } else if (P.epi == EPI_PARTIAL) {
-                    // fp32 partial sums of this CTA's share of the reduction: slot (cta, seg), row, 256 columns
-                    float* dstf = static_cast<float*>(P.out) +
-                                  (((long long)blockIdx.x * 2 + t.seg) * P.rows + grow) * BN + c;
-                    float4* dst = reinterpret_cast<float4*>(dstf);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        if (j * 4 < ncol)
-                            dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                                 __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                    for (int j = 0; j < 4; ++j) dst[j] = pk[j];
                 } else if (P.out_f32) {
-                    const long long o = grow * P.ld_out + t.out_col0 + c;
                     float4* dst = reinterpret_cast<float4*>(static_cast<float*>(P.out) + o);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        if (j * 4 < ncol)
-                            dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                                 __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                        dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                             __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
                 } else {
-                    const long long o = grow * P.ld_out + t.out_col0 + c;
                     uint4 pk[4];
                     __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
 #pragma unroll
@@ -400,8 +319,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         hv[j] = __floats2bfloat162_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
                     uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) + o);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        if (j * 8 < ncol) dst[j] = pk[j];
+                    for (int j = 0; j < 4; ++j) dst[j] = pk[j];
                 }
             }
             ptx::tc_fence_before();
@@ -427,35 +345,603 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 }
 
-// Adds the partial sums of SMALL_DOWN in a fixed order (ascending CTA) and writes out[T,d].
-// Grid (column ranges of 256, T); the partition arithmetic mirrors TileIter::init / next.
-__global__ void __launch_bounds__(BN) small_fixup_kernel(const float* __restrict__ partial, const uint64_t* __restrict__ mask,
-                                                         void* __restrict__ out, int T, int d, int E, int kbpe, int G,
-                                                         int out_f32) {
-    __shared__ unsigned long long act;
-    if (threadIdx.x == 0) act = 0ull;
-    __syncthreads();
-    if (threadIdx.x < T) atomicOr(&act, (unsigned long long)mask[threadIdx.x]);
-    __syncthreads();
-    unsigned long long m = act;
-    if (E < 64) m &= (1ull << E) - 1ull;
-    const int U = __popcll(m) * kbpe;
-    const int r = blockIdx.x, t = blockIdx.y;
-    const int c = r * BN + threadIdx.x;
-    if (c >= d) return;
-    float sum = 0.f;
-    if (U > 0) {
-        const int nr = (d + BN - 1) / BN;
-        const int total = nr * U;
-        const int per = (total + G - 1) / G;
-        const int i0 = (r * U) / per, i1 = ((r + 1) * U - 1) / per;
-        for (int i = i0; i <= i1; ++i) {
-            const int seg = r - (i * per) / U;
-            sum += partial[(((long long)i * 2 + seg) * T + t) * BN + threadIdx.x];
+// ---------------------------------------------------------------- whole small-T layer in one launch
+//
+// Decode-sized calls are bound by reading the selected experts' weights once, and a 134 MB phase is
+// too short to amortise a kernel launch, a prologue and a drained pipeline (about a quarter of its
+// time).  So the whole layer runs as ONE cooperative launch of one CTA per SM.  All T <= 128 tokens
+// ride in the one 128-row MMA tile, so the layer is evaluated in its gated dense form restricted to
+// the experts that at least one token selected -- no grouping, no aggregation pass:
+//
+//   router   the reduction over d of every token cut into slices, one CTA each  -> grid barrier
+//            CTA t adds token t's slices: softmax, selection                    -> grid barrier
+//   up       hg[t,(e,j)] = [e in sel(t)] S[t,e] GeLU(x[t].W1[e][:,j]); a CTA takes a contiguous run of
+//            16-row units of the selected experts' W1 (a tile may cross one expert boundary) -> grid barrier
+//   down     out = hg . W2cat as stream-K: units of (256 output columns, expert, 64-wide reduction
+//            block); fp32 partial tiles, at most two per CTA                    -> grid barrier
+//   fix-up   every CTA adds the partial tiles of its share of out[T,d] in ascending-CTA order
+//
+// The operand ring keeps running across the up/down barrier: the producer prefetches the first W2
+// tiles (which do not depend on hg) while other CTAs finish, and adds the hg tiles once the barrier
+// has passed.  Every wait, on an mbarrier or on a grid barrier, is bounded.
+
+struct SmallParams {
+    int T, d, H, E, t_pad;
+    const __nv_bfloat16* x;
+    const float* Wr;
+    const float* br;
+    SelParams sel;
+    float* scores;
+    uint64_t* mask;
+    int32_t* k_t;
+    int32_t* counts_out;     // nullable
+    __nv_bfloat16* hg;       // [T, E*H]
+    float* partial;          // [grid][2][T][256]; doubles as the router's slice buffer
+    void* out;
+    int out_f32;
+    int* sync;               // 8 ints, zero at launch: four barrier counters [0..3] and an abort flag [4]
+    int32_t* dev_status;
+};
+
+// One thread per CTA arrives at grid barrier `idx`; grid_wait spins (bounded) until all CTAs have.
+__device__ __forceinline__ void grid_arrive(int* sync, int idx) {
+    __threadfence();
+    atomicAdd(sync + idx, 1);
+}
+__device__ __forceinline__ bool grid_wait(int* sync, int idx, int target, volatile int* abort_flag) {
+    const uint64_t t0 = ptx::globaltimer_ns();
+    for (uint32_t spin = 0;; ++spin) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(sync + idx) : "memory");
+        if (v >= target) return true;
+        if ((spin & 0x3f) == 0x3f) {
+            int ab;
+            asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(ab) : "l"(sync + 4) : "memory");
+            if (ab || *abort_flag || ptx::globaltimer_ns() - t0 > ptx::kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(sync + 4, 1);
+                return false;
+            }
         }
     }
-    if (out_f32) static_cast<float*>(out)[(long long)t * d + c] = sum;
-    else static_cast<__nv_bfloat16*>(out)[(long long)t * d + c] = __float2bfloat16_rn(sum);
+}
+
+struct SmallTile {
+    int phase;                       // 0 up, 1 down
+    int e, n0, bn, bn1, e2, nk;      // up: columns [0,bn1) are rows n0.. of expert e, [bn1,bn) rows 0.. of expert e2
+    int out_col0, out_col0_2;
+    int kstart, seg;                 // down: first global reduction block, partial-sum slot
+};
+
+struct SmallIter {
+    int phase, u0, u1, r_first, down_u0, down_u1;
+
+    __device__ __forceinline__ void init(const SmallParams& P, int n_act) {
+        const int G = gridDim.x;
+        {
+            const int total = n_act * (P.H / kUpUnit);
+            const int per = (total + G - 1) / G;
+            u0 = min(total, (int)blockIdx.x * per);
+            u1 = min(total, u0 + per);
+        }
+        {
+            const int U = n_act * (P.H / BK);
+            const int total = ((P.d + BN - 1) / BN) * U;
+            const int per = (total + G - 1) / G;
+            down_u0 = min(total, (int)blockIdx.x * per);
+            down_u1 = min(total, down_u0 + per);
+            r_first = U > 0 ? down_u0 / U : 0;
+        }
+        phase = 0;
+    }
+
+    __device__ __forceinline__ bool next(const SmallParams& P, const int* active, int n_act, SmallTile& t) {
+        if (phase == 0 && u0 >= u1) {
+            phase = 1;
+            u0 = down_u0;
+            u1 = down_u1;
+        }
+        if (u0 >= u1) return false;
+        t.phase = phase;
+        t.e2 = 0;
+        t.out_col0_2 = 0;
+        t.kstart = 0;
+        t.seg = 0;
+        if (phase == 0) {
+            const int upe = P.H / kUpUnit;
+            const int ei = u0 / upe, in_e = u0 % upe;
+            int len = min(u1 - u0, kUpTileUnits);
+            const int len1 = min(len, upe - in_e);
+            const int len2 = min(len - len1, upe);
+            len = len1 + len2;
+            t.e = active[ei];
+            t.n0 = in_e * kUpUnit;
+            t.bn1 = len1 * kUpUnit;
+            t.bn = len * kUpUnit;
+            t.nk = P.d / BK;
+            t.out_col0 = t.e * P.H + t.n0;
+            if (len2 > 0) {
+                t.e2 = active[ei + 1];
+                t.out_col0_2 = t.e2 * P.H;
+            }
+            u0 += len;
+        } else {
+            const int U = n_act * (P.H / BK);
+            const int r = u0 / U, start = u0 % U;
+            const int len = min(u1 - u0, U - start);
+            t.e = 0;
+            t.n0 = r * BN;
+            t.bn = min(BN, P.d - t.n0);
+            t.bn1 = t.bn;
+            t.nk = len;
+            t.kstart = start;
+            t.seg = r - r_first;
+            t.out_col0 = 0;
+            u0 += len;
+        }
+        return true;
+    }
+};
+
+// One ring slot's loads.  what: bit 0 = the token operand (x or hg), bit 1 = the weight rows.
+__device__ __forceinline__ void small_issue(const SmallParams& P, const CUtensorMap* tmX, const BMaps* tmW1,
+                                            const CUtensorMap* tmHg, const BMaps* tmW2, const int* active,
+                                            const SmallTile& t, int i, uint32_t slotA, uint32_t slotB, uint32_t bar,
+                                            int what) {
+    if (t.phase == 0) {
+        if (what & 1) ptx::tma_load_2d(slotA, tmX, bar, i * BK, 0);
+        if (what & 2) {
+            load_weight_rows(tmW1, slotB, bar, i * BK, t.n0, t.bn1, t.e);
+            if (t.bn > t.bn1) load_weight_rows(tmW1, slotB + t.bn1 * (BK * 2), bar, i * BK, 0, t.bn - t.bn1, t.e2);
+        }
+    } else {
+        const int kbpe = P.H / BK;
+        const int g = t.kstart + i;
+        const int e = active[g / kbpe], kb = g % kbpe;
+        if (what & 1) ptx::tma_load_2d(slotA, tmHg, bar, e * P.H + kb * BK, 0);
+        if (what & 2) load_weight_rows(tmW2, slotB, bar, kb * BK, t.n0, t.bn, e);
+    }
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ BMaps tmW1,
+                   const __grid_constant__ CUtensorMap tmHg, const __grid_constant__ BMaps tmW2, const SmallParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = ptx::smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    Shared& sh = *reinterpret_cast<Shared*>(smem_raw + (base - raw) + RING_BYTES);
+    float* stg = reinterpret_cast<float*>(smem_raw + (base - raw) + RING_BYTES + SHARED_BYTES);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = gridDim.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_STAGES; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&sh.full[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh.empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(ptx::smem_u32(&sh.tfull[a]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh.tempty[a]), 4);
+        }
+        sh.abort_flag = 0;
+        sh.active_mask = 0ull;
+        ptx::fence_barrier_init();
+        ptx::prefetch_tensormap(&tmX);
+        ptx::prefetch_tensormap(&tmHg);
+        for (int i = 0; i < 5; ++i) {
+            ptx::prefetch_tensormap(&tmW1.m[i]);
+            ptx::prefetch_tensormap(&tmW2.m[i]);
+        }
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+
+    // ------------------------------------------------------------ router, step 1
+    // The reduction over d of every token is cut into KS slices, one CTA per (token, slice); a thread takes
+    // whole rows of Wr (E contiguous floats), two rows at a time, so many independent loads are in flight.
+    const int KS = max(1, min(16, G / P.T));
+    if ((int)blockIdx.x < P.T * KS) {
+        const int t = blockIdx.x / KS, sl = blockIdx.x % KS, E = P.E;
+        const int klen = (P.d + KS - 1) / KS, kbeg = sl * klen, kend = min(P.d, kbeg + klen);
+        const __nv_bfloat16* __restrict__ xr = P.x + (size_t)t * P.d;
+        const float* __restrict__ Wr = P.Wr;
+        float acc[kMaxExperts];
+#pragma unroll
+        for (int e = 0; e < kMaxExperts; ++e) acc[e] = 0.f;
+        if ((E & 3) == 0) {
+            for (int k0 = kbeg + (int)threadIdx.x; k0 < kend; k0 += 2 * NUM_THREADS) {
+                const int k1 = k0 + NUM_THREADS;
+                const bool has1 = k1 < kend;
+                const float4* p0 = reinterpret_cast<const float4*>(Wr + (size_t)k0 * E);
+                const float4* p1 = reinterpret_cast<const float4*>(Wr + (size_t)(has1 ? k1 : k0) * E);
+                float4 w0[kMaxExperts / 4], w1[kMaxExperts / 4];
+#pragma unroll
+                for (int e4 = 0; e4 < kMaxExperts / 4; ++e4)
+                    if (e4 * 4 < E) {
+                        w0[e4] = __ldg(p0 + e4);
+                        w1[e4] = __ldg(p1 + e4);
+                    }
+                const float x0 = __bfloat162float(xr[k0]);
+                const float x1 = has1 ? __bfloat162float(xr[k1]) : 0.f;
+#pragma unroll
+                for (int e4 = 0; e4 < kMaxExperts / 4; ++e4)
+                    if (e4 * 4 < E) {
+                        acc[e4 * 4 + 0] = fmaf(x1, w1[e4].x, fmaf(x0, w0[e4].x, acc[e4 * 4 + 0]));
+                        acc[e4 * 4 + 1] = fmaf(x1, w1[e4].y, fmaf(x0, w0[e4].y, acc[e4 * 4 + 1]));
+                        acc[e4 * 4 + 2] = fmaf(x1, w1[e4].z, fmaf(x0, w0[e4].z, acc[e4 * 4 + 2]));
+                        acc[e4 * 4 + 3] = fmaf(x1, w1[e4].w, fmaf(x0, w0[e4].w, acc[e4 * 4 + 3]));
+                    }
+            }
+        } else {
+            for (int k = kbeg + (int)threadIdx.x; k < kend; k += NUM_THREADS) {
+                const float xv = __bfloat162float(xr[k]);
+#pragma unroll
+                for (int e = 0; e < kMaxExperts; ++e)
+                    if (e < E) acc[e] = fmaf(xv, __ldg(Wr + (size_t)k * E + e), acc[e]);
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < kMaxExperts; ++e) {
+            if (e < E) {
+                const float v = warp_sum(acc[e]);
+                if (lane == 0) stg[warp * kMaxExperts + e] = v;
+            }
+        }
+        __syncthreads();
+        if ((int)threadIdx.x < E) {
+            float v = 0.f;
+#pragma unroll
+            for (int w = 0; w < NUM_THREADS / 32; ++w) v += stg[w * kMaxExperts + threadIdx.x];
+            P.partial[((size_t)t * KS + sl) * kMaxExperts + threadIdx.x] = v;   // free until the down-projection
+        }
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    if (threadIdx.x == 0) {
+        grid_arrive(P.sync, 0);
+        grid_wait(P.sync, 0, G, &sh.abort_flag);
+    }
+    __syncthreads();
+    // ------------------------------------------------------------ router, step 2
+    // CTA t adds the slices of token t in a fixed order; softmax and selection in one warp
+    if ((int)blockIdx.x < P.T && warp == 0 && !sh.abort_flag) {
+        const int t = blockIdx.x, E = P.E;
+        const bool v_lo = lane < E, v_hi = lane + 32 < E;
+        float l_lo = (P.br && v_lo) ? P.br[lane] : 0.f, l_hi = (P.br && v_hi) ? P.br[lane + 32] : 0.f;
+        for (int sl = 0; sl < KS; ++sl) {
+            const float* pl = P.partial + ((size_t)t * KS + sl) * kMaxExperts;
+            if (v_lo) l_lo += __ldcg(pl + lane);
+            if (v_hi) l_hi += __ldcg(pl + lane + 32);
+        }
+        softmax_select_store(l_lo, l_hi, t, P.sel, lane, P.scores, P.mask, P.k_t);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        grid_arrive(P.sync, 3);
+        grid_wait(P.sync, 3, G, &sh.abort_flag);
+    }
+    __syncthreads();
+    // every CTA derives the set of selected experts from the T selection words
+    if ((int)threadIdx.x < P.T) {
+        unsigned long long m;
+        asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(m) : "l"(P.mask + threadIdx.x) : "memory");
+        atomicOr(&sh.active_mask, m);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long m = sh.active_mask;
+        if (P.E < 64) m &= (1ull << P.E) - 1ull;
+        int n = 0;
+        for (int e = 0; e < P.E; ++e)
+            if ((m >> e) & 1ull) sh.active[n++] = e;
+        sh.n_act = n;
+        // ring geometry: a slot holds the tokens' 64-wide block and up to 256 weight rows
+        sh.a_bytes = P.t_pad * BK * 2;
+        sh.slot_bytes = sh.a_bytes + B_STAGE_BYTES;
+        sh.n_stages = min(MAX_STAGES, RING_BYTES / sh.slot_bytes);
+    }
+    __syncthreads();
+    const uint32_t tmem_base = sh.tmem_base;
+    const int n_act = sh.n_act, n_stages = sh.n_stages;
+    const uint32_t slot_bytes = (uint32_t)sh.slot_bytes, a_bytes = (uint32_t)sh.a_bytes;
+    const uint32_t smA = base, smB = base + a_bytes;
+    const bool aborted_early = sh.abort_flag != 0;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0 && !aborted_early) {
+            int s = 0;
+            uint32_t ph = 0;
+            bool alive = true;
+            SmallIter it;
+            it.init(P, n_act);
+            SmallTile t;
+            bool have = it.next(P, sh.active, n_act, t);
+            // up-projection
+            while (alive && have && t.phase == 0) {
+                for (int i = 0; i < t.nk; ++i) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    const uint32_t bar = ptx::smem_u32(&sh.full[s]);
+                    ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
+                    small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, sh.active, t, i, smA + s * slot_bytes, smB + s * slot_bytes, bar, 3);
+                    if (++s == n_stages) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
+                }
+                have = it.next(P, sh.active, n_act, t);
+            }
+            // down-projection: weight tiles first, for as many slots as the ring has; their hg tiles follow
+            // once every CTA has finished writing hg
+            SmallTile pend_t[MAX_STAGES];
+            int pend_i[MAX_STAGES], pend_s[MAX_STAGES];
+            int npend = 0, i_cur = 0;
+            while (alive && have && npend < n_stages) {
+                if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
+                    alive = false;
+                    break;
+                }
+                const uint32_t bar = ptx::smem_u32(&sh.full[s]);
+                ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
+                small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, sh.active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 2);
+                pend_t[npend] = t;
+                pend_i[npend] = i_cur;
+                pend_s[npend] = s;
+                ++npend;
+                if (++s == n_stages) {
+                    s = 0;
+                    ph ^= 1u;
+                }
+                if (++i_cur == t.nk) {
+                    i_cur = 0;
+                    have = it.next(P, sh.active, n_act, t);
+                }
+            }
+            if (alive && !grid_wait(P.sync, 1, G, &sh.abort_flag)) alive = false;
+            asm volatile("fence.proxy.async;" ::: "memory");   // hg was written through the generic proxy, TMA reads it
+            for (int j = 0; alive && j < npend; ++j)
+                small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, sh.active, pend_t[j], pend_i[j], smA + pend_s[j] * slot_bytes,
+                            smB + pend_s[j] * slot_bytes, ptx::smem_u32(&sh.full[pend_s[j]]), 1);
+            while (alive && have) {
+                for (; i_cur < t.nk; ++i_cur) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    const uint32_t bar = ptx::smem_u32(&sh.full[s]);
+                    ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
+                    small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, sh.active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 3);
+                    if (++s == n_stages) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
+                }
+                if (!alive) break;
+                i_cur = 0;
+                have = it.next(P, sh.active, n_act, t);
+            }
+            if (!alive) {
+                const uint64_t t0 = ptx::globaltimer_ns();   // copies already issued still land in this CTA's smem
+                while (ptx::globaltimer_ns() - t0 < 200000ull) {
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0 && !aborted_early) {
+            int s = 0, acc = 0;
+            uint32_t ph = 0, aph = 0;
+            bool alive = true;
+            SmallIter it;
+            it.init(P, n_act);
+            SmallTile t;
+            while (alive && it.next(P, sh.active, n_act, t)) {
+                if (!ptx::mbar_wait(ptx::smem_u32(&sh.tempty[acc]), aph ^ 1u, &sh.abort_flag)) break;
+                ptx::tc_fence_after();
+                const uint32_t idesc = ptx::make_idesc_bf16(BM, (uint32_t)t.bn);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int i = 0; i < t.nk; ++i) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.full[s]), ph, &sh.abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    ptx::tc_fence_after();
+                    // M = 128 although only t_pad rows were loaded: the rows beyond are whatever the ring holds,
+                    // they only reach TMEM lanes that nobody reads
+                    const uint32_t a0 = smA + s * slot_bytes, b0 = smB + s * slot_bytes;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        ptx::umma_bf16(d_tmem, ptx::make_desc_k_sw128(a0 + k * 32), ptx::make_desc_k_sw128(b0 + k * 32),
+                                       idesc, (uint32_t)((i | k) != 0));
+                    ptx::umma_commit(ptx::smem_u32(&sh.empty[s]));
+                    if (++s == n_stages) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
+                }
+                if (!alive) break;
+                ptx::umma_commit(ptx::smem_u32(&sh.tfull[acc]));
+                if (++acc == 2) {
+                    acc = 0;
+                    aph ^= 1u;
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (4 warps)
+        const int q = warp & 3;
+        const int etid = (int)threadIdx.x - 64;
+        int acc = 0;
+        uint32_t aph = 0;
+        bool dead = aborted_early;     // a dead warp still takes part in every named barrier below
+        bool up_done = false;
+        SmallIter it;
+        it.init(P, n_act);
+        SmallTile t;
+        const int row = q * 32 + lane;
+        for (;;) {
+            const bool have = it.next(P, sh.active, n_act, t);
+            if (!up_done && (!have || t.phase == 1)) {
+                // this CTA's part of hg is complete: publish it, then signal the up/down grid barrier
+                __threadfence();
+                asm volatile("fence.proxy.async;" ::: "memory");
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (etid == 0) grid_arrive(P.sync, 1);
+                up_done = true;
+            }
+            if (!have) break;
+            if (t.phase == 0 && etid < P.T) {
+                // router gate of every token for this tile's expert(s), 0 where the token did not select it;
+                // fetched while the mainloop is still running (the previous tile ended on a barrier)
+                const uint64_t mk = P.mask[etid];
+                sh.gate_s[etid] = ((mk >> t.e) & 1ull) ? P.scores[(long long)etid * P.E + t.e] : 0.f;
+                sh.gate2_s[etid] = ((mk >> t.e2) & 1ull) ? P.scores[(long long)etid * P.E + t.e2] : 0.f;
+            }
+            if (!dead && !ptx::mbar_wait(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag)) dead = true;
+            dead = __any_sync(0xffffffffu, dead);     // the TMEM reads below are warp-collective
+            ptx::tc_fence_after();
+            const uint32_t taddr = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
+            if (t.phase == 0) {
+                // Few tokens fill only the first TMEM lanes, so one warp would do all the GeLU work.  Instead the
+                // warps that own valid lanes copy each 32-column chunk to shared memory and all 128 epilogue
+                // threads share the arithmetic.
+                for (int c = 0; c < t.bn; c += 32) {
+                    if (!dead && q * 32 < P.T) {
+                        uint32_t r[32];
+                        ptx::tmem_ld32(taddr + (uint32_t)c, r);
+                        ptx::tmem_ld_wait();
+                        if (row < P.T) {
+                            float4* dst = reinterpret_cast<float4*>(stg + row * STG_LD);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                                     __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                        }
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    const int groups = min(32, t.bn - c) / 8;
+                    const int items = P.T * groups;
+                    for (int item = etid; !dead && item < items; item += 128) {
+                        const int rr = item / groups, cg = item % groups;
+                        const float4 a = *reinterpret_cast<const float4*>(stg + rr * STG_LD + cg * 8);
+                        const float4 b = *reinterpret_cast<const float4*>(stg + rr * STG_LD + cg * 8 + 4);
+                        const int col = c + cg * 8;            // 8-column groups never straddle the expert boundary
+                        const bool second = col >= t.bn1;
+                        const float g = second ? sh.gate2_s[rr] : sh.gate_s[rr];
+                        const long long ocol = second ? (long long)t.out_col0_2 + (col - t.bn1) : (long long)t.out_col0 + col;
+                        uint4 pk;
+                        __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&pk);
+                        hv[0] = __floats2bfloat162_rn(g * gelu_erf(a.x), g * gelu_erf(a.y));
+                        hv[1] = __floats2bfloat162_rn(g * gelu_erf(a.z), g * gelu_erf(a.w));
+                        hv[2] = __floats2bfloat162_rn(g * gelu_erf(b.x), g * gelu_erf(b.y));
+                        hv[3] = __floats2bfloat162_rn(g * gelu_erf(b.z), g * gelu_erf(b.w));
+                        *reinterpret_cast<uint4*>(P.hg + (long long)rr * ((long long)P.E * P.H) + ocol) = pk;
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                }
+            } else {
+                // fp32 partial sums of this CTA's share of the reduction: slot (cta, seg), row, 256 columns
+                for (int c = 0; !dead && q * 32 < P.T && c < t.bn; c += 32) {
+                    uint32_t r[32];
+                    ptx::tmem_ld32(taddr + (uint32_t)c, r);
+                    ptx::tmem_ld_wait();
+                    if (row < P.T) {
+                        float4* dst = reinterpret_cast<float4*>(P.partial + (((long long)blockIdx.x * 2 + t.seg) * P.T + row) * BN + c);
+                        const int ncol = min(32, t.bn - c);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            if (j * 4 < ncol)
+                                dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                                     __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                    }
+                }
+            }
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0 && !dead) ptx::mbar_arrive(ptx::smem_u32(&sh.tempty[acc]));
+            if (++acc == 2) {
+                acc = 0;
+                aph ^= 1u;
+            }
+        }
+        // ---- last grid barrier, then the fix-up: out[t,c] = sum of the partial tiles covering column c in
+        // ascending CTA order (the partition arithmetic mirrors SmallIter)
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (etid == 0) {
+            grid_arrive(P.sync, 2);
+            if (!grid_wait(P.sync, 2, G, &sh.abort_flag)) sh.abort_flag = 1;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (!sh.abort_flag) {
+            const int kbpe = P.H / BK;
+            const int U = n_act * kbpe;
+            const int nr = (P.d + BN - 1) / BN;
+            const int total = nr * U;
+            const int per = total > 0 ? (total + G - 1) / G : 1;
+            // a thread owns 4 consecutive columns of one token; its partial loads are issued in batches before
+            // the additions, which run in ascending CTA order
+            const int d4 = P.d / 4;
+            const long long n_out4 = (long long)P.T * d4;
+            for (long long idx = (long long)blockIdx.x * 128 + etid; idx < n_out4; idx += (long long)G * 128) {
+                const int tt = (int)(idx / d4), col = (int)(idx % d4) * 4;
+                const int r = col / BN, cc = col % BN;
+                float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (U > 0) {
+                    const int i0 = (r * U) / per, i1 = ((r + 1) * U - 1) / per;
+                    for (int ib = i0; ib <= i1; ib += kFixBatch) {
+                        float4 v[kFixBatch];
+#pragma unroll
+                        for (int j = 0; j < kFixBatch; ++j) {
+                            const int i = ib + j;
+                            const int seg = r - (i * per) / U;
+                            v[j] = i <= i1 ? __ldcg(reinterpret_cast<const float4*>(
+                                                 P.partial + (((long long)i * 2 + seg) * P.T + tt) * BN + cc))
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int j = 0; j < kFixBatch; ++j) {
+                            sum.x += v[j].x;
+                            sum.y += v[j].y;
+                            sum.z += v[j].z;
+                            sum.w += v[j].w;
+                        }
+                    }
+                }
+                if (P.out_f32) {
+                    reinterpret_cast<float4*>(P.out)[idx] = sum;
+                } else {
+                    uint2 pk;
+                    *reinterpret_cast<__nv_bfloat162*>(&pk.x) = __floats2bfloat162_rn(sum.x, sum.y);
+                    *reinterpret_cast<__nv_bfloat162*>(&pk.y) = __floats2bfloat162_rn(sum.z, sum.w);
+                    reinterpret_cast<uint2*>(P.out)[idx] = pk;
+                }
+            }
+            if (P.counts_out && blockIdx.x == 0 && etid < P.E) {
+                int n = 0;
+                for (int tt = 0; tt < P.T; ++tt) n += (int)((P.mask[tt] >> etid) & 1ull);
+                P.counts_out[etid] = n;
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+    if (threadIdx.x == 0 && sh.abort_flag) {
+        atomicExch(P.sync + 4, 1);
+        if (P.dev_status) *P.dev_status = DSMOE_ERR_TIMEOUT;
+    }
 }
 
 // ---------------------------------------------------------------- host side
@@ -505,6 +991,12 @@ dsmoe_status make_map_3d(CUtensorMap* m, const void* ptr, uint64_t E, uint64_t n
     return r == CUDA_SUCCESS ? DSMOE_OK : DSMOE_ERR_CUDA;
 }
 
+// the five box heights of one packed weight tensor
+dsmoe_status make_bmaps(BMaps* b, const void* ptr, uint64_t E, uint64_t n, uint64_t k) {
+    for (int lvl = 0; lvl < 5; ++lvl) DSMOE_TRY(make_map_3d(&b->m[lvl], ptr, E, n, k, 16u << lvl));
+    return DSMOE_OK;
+}
+
 int sm_count() {
     static int n = 0;
     if (!n) {
@@ -515,7 +1007,7 @@ int sm_count() {
     return n;
 }
 
-// Optional per-launch timing of the expert GEMMs (a measurement aid for benchmarks): event pairs
+// Optional per-launch timing of the tensor-core kernels (a measurement aid for benchmarks): event pairs
 // around each launch of the most recent call.
 constexpr int kMaxTimed = 8;
 struct Timing {
@@ -524,7 +1016,7 @@ struct Timing {
     cudaEvent_t start[kMaxTimed], stop[kMaxTimed];
 } g_timing;
 
-dsmoe_status launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& P, int grid, cudaStream_t s) {
+dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams& P, int grid, cudaStream_t s) {
     static bool attr_set = false;
     if (!attr_set) {
         DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
@@ -577,46 +1069,68 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
     const size_t amax = amax_of(p);
     const __nv_bfloat16* w1t = static_cast<const __nv_bfloat16*>(packed);
     const __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
-    CUtensorMap mA1, mB1, mA2, mB2;
+    CUtensorMap mA1, mA2;
+    BMaps mB1, mB2;
     DSMOE_TRY(make_map_2d(&mA1, xp, amax, p.d, BM));
-    DSMOE_TRY(make_map_3d(&mB1, w1t, p.E, p.H, p.d, BN));
+    DSMOE_TRY(make_bmaps(&mB1, w1t, p.E, p.H, p.d));
     DSMOE_TRY(make_map_2d(&mA2, hbuf, amax, p.H, BM));
-    DSMOE_TRY(make_map_3d(&mB2, w2t, p.E, p.d, p.H, BN));
-    GemmParams up{GEMM_GROUPED, EPI_GELU, p.E, p.H, p.d, (int)amax, offsets, nullptr, hbuf, p.H, 0, dev_status,
-                  nullptr, BM, BN};
-    GemmParams down{GEMM_GROUPED, EPI_STORE, p.E, p.d, p.H, (int)amax, offsets, nullptr, yp, p.d, 0, dev_status,
-                    nullptr, BM, BN};
+    DSMOE_TRY(make_bmaps(&mB2, w2t, p.E, p.d, p.H));
+    GemmParams up{GEMM_GROUPED, EPI_GELU, p.E, p.H, p.d, (int)amax, offsets, nullptr, hbuf, p.H, 0, dev_status};
+    GemmParams down{GEMM_GROUPED, EPI_STORE, p.E, p.d, p.H, (int)amax, offsets, nullptr, yp, p.d, 0, dev_status};
     DSMOE_TRY(launch_gemm(mA1, mB1, up, sm_count(), s));
     DSMOE_TRY(launch_gemm(mA2, mB2, down, sm_count(), s));
     return DSMOE_OK;
 }
 
-// Few tokens (decode): every token rides in one 128-row tile, only the selected experts' weights are
-// streamed, and the router gate (zero for an unselected pair) is folded into h, so the layer needs no
-// grouping and no aggregation pass.
-static dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const void* packed,
-                                       const float* scores, const uint64_t* mask, void* out, char* ws,
-                                       const WsLayout& L, int32_t* dev_status, cudaStream_t s) {
+// Few tokens (decode): one cooperative launch of small_layer_kernel runs router, both projections and the
+// fix-up.
+bool small_supported(const dsmoe_layer_desc& p) {
+    const int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
+    return umma_supported(p) && p.T >= 1 && p.T <= kSmallMaxT && p.T <= G && ceil_div(p.d, BN) <= G;
+}
+
+dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
+                                const void* packed, float* scores, uint64_t* mask, int32_t* k_t, int32_t* counts_out,
+                                void* out, char* ws, const WsLayout& L, int32_t* dev_status, cudaStream_t s) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        DSMOE_CUDA_TRY(cudaFuncSetAttribute(small_layer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+        attr_set = true;
+    }
     const __nv_bfloat16* w1t = static_cast<const __nv_bfloat16*>(packed);
     const __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
-    void* hg = ws + L.h;                                        // [T, E*H] bf16
-    float* partial = reinterpret_cast<float*>(ws + L.partial);
     const int t_pad = (p.T + 7) / 8 * 8;
-    const int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
-    CUtensorMap mA1, mB1, mA2, mB2;
-    DSMOE_TRY(make_map_2d(&mA1, x, p.T, p.d, t_pad));
-    DSMOE_TRY(make_map_3d(&mB1, w1t, p.E, p.H, p.d, kUpUnit));
-    DSMOE_TRY(make_map_2d(&mA2, hg, p.T, (uint64_t)p.E * p.H, t_pad));
-    DSMOE_TRY(make_map_3d(&mB2, w2t, p.E, p.d, p.H, BN));
-    GemmParams up{GEMM_SMALL_UP, EPI_GELU, p.E, p.H, p.d, p.T, nullptr, scores, hg, (long long)p.E * p.H, 0,
-                  dev_status, mask, t_pad, kUpUnit};
-    GemmParams down{GEMM_SMALL_DOWN, EPI_PARTIAL, p.E, p.d, p.H, p.T, nullptr, nullptr, partial, BN, 1,
-                    dev_status, mask, t_pad, BN};
-    DSMOE_TRY(launch_gemm(mA1, mB1, up, G, s));
-    DSMOE_TRY(launch_gemm(mA2, mB2, down, G, s));
-    small_fixup_kernel<<<dim3(ceil_div(p.d, BN), p.T), BN, 0, s>>>(partial, mask, out, p.T, p.d, p.E, p.H / BK, G,
-                                                                  (p.out_fp32 || p.dtype == DSMOE_F32) ? 1 : 0);
-    DSMOE_CUDA_TRY(cudaGetLastError());
+    int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
+    CUtensorMap mX, mHg;
+    BMaps mW1, mW2;
+    void* hg = ws + L.h;
+    DSMOE_TRY(make_map_2d(&mX, x, p.T, p.d, t_pad));
+    DSMOE_TRY(make_bmaps(&mW1, w1t, p.E, p.H, p.d));
+    DSMOE_TRY(make_map_2d(&mHg, hg, p.T, (uint64_t)p.E * p.H, t_pad));
+    DSMOE_TRY(make_bmaps(&mW2, w2t, p.E, p.d, p.H));
+    SmallParams P;
+    P.T = p.T; P.d = p.d; P.H = p.H; P.E = p.E; P.t_pad = t_pad;
+    P.x = static_cast<const __nv_bfloat16*>(x);
+    P.Wr = Wr;
+    P.br = br;
+    P.sel = SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k};
+    P.scores = scores;
+    P.mask = mask;
+    P.k_t = k_t;
+    P.counts_out = counts_out;
+    P.hg = static_cast<__nv_bfloat16*>(hg);
+    P.partial = reinterpret_cast<float*>(ws + L.partial);
+    P.out = out;
+    P.out_f32 = p.out_fp32 ? 1 : 0;
+    P.sync = reinterpret_cast<int*>(ws + L.sync);
+    P.dev_status = dev_status;
+    DSMOE_CUDA_TRY(cudaMemsetAsync(P.sync, 0, 32, s));
+    void* args[] = {&mX, &mW1, &mHg, &mW2, &P};
+    const bool timed = g_timing.on && g_timing.n < kMaxTimed;
+    if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
+    DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(small_layer_kernel), dim3(G), dim3(NUM_THREADS),
+                                               args, SMEM_BYTES, s));
+    if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.stop[g_timing.n++], s));
     return DSMOE_OK;
 }
 
@@ -625,32 +1139,24 @@ dsmoe_status launch_layer_umma(const dsmoe_layer_desc& p, const void* x, const v
                                const WsLayout& L, int32_t* dev_status, cudaStream_t s, bool* done) {
     *done = false;
     (void)k_t;
-    if (!umma_supported(p)) return DSMOE_OK;
-    const int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
-    if (p.T <= kSmallMaxT && ceil_div(p.d, BN) <= G) {
-        DSMOE_TRY(launch_layer_small(p, x, packed, scores, mask, out, ws, L, dev_status, s));
-    } else if (p.mode == DSMOE_SELECT_ALL) {
-        // Dense forward: gate folded into h, aggregation folded into the down-projection's reduction.
-        const __nv_bfloat16* w1t = static_cast<const __nv_bfloat16*>(packed);
-        const __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
-        void* hg = ws + L.h;                                        // [T, E*H] bf16
-        CUtensorMap mA1, mB1, mA2, mB2;
-        DSMOE_TRY(make_map_2d(&mA1, x, p.T, p.d, BM));
-        DSMOE_TRY(make_map_3d(&mB1, w1t, p.E, p.H, p.d, BN));
-        DSMOE_TRY(make_map_2d(&mA2, hg, p.T, (uint64_t)p.E * p.H, BM));
-        DSMOE_TRY(make_map_3d(&mB2, w2t, p.E, p.d, p.H, BN));
-        const int out_f32 = p.out_fp32 ? 1 : 0;
-        GemmParams up{GEMM_DENSE_UP, EPI_GELU, p.E, p.H, p.d, p.T, nullptr, scores, hg, (long long)p.E * p.H, 0,
-                      dev_status, nullptr, BM, BN};
-        GemmParams down{GEMM_DENSE_DOWN, EPI_STORE, p.E, p.d, p.H, p.T, nullptr, nullptr, out, p.d, out_f32,
-                        dev_status, nullptr, BM, BN};
-        const int mt = ceil_div(p.T, BM);
-        const int tiles_up = mt * ceil_div(p.H, BN) * p.E, tiles_down = mt * ceil_div(p.d, BN);
-        DSMOE_TRY(launch_gemm(mA1, mB1, up, tiles_up < sm_count() ? tiles_up : sm_count(), s));
-        DSMOE_TRY(launch_gemm(mA2, mB2, down, tiles_down < sm_count() ? tiles_down : sm_count(), s));
-    } else {
-        return DSMOE_OK;
-    }
+    if (!umma_supported(p) || p.mode != DSMOE_SELECT_ALL) return DSMOE_OK;
+    // Dense forward: gate folded into h, aggregation folded into the down-projection's reduction.
+    const __nv_bfloat16* w1t = static_cast<const __nv_bfloat16*>(packed);
+    const __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
+    void* hg = ws + L.h;                                        // [T, E*H] bf16
+    CUtensorMap mA1, mA2;
+    BMaps mB1, mB2;
+    DSMOE_TRY(make_map_2d(&mA1, x, p.T, p.d, BM));
+    DSMOE_TRY(make_bmaps(&mB1, w1t, p.E, p.H, p.d));
+    DSMOE_TRY(make_map_2d(&mA2, hg, p.T, (uint64_t)p.E * p.H, BM));
+    DSMOE_TRY(make_bmaps(&mB2, w2t, p.E, p.d, p.H));
+    const int out_f32 = p.out_fp32 ? 1 : 0;
+    GemmParams up{GEMM_DENSE_UP, EPI_GELU, p.E, p.H, p.d, p.T, nullptr, scores, hg, (long long)p.E * p.H, 0, dev_status};
+    GemmParams down{GEMM_DENSE_DOWN, EPI_STORE, p.E, p.d, p.H, p.T, nullptr, nullptr, out, p.d, out_f32, dev_status};
+    const int mt = ceil_div(p.T, BM);
+    const int tiles_up = mt * ceil_div(p.H, BN) * p.E, tiles_down = mt * ceil_div(p.d, BN);
+    DSMOE_TRY(launch_gemm(mA1, mB1, up, tiles_up < sm_count() ? tiles_up : sm_count(), s));
+    DSMOE_TRY(launch_gemm(mA2, mB2, down, tiles_down < sm_count() ? tiles_down : sm_count(), s));
     if (counts_out) {
         int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
         int32_t* offsets = reinterpret_cast<int32_t*>(ws + L.offsets);
