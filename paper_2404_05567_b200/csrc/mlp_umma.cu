@@ -32,6 +32,7 @@ constexpr int SHARED_BYTES = 3072;                                     // barrie
 constexpr int STG_LD = 36;                                             // floats per row of the epilogue staging tile
 constexpr int STG_BYTES = BM * STG_LD * 4;
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)RING_BYTES + SHARED_BYTES + STG_BYTES;
+constexpr size_t SMEM_GEMM_BYTES = 1024 + (size_t)RING_BYTES + SHARED_BYTES;   // umma_gemm_kernel needs no staging tile
 
 enum { GEMM_GROUPED = 0, GEMM_DENSE_UP = 1, GEMM_DENSE_DOWN = 2 };
 enum { EPI_GELU = 0, EPI_STORE = 1 };
@@ -221,7 +222,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         a_col = b_k;
                     }
                     ptx::tma_load_2d(smA + s * A_STAGE_BYTES, &tmA, bar, a_col, t.row0);
-                    load_weight_rows(&tmB, smB + s * B_STAGE_BYTES, bar, b_k, t.n0, t.bn, b_e);
+                    // full-width tiles take the one 256-row copy directly (measurably faster than walking the
+                    // box sizes); only a ragged last column tile needs the decomposition
+                    if (t.bn == BN) ptx::tma_load_3d(smB + s * B_STAGE_BYTES, &tmB.m[4], bar, b_k, t.n0, b_e);
+                    else load_weight_rows(&tmB, smB + s * B_STAGE_BYTES, bar, b_k, t.n0, t.bn, b_e);
                     if (++s == STAGES) {
                         s = 0;
                         ph ^= 1u;
@@ -1019,12 +1023,12 @@ struct Timing {
 dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams& P, int grid, cudaStream_t s) {
     static bool attr_set = false;
     if (!attr_set) {
-        DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+        DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_BYTES));
         attr_set = true;
     }
     const bool timed = g_timing.on && g_timing.n < kMaxTimed;
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
-    umma_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(a, b, P);
+    umma_gemm_kernel<<<grid, NUM_THREADS, SMEM_GEMM_BYTES, s>>>(a, b, P);
     DSMOE_CUDA_TRY(cudaGetLastError());
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.stop[g_timing.n++], s));
     return DSMOE_OK;
