@@ -60,6 +60,12 @@ struct BMaps {
     CUtensorMap m[5];
 };
 
+// ... and, for the small-T up-projection whose tile widths are arbitrary multiples of 16, one map per height
+// 16, 32, ..., 256, so that a tile (or each of its two parts) is a single copy.
+struct BMaps16 {
+    CUtensorMap m[16];
+};
+
 struct Tile {
     int row0, rows_valid, e, n0, bn, nk, out_col0;
 };
@@ -70,6 +76,7 @@ struct Shared {
     volatile int abort_flag;
     int bad_offsets;
     int n_stages, slot_bytes, a_bytes;   // ring geometry (small_layer_kernel)
+    int bn_down;                         // small_layer_kernel: column-range width of the down-projection
     int tile_prefix[kMaxExperts + 1];
     int seg0[kMaxExperts], seg1[kMaxExperts];
     unsigned long long active_mask;      // experts selected by at least one token
@@ -420,8 +427,11 @@ struct SmallTile {
 struct SmallIter {
     int phase, u0, u1, r_first, down_u0, down_u1;
 
-    __device__ __forceinline__ void init(const SmallParams& P, int n_act) {
+    int bn_down;
+
+    __device__ __forceinline__ void init(const SmallParams& P, int n_act, int bn_down_) {
         const int G = gridDim.x;
+        bn_down = bn_down_;
         {
             const int total = n_act * (P.H / kUpUnit);
             const int per = (total + G - 1) / G;
@@ -430,7 +440,7 @@ struct SmallIter {
         }
         {
             const int U = n_act * (P.H / BK);
-            const int total = ((P.d + BN - 1) / BN) * U;
+            const int total = ((P.d + bn_down - 1) / bn_down) * U;
             const int per = (total + G - 1) / G;
             down_u0 = min(total, (int)blockIdx.x * per);
             down_u1 = min(total, down_u0 + per);
@@ -474,8 +484,8 @@ struct SmallIter {
             const int r = u0 / U, start = u0 % U;
             const int len = min(u1 - u0, U - start);
             t.e = 0;
-            t.n0 = r * BN;
-            t.bn = min(BN, P.d - t.n0);
+            t.n0 = r * bn_down;
+            t.bn = min(bn_down, P.d - t.n0);
             t.bn1 = t.bn;
             t.nk = len;
             t.kstart = start;
@@ -488,27 +498,32 @@ struct SmallIter {
 };
 
 // One ring slot's loads.  what: bit 0 = the token operand (x or hg), bit 1 = the weight rows.
-__device__ __forceinline__ void small_issue(const SmallParams& P, const CUtensorMap* tmX, const BMaps* tmW1,
+__device__ __forceinline__ void small_issue(const SmallParams& P, const CUtensorMap* tmX, const BMaps16* tmW1,
                                             const CUtensorMap* tmHg, const BMaps* tmW2, const int* active,
                                             const SmallTile& t, int i, uint32_t slotA, uint32_t slotB, uint32_t bar,
                                             int what) {
     if (t.phase == 0) {
         if (what & 1) ptx::tma_load_2d(slotA, tmX, bar, i * BK, 0);
         if (what & 2) {
-            load_weight_rows(tmW1, slotB, bar, i * BK, t.n0, t.bn1, t.e);
-            if (t.bn > t.bn1) load_weight_rows(tmW1, slotB + t.bn1 * (BK * 2), bar, i * BK, 0, t.bn - t.bn1, t.e2);
+            ptx::tma_load_3d(slotB, &tmW1->m[t.bn1 / 16 - 1], bar, i * BK, t.n0, t.e);
+            if (t.bn > t.bn1)
+                ptx::tma_load_3d(slotB + t.bn1 * (BK * 2), &tmW1->m[(t.bn - t.bn1) / 16 - 1], bar, i * BK, 0, t.e2);
         }
     } else {
         const int kbpe = P.H / BK;
         const int g = t.kstart + i;
         const int e = active[g / kbpe], kb = g % kbpe;
         if (what & 1) ptx::tma_load_2d(slotA, tmHg, bar, e * P.H + kb * BK, 0);
-        if (what & 2) load_weight_rows(tmW2, slotB, bar, kb * BK, t.n0, t.bn, e);
+        if (what & 2) {
+            // column ranges are 64, 128 or 256 wide: one copy; only a ragged last range needs the decomposition
+            if ((t.bn & (t.bn - 1)) == 0) ptx::tma_load_3d(slotB, &tmW2->m[__ffs(t.bn) - 5], bar, kb * BK, t.n0, e);
+            else load_weight_rows(tmW2, slotB, bar, kb * BK, t.n0, t.bn, e);
+        }
     }
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ BMaps tmW1,
+small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ BMaps16 tmW1,
                    const __grid_constant__ CUtensorMap tmHg, const __grid_constant__ BMaps tmW2, const SmallParams P) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -532,10 +547,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&tmX);
         ptx::prefetch_tensormap(&tmHg);
-        for (int i = 0; i < 5; ++i) {
-            ptx::prefetch_tensormap(&tmW1.m[i]);
-            ptx::prefetch_tensormap(&tmW2.m[i]);
-        }
+        for (int i = 2; i < 5; ++i) ptx::prefetch_tensormap(&tmW2.m[i]);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), TMEM_COLS);
@@ -642,10 +654,16 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         for (int e = 0; e < P.E; ++e)
             if ((m >> e) & 1ull) sh.active[n++] = e;
         sh.n_act = n;
-        // ring geometry: a slot holds the tokens' 64-wide block and up to 256 weight rows
+        // Ring geometry: a slot holds the tokens' 64-wide block and one weight tile.  With few selected experts
+        // the tiles are narrow, so the down-projection takes narrower column ranges too and the ring has more
+        // slots: more loads in flight, which is what hides memory latency when each load is small.
+        const int up_units = (n * (P.H / kUpUnit) + G - 1) / G;
+        const int up_rows = max(1, min(up_units, kUpTileUnits)) * kUpUnit;
+        sh.bn_down = up_rows <= 64 ? 64 : up_rows <= 128 ? 128 : BN;
         sh.a_bytes = P.t_pad * BK * 2;
-        sh.slot_bytes = sh.a_bytes + B_STAGE_BYTES;
+        sh.slot_bytes = sh.a_bytes + sh.bn_down * BK * 2;
         sh.n_stages = min(MAX_STAGES, RING_BYTES / sh.slot_bytes);
+        ptx::prefetch_tensormap(&tmW1.m[up_rows / 16 - 1]);
     }
     __syncthreads();
     const uint32_t tmem_base = sh.tmem_base;
@@ -661,7 +679,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             uint32_t ph = 0;
             bool alive = true;
             SmallIter it;
-            it.init(P, n_act);
+            it.init(P, n_act, sh.bn_down);
             SmallTile t;
             bool have = it.next(P, sh.active, n_act, t);
             // up-projection
@@ -743,7 +761,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             uint32_t ph = 0, aph = 0;
             bool alive = true;
             SmallIter it;
-            it.init(P, n_act);
+            it.init(P, n_act, sh.bn_down);
             SmallTile t;
             while (alive && it.next(P, sh.active, n_act, t)) {
                 if (!ptx::mbar_wait(ptx::smem_u32(&sh.tempty[acc]), aph ^ 1u, &sh.abort_flag)) break;
@@ -786,7 +804,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         bool dead = aborted_early;     // a dead warp still takes part in every named barrier below
         bool up_done = false;
         SmallIter it;
-        it.init(P, n_act);
+        it.init(P, n_act, sh.bn_down);
         SmallTile t;
         const int row = q * 32 + lane;
         for (;;) {
@@ -886,7 +904,8 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         if (!sh.abort_flag) {
             const int kbpe = P.H / BK;
             const int U = n_act * kbpe;
-            const int nr = (P.d + BN - 1) / BN;
+            const int bnd = sh.bn_down;
+            const int nr = (P.d + bnd - 1) / bnd;
             const int total = nr * U;
             const int per = total > 0 ? (total + G - 1) / G : 1;
             // a thread owns 4 consecutive columns of one token; its partial loads are issued in batches before
@@ -895,7 +914,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             const long long n_out4 = (long long)P.T * d4;
             for (long long idx = (long long)blockIdx.x * 128 + etid; idx < n_out4; idx += (long long)G * 128) {
                 const int tt = (int)(idx / d4), col = (int)(idx % d4) * 4;
-                const int r = col / BN, cc = col % BN;
+                const int r = col / bnd, cc = col % bnd;
                 float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (U > 0) {
                     const int i0 = (r * U) / per, i1 = ((r + 1) * U - 1) / per;
@@ -995,6 +1014,11 @@ dsmoe_status make_map_3d(CUtensorMap* m, const void* ptr, uint64_t E, uint64_t n
     return r == CUDA_SUCCESS ? DSMOE_OK : DSMOE_ERR_CUDA;
 }
 
+dsmoe_status make_bmaps16(BMaps16* b, const void* ptr, uint64_t E, uint64_t n, uint64_t k) {
+    for (int i = 0; i < 16; ++i) DSMOE_TRY(make_map_3d(&b->m[i], ptr, E, n, k, 16u * (i + 1)));
+    return DSMOE_OK;
+}
+
 // the five box heights of one packed weight tensor
 dsmoe_status make_bmaps(BMaps* b, const void* ptr, uint64_t E, uint64_t n, uint64_t k) {
     for (int lvl = 0; lvl < 5; ++lvl) DSMOE_TRY(make_map_3d(&b->m[lvl], ptr, E, n, k, 16u << lvl));
@@ -1090,7 +1114,7 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
 // fix-up.
 bool small_supported(const dsmoe_layer_desc& p) {
     const int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
-    return umma_supported(p) && p.T >= 1 && p.T <= kSmallMaxT && p.T <= G && ceil_div(p.d, BN) <= G;
+    return umma_supported(p) && p.T >= 1 && p.T <= kSmallMaxT && p.T <= G && ceil_div(p.d, 64) <= G;
 }
 
 dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
@@ -1105,13 +1129,38 @@ dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const 
     const __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
     const int t_pad = (p.T + 7) / 8 * 8;
     int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
-    CUtensorMap mX, mHg;
-    BMaps mW1, mW2;
     void* hg = ws + L.h;
-    DSMOE_TRY(make_map_2d(&mX, x, p.T, p.d, t_pad));
-    DSMOE_TRY(make_bmaps(&mW1, w1t, p.E, p.H, p.d));
-    DSMOE_TRY(make_map_2d(&mHg, hg, p.T, (uint64_t)p.E * p.H, t_pad));
-    DSMOE_TRY(make_bmaps(&mW2, w2t, p.E, p.d, p.H));
+    // The 23 tensor maps of a call depend only on the buffers and the shape: encoded once, then reused
+    // (decode loops call with the same buffers every step).  Not thread-safe, like the timing aid.
+    struct MapSet {
+        const void *x, *hg, *packed;
+        int T, d, H, E;
+        CUtensorMap mX, mHg;
+        BMaps16 mW1;
+        BMaps mW2;
+    };
+    constexpr int kCache = 64;
+    static MapSet cache[kCache];
+    static int n_cached = 0, next_slot = 0;
+    MapSet* ms = nullptr;
+    for (int i = 0; i < n_cached; ++i) {
+        MapSet& c = cache[i];
+        if (c.x == x && c.hg == hg && c.packed == packed && c.T == p.T && c.d == p.d && c.H == p.H && c.E == p.E) {
+            ms = &c;
+            break;
+        }
+    }
+    if (!ms) {
+        MapSet c;
+        c.x = x; c.hg = hg; c.packed = packed; c.T = p.T; c.d = p.d; c.H = p.H; c.E = p.E;
+        DSMOE_TRY(make_map_2d(&c.mX, x, p.T, p.d, t_pad));
+        DSMOE_TRY(make_bmaps16(&c.mW1, w1t, p.E, p.H, p.d));
+        DSMOE_TRY(make_map_2d(&c.mHg, hg, p.T, (uint64_t)p.E * p.H, t_pad));
+        DSMOE_TRY(make_bmaps(&c.mW2, w2t, p.E, p.d, p.H));
+        const int slot = n_cached < kCache ? n_cached++ : (next_slot++ % kCache);
+        cache[slot] = c;
+        ms = &cache[slot];
+    }
     SmallParams P;
     P.T = p.T; P.d = p.d; P.H = p.H; P.E = p.E; P.t_pad = t_pad;
     P.x = static_cast<const __nv_bfloat16*>(x);
@@ -1129,7 +1178,7 @@ dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const 
     P.sync = reinterpret_cast<int*>(ws + L.sync);
     P.dev_status = dev_status;
     DSMOE_CUDA_TRY(cudaMemsetAsync(P.sync, 0, 32, s));
-    void* args[] = {&mX, &mW1, &mHg, &mW2, &P};
+    void* args[] = {&ms->mX, &ms->mW1, &ms->mHg, &ms->mW2, &P};
     const bool timed = g_timing.on && g_timing.n < kMaxTimed;
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
     DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(small_layer_kernel), dim3(G), dim3(NUM_THREADS),
