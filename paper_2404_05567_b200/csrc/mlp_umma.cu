@@ -28,9 +28,8 @@ constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr int RING_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);   // operand ring: 4 x 48 KB, or more, smaller slots
-constexpr int SHARED_BYTES = 3072;                                     // barriers and small tables (struct Shared)
-constexpr int STG_LD = 36;                                             // floats per row of the epilogue staging tile
-constexpr int STG_BYTES = BM * STG_LD * 4;
+constexpr int SHARED_BYTES = 3072 + 256;                                     // barriers and small tables (struct Shared)
+constexpr int STG_BYTES = BM * 36 * 4;                                 // epilogue staging tile: T rows x (32..256 + 4) floats
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)RING_BYTES + SHARED_BYTES + STG_BYTES;
 constexpr size_t SMEM_GEMM_BYTES = 1024 + (size_t)RING_BYTES + SHARED_BYTES;   // umma_gemm_kernel needs no staging tile
 
@@ -38,6 +37,7 @@ enum { GEMM_GROUPED = 0, GEMM_DENSE_UP = 1, GEMM_DENSE_DOWN = 2 };
 enum { EPI_GELU = 0, EPI_STORE = 1 };
 constexpr int kUpUnit = 16;          // small-T up-projection: weight rows per work unit
 constexpr int kUpTileUnits = 16;     // ... and units per tile (256 rows)
+constexpr int kRouterBatch = 12;     // rows of Wr a router thread loads at once
 constexpr int kFixBatch = 24;        // partial tiles a fix-up thread loads at once
 
 struct GemmParams {
@@ -83,8 +83,19 @@ struct Shared {
     int n_act;
     int active[kMaxExperts];
     float gate_s[BM], gate2_s[BM];
+#ifdef DSMOE_TRACE
+    unsigned long long trace[32];
+#endif
 };
 static_assert(sizeof(Shared) <= SHARED_BYTES, "Shared must fit its slot");
+
+#ifdef DSMOE_TRACE
+// Diagnostic build only (-DDSMOE_TRACE): per-CTA time stamps (globaltimer ns) of small_layer_kernel's milestones.
+__device__ unsigned long long g_trace[192][32];
+#define TRACE(i) sh.trace[i] = ptx::globaltimer_ns()
+#else
+#define TRACE(i)
+#endif
 
 __device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f)); }
 
@@ -544,6 +555,10 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         }
         sh.abort_flag = 0;
         sh.active_mask = 0ull;
+#ifdef DSMOE_TRACE
+        for (int i = 0; i < 32; ++i) sh.trace[i] = 0;
+        TRACE(0);
+#endif
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&tmX);
         ptx::prefetch_tensormap(&tmHg);
@@ -555,70 +570,72 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
 
     // ------------------------------------------------------------ router, step 1
-    // The reduction over d of every token is cut into KS slices, one CTA per (token, slice); a thread takes
-    // whole rows of Wr (E contiguous floats), two rows at a time, so many independent loads are in flight.
+    // The reduction over d of every token is cut into KS slices, one CTA per (token, slice).  A row of Wr
+    // (E floats) is covered by E/4 neighbouring threads with one 16-byte load each, so a warp reads whole
+    // rows, coalesced, and a thread keeps only its four experts' sums over every rpp-th row; all its loads are
+    // independent.  The threads' sums meet in shared memory.
     const int KS = max(1, min(16, G / P.T));
     if ((int)blockIdx.x < P.T * KS) {
         const int t = blockIdx.x / KS, sl = blockIdx.x % KS, E = P.E;
         const int klen = (P.d + KS - 1) / KS, kbeg = sl * klen, kend = min(P.d, kbeg + klen);
         const __nv_bfloat16* __restrict__ xr = P.x + (size_t)t * P.d;
         const float* __restrict__ Wr = P.Wr;
-        float acc[kMaxExperts];
+        const int quads = (E + 3) / 4;                  // threads per row
+        const int rpp = NUM_THREADS / quads;            // rows per pass
+        const int qd = threadIdx.x % quads, r0 = threadIdx.x / quads;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (threadIdx.x == 32) TRACE(12);
+        if (r0 < rpp) {
+            if ((E & 3) == 0) {
+                // batches of kRouterBatch rows: every load of a batch is issued before its first use
+                for (int kb = kbeg + r0; kb < kend; kb += kRouterBatch * rpp) {
+                    float4 w[kRouterBatch];
+                    float xs[kRouterBatch];
 #pragma unroll
-        for (int e = 0; e < kMaxExperts; ++e) acc[e] = 0.f;
-        if ((E & 3) == 0) {
-            for (int k0 = kbeg + (int)threadIdx.x; k0 < kend; k0 += 2 * NUM_THREADS) {
-                const int k1 = k0 + NUM_THREADS;
-                const bool has1 = k1 < kend;
-                const float4* p0 = reinterpret_cast<const float4*>(Wr + (size_t)k0 * E);
-                const float4* p1 = reinterpret_cast<const float4*>(Wr + (size_t)(has1 ? k1 : k0) * E);
-                float4 w0[kMaxExperts / 4], w1[kMaxExperts / 4];
-#pragma unroll
-                for (int e4 = 0; e4 < kMaxExperts / 4; ++e4)
-                    if (e4 * 4 < E) {
-                        w0[e4] = __ldg(p0 + e4);
-                        w1[e4] = __ldg(p1 + e4);
+                    for (int j = 0; j < kRouterBatch; ++j) {
+                        const int k = kb + j * rpp;
+                        const bool ok = k < kend;
+                        w[j] = ok ? __ldg(reinterpret_cast<const float4*>(Wr + (size_t)k * E) + qd) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        xs[j] = ok ? __bfloat162float(xr[k]) : 0.f;
                     }
-                const float x0 = __bfloat162float(xr[k0]);
-                const float x1 = has1 ? __bfloat162float(xr[k1]) : 0.f;
 #pragma unroll
-                for (int e4 = 0; e4 < kMaxExperts / 4; ++e4)
-                    if (e4 * 4 < E) {
-                        acc[e4 * 4 + 0] = fmaf(x1, w1[e4].x, fmaf(x0, w0[e4].x, acc[e4 * 4 + 0]));
-                        acc[e4 * 4 + 1] = fmaf(x1, w1[e4].y, fmaf(x0, w0[e4].y, acc[e4 * 4 + 1]));
-                        acc[e4 * 4 + 2] = fmaf(x1, w1[e4].z, fmaf(x0, w0[e4].z, acc[e4 * 4 + 2]));
-                        acc[e4 * 4 + 3] = fmaf(x1, w1[e4].w, fmaf(x0, w0[e4].w, acc[e4 * 4 + 3]));
+                    for (int j = 0; j < kRouterBatch; ++j) {
+                        acc.x = fmaf(xs[j], w[j].x, acc.x);
+                        acc.y = fmaf(xs[j], w[j].y, acc.y);
+                        acc.z = fmaf(xs[j], w[j].z, acc.z);
+                        acc.w = fmaf(xs[j], w[j].w, acc.w);
                     }
-            }
-        } else {
-            for (int k = kbeg + (int)threadIdx.x; k < kend; k += NUM_THREADS) {
-                const float xv = __bfloat162float(xr[k]);
-#pragma unroll
-                for (int e = 0; e < kMaxExperts; ++e)
-                    if (e < E) acc[e] = fmaf(xv, __ldg(Wr + (size_t)k * E + e), acc[e]);
+                }
+            } else {
+                const int e0 = qd * 4;
+                for (int k = kbeg + r0; k < kend; k += rpp) {
+                    const float xv = __bfloat162float(xr[k]);
+                    const float* w = Wr + (size_t)k * E + e0;
+                    acc.x = fmaf(xv, __ldg(w), acc.x);
+                    if (e0 + 1 < E) acc.y = fmaf(xv, __ldg(w + 1), acc.y);
+                    if (e0 + 2 < E) acc.z = fmaf(xv, __ldg(w + 2), acc.z);
+                    if (e0 + 3 < E) acc.w = fmaf(xv, __ldg(w + 3), acc.w);
+                }
             }
         }
-#pragma unroll
-        for (int e = 0; e < kMaxExperts; ++e) {
-            if (e < E) {
-                const float v = warp_sum(acc[e]);
-                if (lane == 0) stg[warp * kMaxExperts + e] = v;
-            }
-        }
+        if (threadIdx.x == 32) TRACE(13);
+        reinterpret_cast<float4*>(stg)[threadIdx.x] = acc;      // stg[(r0 * quads + qd) * 4 + j]
         __syncthreads();
         if ((int)threadIdx.x < E) {
+            const int e = threadIdx.x;
             float v = 0.f;
-#pragma unroll
-            for (int w = 0; w < NUM_THREADS / 32; ++w) v += stg[w * kMaxExperts + threadIdx.x];
-            P.partial[((size_t)t * KS + sl) * kMaxExperts + threadIdx.x] = v;   // free until the down-projection
+            for (int r = 0; r < rpp; ++r) v += stg[(r * quads + (e >> 2)) * 4 + (e & 3)];
+            P.partial[((size_t)t * KS + sl) * kMaxExperts + e] = v;   // the partial-sum buffer is free until the down-projection
         }
     }
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
     if (threadIdx.x == 0) {
+        TRACE(1);
         grid_arrive(P.sync, 0);
         grid_wait(P.sync, 0, G, &sh.abort_flag);
+        TRACE(14);
     }
     __syncthreads();
     // ------------------------------------------------------------ router, step 2
@@ -636,8 +653,10 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
     __syncthreads();
     if (threadIdx.x == 0) {
+        TRACE(15);
         grid_arrive(P.sync, 3);
         grid_wait(P.sync, 3, G, &sh.abort_flag);
+        TRACE(2);
     }
     __syncthreads();
     // every CTA derives the set of selected experts from the T selection words
@@ -671,6 +690,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     const uint32_t slot_bytes = (uint32_t)sh.slot_bytes, a_bytes = (uint32_t)sh.a_bytes;
     const uint32_t smA = base, smB = base + a_bytes;
     const bool aborted_early = sh.abort_flag != 0;
+    if (threadIdx.x == 0) TRACE(3);
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -725,7 +745,9 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     have = it.next(P, sh.active, n_act, t);
                 }
             }
+            TRACE(5);
             if (alive && !grid_wait(P.sync, 1, G, &sh.abort_flag)) alive = false;
+            TRACE(6);
             asm volatile("fence.proxy.async;" ::: "memory");   // hg was written through the generic proxy, TMA reads it
             for (int j = 0; alive && j < npend; ++j)
                 small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, sh.active, pend_t[j], pend_i[j], smA + pend_s[j] * slot_bytes,
@@ -773,6 +795,12 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                         alive = false;
                         break;
                     }
+#ifdef DSMOE_TRACE
+                    if (sh.trace[4] == 0) TRACE(4);
+                    if (t.phase == 1 && sh.trace[8] == 0) TRACE(8);
+                    if (t.phase == 0 && i < 8) TRACE(16 + i);
+                    if (t.phase == 0 && i >= t.nk - 4) TRACE(24 + i - (t.nk - 4));
+#endif
                     ptx::tc_fence_after();
                     // M = 128 although only t_pad rows were loaded: the rows beyond are whatever the ring holds,
                     // they only reach TMEM lanes that nobody reads
@@ -810,11 +838,14 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         for (;;) {
             const bool have = it.next(P, sh.active, n_act, t);
             if (!up_done && (!have || t.phase == 1)) {
-                // this CTA's part of hg is complete: publish it, then signal the up/down grid barrier
-                __threadfence();
+                // this CTA's part of hg is complete: publish it (the arriving thread's fence, after the barrier,
+                // covers the other threads' stores), then signal the up/down grid barrier
                 asm volatile("fence.proxy.async;" ::: "memory");
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (etid == 0) grid_arrive(P.sync, 1);
+                if (etid == 0) {
+                    grid_arrive(P.sync, 1);
+                    TRACE(7);
+                }
                 up_done = true;
             }
             if (!have) break;
@@ -827,33 +858,44 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             }
             if (!dead && !ptx::mbar_wait(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag)) dead = true;
             dead = __any_sync(0xffffffffu, dead);     // the TMEM reads below are warp-collective
+#ifdef DSMOE_TRACE
+            if (etid == 0 && t.phase == 0) TRACE(28);
+#endif
             ptx::tc_fence_after();
             const uint32_t taddr = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
             if (t.phase == 0) {
                 // Few tokens fill only the first TMEM lanes, so one warp would do all the GeLU work.  Instead the
-                // warps that own valid lanes copy each 32-column chunk to shared memory and all 128 epilogue
-                // threads share the arithmetic.
-                for (int c = 0; c < t.bn; c += 32) {
+                // warps that own valid lanes copy the accumulators to shared memory, as many columns per round as the
+                // staging tile holds for T rows, and all 128 epilogue threads share the arithmetic.
+                const int CH = P.T <= 16 ? 256 : P.T <= 32 ? 128 : P.T <= 64 ? 64 : 32;   // columns per round
+                const int ld = CH + 4;                                                    // floats per staged row
+                for (int c0 = 0; c0 < t.bn; c0 += CH) {
+                    const int cw = min(CH, t.bn - c0);
                     if (!dead && q * 32 < P.T) {
-                        uint32_t r[32];
-                        ptx::tmem_ld32(taddr + (uint32_t)c, r);
-                        ptx::tmem_ld_wait();
-                        if (row < P.T) {
-                            float4* dst = reinterpret_cast<float4*>(stg + row * STG_LD);
+                        for (int c = 0; c < cw; c += 32) {
+                            uint32_t r[32];
+                            ptx::tmem_ld32(taddr + (uint32_t)(c0 + c), r);
+                            ptx::tmem_ld_wait();
+                            if (row < P.T) {
+                                float4* dst = reinterpret_cast<float4*>(stg + row * ld + c);
 #pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                                     __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                                for (int j = 0; j < 8; ++j)
+                                    dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                                         __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                            }
                         }
                     }
                     asm volatile("bar.sync 1, 128;" ::: "memory");
-                    const int groups = min(32, t.bn - c) / 8;
+#ifdef DSMOE_TRACE
+                    if (etid == 0) TRACE(29 + (c0 > 0));
+#endif
+                    const int groups = cw / 8;
                     const int items = P.T * groups;
                     for (int item = etid; !dead && item < items; item += 128) {
                         const int rr = item / groups, cg = item % groups;
-                        const float4 a = *reinterpret_cast<const float4*>(stg + rr * STG_LD + cg * 8);
-                        const float4 b = *reinterpret_cast<const float4*>(stg + rr * STG_LD + cg * 8 + 4);
-                        const int col = c + cg * 8;            // 8-column groups never straddle the expert boundary
+                        const float4 a = *reinterpret_cast<const float4*>(stg + rr * ld + cg * 8);
+                        const float4 b = *reinterpret_cast<const float4*>(stg + rr * ld + cg * 8 + 4);
+                        const int col = c0 + cg * 8;           // 8-column groups never straddle the expert boundary
                         const bool second = col >= t.bn1;
                         const float g = second ? sh.gate2_s[rr] : sh.gate_s[rr];
                         const long long ocol = second ? (long long)t.out_col0_2 + (col - t.bn1) : (long long)t.out_col0 + col;
@@ -897,8 +939,10 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         __threadfence();
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (etid == 0) {
+            TRACE(9);
             grid_arrive(P.sync, 2);
             if (!grid_wait(P.sync, 2, G, &sh.abort_flag)) sh.abort_flag = 1;
+            TRACE(10);
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (!sh.abort_flag) {
@@ -961,6 +1005,12 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, TMEM_COLS);
     }
+#ifdef DSMOE_TRACE
+    if (threadIdx.x == 0 && blockIdx.x < 192) {
+        TRACE(11);
+        for (int i = 0; i < 32; ++i) g_trace[blockIdx.x][i] = sh.trace[i];
+    }
+#endif
     if (threadIdx.x == 0 && sh.abort_flag) {
         atomicExch(P.sync + 4, 1);
         if (P.dev_status) *P.dev_status = DSMOE_ERR_TIMEOUT;
@@ -1059,6 +1109,12 @@ dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams&
 }
 
 }  // namespace
+
+#ifdef DSMOE_TRACE
+extern "C" __attribute__((visibility("default"))) int dsmoe_trace_read(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(unsigned long long) * 192 * 32);
+}
+#endif
 
 void timing_reset() { g_timing.n = 0; }
 
