@@ -26,6 +26,8 @@ constexpr int BM = 128, BK = 64, BN = 256, STAGES = 4, MAX_STAGES = 16;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int NUM_THREADS = 192;
+constexpr int SMALL_THREADS = 448;    // small_layer_kernel: 2 + 4 warps as above, plus 8 warps that share the epilogue arithmetic
+constexpr int kEpiThreads = SMALL_THREADS - 64;
 constexpr int TMEM_COLS = 512;
 constexpr int RING_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);   // operand ring: 4 x 48 KB, or more, smaller slots
 constexpr int SHARED_BYTES = 3072 + 256;                                     // barriers and small tables (struct Shared)
@@ -533,7 +535,7 @@ __device__ __forceinline__ void small_issue(const SmallParams& P, const CUtensor
     }
 }
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(SMALL_THREADS, 1)
 small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ BMaps16 tmW1,
                    const __grid_constant__ CUtensorMap tmHg, const __grid_constant__ BMaps tmW2, const SmallParams P) {
     extern __shared__ uint8_t smem_raw[];
@@ -581,7 +583,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         const __nv_bfloat16* __restrict__ xr = P.x + (size_t)t * P.d;
         const float* __restrict__ Wr = P.Wr;
         const int quads = (E + 3) / 4;                  // threads per row
-        const int rpp = NUM_THREADS / quads;            // rows per pass
+        const int rpp = SMALL_THREADS / quads;            // rows per pass
         const int qd = threadIdx.x % quads, r0 = threadIdx.x / quads;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (threadIdx.x == 32) TRACE(12);
@@ -826,7 +828,8 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     } else {
         // ------------------------------------------------------------ epilogue (4 warps)
         const int q = warp & 3;
-        const int etid = (int)threadIdx.x - 64;
+        const int etid = (int)threadIdx.x - 64;         // 0 .. kEpiThreads-1
+        const bool tmem_warp = warp < 6;                 // warps 2..5 read TMEM; warps 6.. only share the arithmetic
         int acc = 0;
         uint32_t aph = 0;
         bool dead = aborted_early;     // a dead warp still takes part in every named barrier below
@@ -841,7 +844,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 // this CTA's part of hg is complete: publish it (the arriving thread's fence, after the barrier,
                 // covers the other threads' stores), then signal the up/down grid barrier
                 asm volatile("fence.proxy.async;" ::: "memory");
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
                 if (etid == 0) {
                     grid_arrive(P.sync, 1);
                     TRACE(7);
@@ -856,7 +859,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 sh.gate_s[etid] = ((mk >> t.e) & 1ull) ? P.scores[(long long)etid * P.E + t.e] : 0.f;
                 sh.gate2_s[etid] = ((mk >> t.e2) & 1ull) ? P.scores[(long long)etid * P.E + t.e2] : 0.f;
             }
-            if (!dead && !ptx::mbar_wait(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag)) dead = true;
+            if (tmem_warp && !dead && !ptx::mbar_wait(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag)) dead = true;
             dead = __any_sync(0xffffffffu, dead);     // the TMEM reads below are warp-collective
 #ifdef DSMOE_TRACE
             if (etid == 0 && t.phase == 0) TRACE(28);
@@ -871,7 +874,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 const int ld = CH + 4;                                                    // floats per staged row
                 for (int c0 = 0; c0 < t.bn; c0 += CH) {
                     const int cw = min(CH, t.bn - c0);
-                    if (!dead && q * 32 < P.T) {
+                    if (tmem_warp && !dead && q * 32 < P.T) {
                         for (int c = 0; c < cw; c += 32) {
                             uint32_t r[32];
                             ptx::tmem_ld32(taddr + (uint32_t)(c0 + c), r);
@@ -885,13 +888,13 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                             }
                         }
                     }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 #ifdef DSMOE_TRACE
                     if (etid == 0) TRACE(29 + (c0 > 0));
 #endif
                     const int groups = cw / 8;
                     const int items = P.T * groups;
-                    for (int item = etid; !dead && item < items; item += 128) {
+                    for (int item = etid; !dead && item < items; item += kEpiThreads) {
                         const int rr = item / groups, cg = item % groups;
                         const float4 a = *reinterpret_cast<const float4*>(stg + rr * ld + cg * 8);
                         const float4 b = *reinterpret_cast<const float4*>(stg + rr * ld + cg * 8 + 4);
@@ -907,11 +910,11 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                         hv[3] = __floats2bfloat162_rn(g * gelu_erf(b.z), g * gelu_erf(b.w));
                         *reinterpret_cast<uint4*>(P.hg + (long long)rr * ((long long)P.E * P.H) + ocol) = pk;
                     }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
                 }
             } else {
                 // fp32 partial sums of this CTA's share of the reduction: slot (cta, seg), row, 256 columns
-                for (int c = 0; !dead && q * 32 < P.T && c < t.bn; c += 32) {
+                for (int c = 0; tmem_warp && !dead && q * 32 < P.T && c < t.bn; c += 32) {
                     uint32_t r[32];
                     ptx::tmem_ld32(taddr + (uint32_t)c, r);
                     ptx::tmem_ld_wait();
@@ -928,7 +931,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             }
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0 && !dead) ptx::mbar_arrive(ptx::smem_u32(&sh.tempty[acc]));
+            if (tmem_warp && lane == 0 && !dead) ptx::mbar_arrive(ptx::smem_u32(&sh.tempty[acc]));
             if (++acc == 2) {
                 acc = 0;
                 aph ^= 1u;
@@ -937,14 +940,14 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         // ---- last grid barrier, then the fix-up: out[t,c] = sum of the partial tiles covering column c in
         // ascending CTA order (the partition arithmetic mirrors SmallIter)
         __threadfence();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
         if (etid == 0) {
             TRACE(9);
             grid_arrive(P.sync, 2);
             if (!grid_wait(P.sync, 2, G, &sh.abort_flag)) sh.abort_flag = 1;
             TRACE(10);
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
         if (!sh.abort_flag) {
             const int kbpe = P.H / BK;
             const int U = n_act * kbpe;
@@ -956,7 +959,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             // the additions, which run in ascending CTA order
             const int d4 = P.d / 4;
             const long long n_out4 = (long long)P.T * d4;
-            for (long long idx = (long long)blockIdx.x * 128 + etid; idx < n_out4; idx += (long long)G * 128) {
+            for (long long idx = (long long)blockIdx.x * kEpiThreads + etid; idx < n_out4; idx += (long long)G * kEpiThreads) {
                 const int tt = (int)(idx / d4), col = (int)(idx % d4) * 4;
                 const int r = col / bnd, cc = col % bnd;
                 float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1237,7 +1240,7 @@ dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const 
     void* args[] = {&ms->mX, &ms->mW1, &ms->mHg, &ms->mW2, &P};
     const bool timed = g_timing.on && g_timing.n < kMaxTimed;
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
-    DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(small_layer_kernel), dim3(G), dim3(NUM_THREADS),
+    DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(small_layer_kernel), dim3(G), dim3(SMALL_THREADS),
                                                args, SMEM_BYTES, s));
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.stop[g_timing.n++], s));
     return DSMOE_OK;
