@@ -535,6 +535,23 @@ __device__ __forceinline__ void small_issue(const SmallParams& P, const CUtensor
     }
 }
 
+// Ring geometry for n selected experts.  A slot holds the tokens' 64-wide block and one weight tile.  With few
+// selected experts the tiles are narrow, so the down-projection takes narrower column ranges too and the ring
+// has more slots: more loads in flight, which is what hides memory latency when each load is small.
+struct SmallGeo {
+    int up_rows, bn_down, a_bytes, slot_bytes, n_stages;
+};
+__device__ __forceinline__ SmallGeo small_geometry(const SmallParams& P, int n, int G) {
+    SmallGeo g;
+    const int up_units = (n * (P.H / kUpUnit) + G - 1) / G;
+    g.up_rows = max(1, min(up_units, kUpTileUnits)) * kUpUnit;
+    g.bn_down = g.up_rows <= 64 ? 64 : g.up_rows <= 128 ? 128 : BN;
+    g.a_bytes = P.t_pad * BK * 2;
+    g.slot_bytes = g.a_bytes + g.bn_down * BK * 2;
+    g.n_stages = min(MAX_STAGES, RING_BYTES / g.slot_bytes);
+    return g;
+}
+
 __global__ void __launch_bounds__(SMALL_THREADS, 1)
 small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ BMaps16 tmW1,
                    const __grid_constant__ CUtensorMap tmHg, const __grid_constant__ BMaps tmW2, const SmallParams P) {
@@ -675,16 +692,12 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         for (int e = 0; e < P.E; ++e)
             if ((m >> e) & 1ull) sh.active[n++] = e;
         sh.n_act = n;
-        // Ring geometry: a slot holds the tokens' 64-wide block and one weight tile.  With few selected experts
-        // the tiles are narrow, so the down-projection takes narrower column ranges too and the ring has more
-        // slots: more loads in flight, which is what hides memory latency when each load is small.
-        const int up_units = (n * (P.H / kUpUnit) + G - 1) / G;
-        const int up_rows = max(1, min(up_units, kUpTileUnits)) * kUpUnit;
-        sh.bn_down = up_rows <= 64 ? 64 : up_rows <= 128 ? 128 : BN;
-        sh.a_bytes = P.t_pad * BK * 2;
-        sh.slot_bytes = sh.a_bytes + sh.bn_down * BK * 2;
-        sh.n_stages = min(MAX_STAGES, RING_BYTES / sh.slot_bytes);
-        ptx::prefetch_tensormap(&tmW1.m[up_rows / 16 - 1]);
+        const SmallGeo g = small_geometry(P, n, G);
+        sh.bn_down = g.bn_down;
+        sh.a_bytes = g.a_bytes;
+        sh.slot_bytes = g.slot_bytes;
+        sh.n_stages = g.n_stages;
+        ptx::prefetch_tensormap(&tmW1.m[g.up_rows / 16 - 1]);
     }
     __syncthreads();
     const uint32_t tmem_base = sh.tmem_base;
@@ -959,7 +972,10 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             // the additions, which run in ascending CTA order
             const int d4 = P.d / 4;
             const long long n_out4 = (long long)P.T * d4;
-            for (long long idx = (long long)blockIdx.x * kEpiThreads + etid; idx < n_out4; idx += (long long)G * kEpiThreads) {
+            const long long per_cta = (n_out4 + G - 1) / G;     // an equal share for every CTA
+            for (long long j = etid; j < per_cta; j += kEpiThreads) {
+                const long long idx = (long long)blockIdx.x * per_cta + j;
+                if (idx >= n_out4) break;
                 const int tt = (int)(idx / d4), col = (int)(idx % d4) * 4;
                 const int r = col / bnd, cc = col % bnd;
                 float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);

@@ -115,3 +115,24 @@ def test_c5_skewed_router_threshold_sweep(eps):
         assert r["empty_experts"] > 0 or r["zero_tokens"] > 0
     # rows differ wildly in scale here (1 to 64 experts per token): the bar is applied per token
     assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
+
+
+# ---------------------------------------------------------------- decode path corner cases
+# The decode kernel streams only the experts that some token selected and cuts that list evenly over
+# the CTAs: few, no, skewed and all experts selected.
+
+@pytest.mark.parametrize("case", [
+    dict(T=24, E=32, mode=gi.MODE_TOPK, K=1),                       # at most 24 of 32 experts selected
+    dict(T=16, E=16, mode=gi.MODE_THRESHOLD, eps=0.4),              # a few experts, many tokens with none
+    dict(T=40, E=8, mode=gi.MODE_THRESHOLD, eps=0.999),             # no expert at all: the output is zero
+    dict(T=128, E=64, mode=gi.MODE_TOPK, K=2, zipf_s=1.1),          # skewed: popular experts only
+    dict(T=17, E=4, mode=gi.MODE_ALL),                              # every expert (the assumption holds)
+], ids=["topk1", "few", "none", "skew", "all"])
+def test_decode_path_when_some_experts_are_unselected(case):
+    s = gi.LayerSpec("dec_" + str(case["T"]), d=512, H=256, dtype="bf16", router_gain=8.0, **case)
+    r = layer_parity(s)
+    assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
+    if case.get("eps") == 0.999:
+        assert r["A"] == 0 and np.all(np_f32(r["layer"].out) == 0.0)
+    if case["mode"] == gi.MODE_TOPK and case["K"] == 1:
+        assert r["empty_experts"] >= 8
