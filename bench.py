@@ -169,6 +169,21 @@ def oracle_tokens_per_s(s: gi.LayerSpec, budget_s: float, steps=None, warmup=0):
 # GPU arm
 # --------------------------------------------------------------------------------------------
 
+def job_throughput(dist, ms_local: float, tokens_local: int, device="cuda"):
+    """Whole-job tokens/s of a token-sharded run: every rank processed `tokens_local` tokens of its own
+    in `ms_local`; the job took as long as its slowest rank.  No data-path collective exists (each token's
+    output depends on its own x and on replicated weights), only this reduction of the timing."""
+    import torch
+    if dist is None:
+        return tokens_local / (ms_local * 1e-3), ms_local, 1
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    n = torch.tensor([float(tokens_local)], dtype=torch.float64, device=device)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    ms = float(t.item())
+    return float(n.item()) / (ms * 1e-3), ms, dist.get_world_size()
+
+
 def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, sampler_index=0):
     import torch
     import paper_2404_05567_b200 as dm
@@ -239,12 +254,7 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
     barrier()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.finish()
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-    world = dist.get_world_size() if dist is not None else 1
-    value = world * s.T * steps / (ms_total * 1e-3)
+    value, ms_total, world = job_throughput(dist, ms_total, s.T * steps)
 
     # ---- per-launch time of the dominant kernel (the tcgen05 expert GEMM), CUDA events inside the library
     dm.dsmoe_timing_enable(True)
@@ -297,12 +307,9 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
         e1.record()
         barrier()
         ms_e2e = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms_e2e], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        e2e_value, ms_e2e, _ = job_throughput(dist, ms_e2e, s.T * steps)
         nbytes = s.T * s.d * 2
-        res["e2e"] = {"value": world * s.T * steps / (ms_e2e * 1e-3), "unit": "tokens/s",
+        res["e2e"] = {"value": e2e_value, "unit": "tokens/s",
                       "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes}
     del packed, ws
     torch.cuda.empty_cache()
