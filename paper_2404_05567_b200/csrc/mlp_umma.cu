@@ -41,6 +41,7 @@ constexpr int kUpUnit = 16;          // small-T up-projection: weight rows per w
 constexpr int kUpTileUnits = 16;     // ... and units per tile (256 rows)
 constexpr int kRouterBatch = 12;     // rows of Wr a router thread loads at once
 constexpr int kFixBatch = 24;        // partial tiles a fix-up thread loads at once
+constexpr int kSpecMinT = 16;        // tokens from which the small-T kernel streams ahead of its router
 
 struct GemmParams {
     int mode, epi;
@@ -72,18 +73,29 @@ struct Tile {
     int row0, rows_valid, e, n0, bn, nk, out_col0;
 };
 
+// small_layer_kernel: the selected experts and the work partition and ring geometry that follow from them
+struct SmallGeo {
+    int n_act;                           // experts selected by at least one token
+    int up_rows, bn_down;                // widest up-projection tile; column-range width of the down-projection
+    int a_bytes, slot_bytes, n_stages;   // ring: token block + weight tile per slot
+    int active[kMaxExperts];             // their indices, ascending
+};
+
 struct Shared {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2];
+    uint64_t drain;                      // small_layer_kernel: "every MMA on speculative tiles has completed"
     uint32_t tmem_base;
     volatile int abort_flag;
     int bad_offsets;
-    int n_stages, slot_bytes, a_bytes;   // ring geometry (small_layer_kernel)
-    int bn_down;                         // small_layer_kernel: column-range width of the down-projection
     int tile_prefix[kMaxExperts + 1];
     int seg0[kMaxExperts], seg1[kMaxExperts];
-    unsigned long long active_mask;      // experts selected by at least one token
-    int n_act;
-    int active[kMaxExperts];
+    unsigned long long active_mask;
+    // small_layer_kernel: geo[0] assumes every expert selected (streaming starts under it while the router still
+    // runs), geo[1] is what the router found.  geo_state: 0 router pending, 1 geo[1] equals geo[0], 2 it differs.
+    SmallGeo geo[2];
+    volatile int geo_state;
+    volatile int spec_issued, spec_stop;   // producer -> MMA issuer: ring slots filled under geo[0]; no more will be
+    volatile int mma_drained;              // MMA issuer -> producer: those slots are consumed, the ring is idle
     float gate_s[BM], gate2_s[BM];
 #ifdef DSMOE_TRACE
     unsigned long long trace[32];
@@ -404,6 +416,7 @@ struct SmallParams {
     void* out;
     int out_f32;
     int* sync;               // 8 ints, zero at launch: four barrier counters [0..3] and an abort flag [4]
+    int spec;                // start streaming under "every expert selected" before the router has finished
     int32_t* dev_status;
 };
 
@@ -538,18 +551,43 @@ __device__ __forceinline__ void small_issue(const SmallParams& P, const CUtensor
 // Ring geometry for n selected experts.  A slot holds the tokens' 64-wide block and one weight tile.  With few
 // selected experts the tiles are narrow, so the down-projection takes narrower column ranges too and the ring
 // has more slots: more loads in flight, which is what hides memory latency when each load is small.
-struct SmallGeo {
-    int up_rows, bn_down, a_bytes, slot_bytes, n_stages;
-};
-__device__ __forceinline__ SmallGeo small_geometry(const SmallParams& P, int n, int G) {
-    SmallGeo g;
+__device__ __forceinline__ void small_geometry(const SmallParams& P, int n, int G, SmallGeo& g) {
     const int up_units = (n * (P.H / kUpUnit) + G - 1) / G;
+    g.n_act = n;
     g.up_rows = max(1, min(up_units, kUpTileUnits)) * kUpUnit;
     g.bn_down = g.up_rows <= 64 ? 64 : g.up_rows <= 128 ? 128 : BN;
     g.a_bytes = P.t_pad * BK * 2;
     g.slot_bytes = g.a_bytes + g.bn_down * BK * 2;
     g.n_stages = min(MAX_STAGES, RING_BYTES / g.slot_bytes);
-    return g;
+}
+
+// Bounded wait for the router's verdict on the speculative geometry; 0 = gave up.
+__device__ __forceinline__ int wait_geo(Shared& sh) {
+    const uint64_t t0 = ptx::globaltimer_ns();
+    for (uint32_t spin = 0;; ++spin) {
+        const int st = sh.geo_state;
+        if (st) return st;
+        if ((spin & 0xff) == 0xff) {
+            if (sh.abort_flag) return 0;
+            if (ptx::globaltimer_ns() - t0 > ptx::kWaitLimitNs) {
+                sh.abort_flag = 1;
+                return 0;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool wait_flag(volatile int* flag, Shared& sh) {
+    const uint64_t t0 = ptx::globaltimer_ns();
+    for (uint32_t spin = 0;; ++spin) {
+        if (*flag) return true;
+        if ((spin & 0xff) == 0xff) {
+            if (sh.abort_flag) return false;
+            if (ptx::globaltimer_ns() - t0 > ptx::kWaitLimitNs) {
+                sh.abort_flag = 1;
+                return false;
+            }
+        }
+    }
 }
 
 __global__ void __launch_bounds__(SMALL_THREADS, 1)
@@ -572,8 +610,14 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             ptx::mbar_init(ptx::smem_u32(&sh.tfull[a]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.tempty[a]), 4);
         }
+        ptx::mbar_init(ptx::smem_u32(&sh.drain), 1);
         sh.abort_flag = 0;
         sh.active_mask = 0ull;
+        sh.geo_state = 0;
+        sh.spec_issued = 0;
+        sh.spec_stop = 0;
+        sh.mma_drained = 0;
+        small_geometry(P, P.E, G, sh.geo[0]);
 #ifdef DSMOE_TRACE
         for (int i = 0; i < 32; ++i) sh.trace[i] = 0;
         TRACE(0);
@@ -581,183 +625,124 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&tmX);
         ptx::prefetch_tensormap(&tmHg);
+        ptx::prefetch_tensormap(&tmW1.m[sh.geo[0].up_rows / 16 - 1]);
         for (int i = 2; i < 5; ++i) ptx::prefetch_tensormap(&tmW2.m[i]);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), TMEM_COLS);
         ptx::tmem_relinquish();
     }
-
-    // ------------------------------------------------------------ router, step 1
-    // The reduction over d of every token is cut into KS slices, one CTA per (token, slice).  A row of Wr
-    // (E floats) is covered by E/4 neighbouring threads with one 16-byte load each, so a warp reads whole
-    // rows, coalesced, and a thread keeps only its four experts' sums over every rpp-th row; all its loads are
-    // independent.  The threads' sums meet in shared memory.
-    const int KS = max(1, min(16, G / P.T));
-    if ((int)blockIdx.x < P.T * KS) {
-        const int t = blockIdx.x / KS, sl = blockIdx.x % KS, E = P.E;
-        const int klen = (P.d + KS - 1) / KS, kbeg = sl * klen, kend = min(P.d, kbeg + klen);
-        const __nv_bfloat16* __restrict__ xr = P.x + (size_t)t * P.d;
-        const float* __restrict__ Wr = P.Wr;
-        const int quads = (E + 3) / 4;                  // threads per row
-        const int rpp = SMALL_THREADS / quads;            // rows per pass
-        const int qd = threadIdx.x % quads, r0 = threadIdx.x / quads;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (threadIdx.x == 32) TRACE(12);
-        if (r0 < rpp) {
-            if ((E & 3) == 0) {
-                // batches of kRouterBatch rows: every load of a batch is issued before its first use
-                for (int kb = kbeg + r0; kb < kend; kb += kRouterBatch * rpp) {
-                    float4 w[kRouterBatch];
-                    float xs[kRouterBatch];
-#pragma unroll
-                    for (int j = 0; j < kRouterBatch; ++j) {
-                        const int k = kb + j * rpp;
-                        const bool ok = k < kend;
-                        w[j] = ok ? __ldg(reinterpret_cast<const float4*>(Wr + (size_t)k * E) + qd) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        xs[j] = ok ? __bfloat162float(xr[k]) : 0.f;
-                    }
-#pragma unroll
-                    for (int j = 0; j < kRouterBatch; ++j) {
-                        acc.x = fmaf(xs[j], w[j].x, acc.x);
-                        acc.y = fmaf(xs[j], w[j].y, acc.y);
-                        acc.z = fmaf(xs[j], w[j].z, acc.z);
-                        acc.w = fmaf(xs[j], w[j].w, acc.w);
-                    }
-                }
-            } else {
-                const int e0 = qd * 4;
-                for (int k = kbeg + r0; k < kend; k += rpp) {
-                    const float xv = __bfloat162float(xr[k]);
-                    const float* w = Wr + (size_t)k * E + e0;
-                    acc.x = fmaf(xv, __ldg(w), acc.x);
-                    if (e0 + 1 < E) acc.y = fmaf(xv, __ldg(w + 1), acc.y);
-                    if (e0 + 2 < E) acc.z = fmaf(xv, __ldg(w + 2), acc.z);
-                    if (e0 + 3 < E) acc.w = fmaf(xv, __ldg(w + 3), acc.w);
-                }
-            }
-        }
-        if (threadIdx.x == 32) TRACE(13);
-        reinterpret_cast<float4*>(stg)[threadIdx.x] = acc;      // stg[(r0 * quads + qd) * 4 + j]
-        __syncthreads();
-        if ((int)threadIdx.x < E) {
-            const int e = threadIdx.x;
-            float v = 0.f;
-            for (int r = 0; r < rpp; ++r) v += stg[(r * quads + (e >> 2)) * 4 + (e & 3)];
-            P.partial[((size_t)t * KS + sl) * kMaxExperts + e] = v;   // the partial-sum buffer is free until the down-projection
-        }
-    }
+    if (warp >= 2 && (int)threadIdx.x - 64 < kMaxExperts) sh.geo[0].active[threadIdx.x - 64] = (int)threadIdx.x - 64;
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
-    if (threadIdx.x == 0) {
-        TRACE(1);
-        grid_arrive(P.sync, 0);
-        grid_wait(P.sync, 0, G, &sh.abort_flag);
-        TRACE(14);
-    }
-    __syncthreads();
-    // ------------------------------------------------------------ router, step 2
-    // CTA t adds the slices of token t in a fixed order; softmax and selection in one warp
-    if ((int)blockIdx.x < P.T && warp == 0 && !sh.abort_flag) {
-        const int t = blockIdx.x, E = P.E;
-        const bool v_lo = lane < E, v_hi = lane + 32 < E;
-        float l_lo = (P.br && v_lo) ? P.br[lane] : 0.f, l_hi = (P.br && v_hi) ? P.br[lane + 32] : 0.f;
-        for (int sl = 0; sl < KS; ++sl) {
-            const float* pl = P.partial + ((size_t)t * KS + sl) * kMaxExperts;
-            if (v_lo) l_lo += __ldcg(pl + lane);
-            if (v_hi) l_hi += __ldcg(pl + lane + 32);
-        }
-        softmax_select_store(l_lo, l_hi, t, P.sel, lane, P.scores, P.mask, P.k_t);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        TRACE(15);
-        grid_arrive(P.sync, 3);
-        grid_wait(P.sync, 3, G, &sh.abort_flag);
-        TRACE(2);
-    }
-    __syncthreads();
-    // every CTA derives the set of selected experts from the T selection words
-    if ((int)threadIdx.x < P.T) {
-        unsigned long long m;
-        asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(m) : "l"(P.mask + threadIdx.x) : "memory");
-        atomicOr(&sh.active_mask, m);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        unsigned long long m = sh.active_mask;
-        if (P.E < 64) m &= (1ull << P.E) - 1ull;
-        int n = 0;
-        for (int e = 0; e < P.E; ++e)
-            if ((m >> e) & 1ull) sh.active[n++] = e;
-        sh.n_act = n;
-        const SmallGeo g = small_geometry(P, n, G);
-        sh.bn_down = g.bn_down;
-        sh.a_bytes = g.a_bytes;
-        sh.slot_bytes = g.slot_bytes;
-        sh.n_stages = g.n_stages;
-        ptx::prefetch_tensormap(&tmW1.m[g.up_rows / 16 - 1]);
-    }
-    __syncthreads();
     const uint32_t tmem_base = sh.tmem_base;
-    const int n_act = sh.n_act, n_stages = sh.n_stages;
-    const uint32_t slot_bytes = (uint32_t)sh.slot_bytes, a_bytes = (uint32_t)sh.a_bytes;
-    const uint32_t smA = base, smB = base + a_bytes;
-    const bool aborted_early = sh.abort_flag != 0;
-    if (threadIdx.x == 0) TRACE(3);
+    const uint32_t smA = base;
 
+    // From here the three roles run side by side.  Warps 2.. compute the router (two grid barriers) and publish the
+    // geometry it implies in geo[1]; warps 0 and 1 either wait for that, or (P.spec) start streaming and multiplying
+    // the up-projection at once under geo[0], "every expert selected" -- the products x.W1 do not depend on the
+    // router, only the partition of the work does.  If the router confirms geo[0] they simply carry on; if not,
+    // the producer stops, the MMA issuer consumes what was loaded and waits for its products to retire, and both
+    // start over under geo[1].  Ring slots keep one phase bit each (phb), so the ring may change its slot count
+    // at that point without touching the barriers.
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0 && !aborted_early) {
+        if (lane == 0) {
             int s = 0;
-            uint32_t ph = 0;
-            bool alive = true;
-            SmallIter it;
-            it.init(P, n_act, sh.bn_down);
-            SmallTile t;
-            bool have = it.next(P, sh.active, n_act, t);
-            // up-projection
-            while (alive && have && t.phase == 0) {
-                for (int i = 0; i < t.nk; ++i) {
-                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
-                        alive = false;
-                        break;
-                    }
-                    const uint32_t bar = ptx::smem_u32(&sh.full[s]);
-                    ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
-                    small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, sh.active, t, i, smA + s * slot_bytes, smB + s * slot_bytes, bar, 3);
-                    if (++s == n_stages) {
-                        s = 0;
-                        ph ^= 1u;
-                    }
-                }
-                have = it.next(P, sh.active, n_act, t);
+            uint32_t phb = 0;
+            bool alive = true, spec = P.spec != 0;
+            const SmallGeo* g = &sh.geo[0];
+            if (!spec) {
+                alive = wait_geo(sh) != 0;
+                g = &sh.geo[1];
             }
+            SmallIter it;
+            SmallTile t;
+            bool have = false;
+            int n_stages = 1;
+            uint32_t slot_bytes = 0, a_bytes = 0, smB = 0;
+            for (int pass = 0; alive && pass < 2; ++pass) {
+                n_stages = g->n_stages;
+                slot_bytes = (uint32_t)g->slot_bytes;
+                a_bytes = (uint32_t)g->a_bytes;
+                smB = base + a_bytes;
+                it.init(P, g->n_act, g->bn_down);
+                have = it.next(P, g->active, g->n_act, t);
+                int issued = 0;
+                bool replaced = false;
+                // up-projection
+                while (alive && have && t.phase == 0 && !replaced) {
+                    for (int i = 0; i < t.nk; ++i) {
+                        const uint32_t ebar = ptx::smem_u32(&sh.empty[s]), epar = ((phb >> s) & 1u) ^ 1u;
+                        if (spec) {
+                            // the slot may never come back: once the router disagrees, the MMA issuer stops too
+                            const uint64_t t0 = ptx::globaltimer_ns();
+                            for (uint32_t spin = 1; !ptx::mbar_try_wait(ebar, epar); ++spin) {
+                                if (sh.geo_state == 2) break;
+                                if ((spin & 0xff) == 0 && (sh.abort_flag || ptx::globaltimer_ns() - t0 > ptx::kWaitLimitNs)) {
+                                    sh.abort_flag = 1;
+                                    alive = false;
+                                    break;
+                                }
+                            }
+                            if (!alive) break;
+                            if (sh.geo_state == 2) {
+                                replaced = true;
+                                break;
+                            }
+                        } else if (!ptx::mbar_wait(ebar, epar, &sh.abort_flag)) {
+                            alive = false;
+                            break;
+                        }
+                        const uint32_t bar = ptx::smem_u32(&sh.full[s]);
+                        ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
+                        small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, t, i, smA + s * slot_bytes, smB + s * slot_bytes, bar, 3);
+                        phb ^= 1u << s;
+                        ++issued;
+                        if (++s == n_stages) s = 0;
+                    }
+                    if (!alive || replaced) break;
+                    have = it.next(P, g->active, g->n_act, t);
+                }
+                if (alive && spec && !replaced) {
+                    // the down-projection's partition needs the router's result
+                    const int st = wait_geo(sh);
+                    if (st == 0) alive = false;
+                    else if (st == 2) replaced = true;
+                }
+                if (!(alive && replaced)) break;
+                sh.spec_issued = issued;
+                __threadfence_block();
+                sh.spec_stop = 1;
+                if (!wait_flag(&sh.mma_drained, sh)) alive = false;
+                spec = false;
+                g = &sh.geo[1];
+                s = 0;
+            }
+            TRACE(3);
             // down-projection: weight tiles first, for as many slots as the ring has; their hg tiles follow
             // once every CTA has finished writing hg
             SmallTile pend_t[MAX_STAGES];
             int pend_i[MAX_STAGES], pend_s[MAX_STAGES];
             int npend = 0, i_cur = 0;
             while (alive && have && npend < n_stages) {
-                if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
+                if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ((phb >> s) & 1u) ^ 1u, &sh.abort_flag)) {
                     alive = false;
                     break;
                 }
                 const uint32_t bar = ptx::smem_u32(&sh.full[s]);
                 ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
-                small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, sh.active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 2);
+                small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 2);
                 pend_t[npend] = t;
                 pend_i[npend] = i_cur;
                 pend_s[npend] = s;
                 ++npend;
-                if (++s == n_stages) {
-                    s = 0;
-                    ph ^= 1u;
-                }
+                phb ^= 1u << s;
+                if (++s == n_stages) s = 0;
                 if (++i_cur == t.nk) {
                     i_cur = 0;
-                    have = it.next(P, sh.active, n_act, t);
+                    have = it.next(P, g->active, g->n_act, t);
                 }
             }
             TRACE(5);
@@ -765,25 +750,23 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             TRACE(6);
             asm volatile("fence.proxy.async;" ::: "memory");   // hg was written through the generic proxy, TMA reads it
             for (int j = 0; alive && j < npend; ++j)
-                small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, sh.active, pend_t[j], pend_i[j], smA + pend_s[j] * slot_bytes,
+                small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, pend_t[j], pend_i[j], smA + pend_s[j] * slot_bytes,
                             smB + pend_s[j] * slot_bytes, ptx::smem_u32(&sh.full[pend_s[j]]), 1);
             while (alive && have) {
                 for (; i_cur < t.nk; ++i_cur) {
-                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ((phb >> s) & 1u) ^ 1u, &sh.abort_flag)) {
                         alive = false;
                         break;
                     }
                     const uint32_t bar = ptx::smem_u32(&sh.full[s]);
                     ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
-                    small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, sh.active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 3);
-                    if (++s == n_stages) {
-                        s = 0;
-                        ph ^= 1u;
-                    }
+                    small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 3);
+                    phb ^= 1u << s;
+                    if (++s == n_stages) s = 0;
                 }
                 if (!alive) break;
                 i_cur = 0;
-                have = it.next(P, sh.active, n_act, t);
+                have = it.next(P, g->active, g->n_act, t);
             }
             if (!alive) {
                 const uint64_t t0 = ptx::globaltimer_ns();   // copies already issued still land in this CTA's smem
@@ -793,71 +776,259 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && !aborted_early) {
+        if (lane == 0) {
             int s = 0, acc = 0;
-            uint32_t ph = 0, aph = 0;
-            bool alive = true;
-            SmallIter it;
-            it.init(P, n_act, sh.bn_down);
-            SmallTile t;
-            while (alive && it.next(P, sh.active, n_act, t)) {
-                if (!ptx::mbar_wait(ptx::smem_u32(&sh.tempty[acc]), aph ^ 1u, &sh.abort_flag)) break;
-                ptx::tc_fence_after();
-                const uint32_t idesc = ptx::make_idesc_bf16(BM, (uint32_t)t.bn);
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                for (int i = 0; i < t.nk; ++i) {
-                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.full[s]), ph, &sh.abort_flag)) {
+            uint32_t phb = 0, aph = 0;
+            bool alive = true, spec = P.spec != 0;
+            const SmallGeo* g = &sh.geo[0];
+            if (!spec) {
+                alive = wait_geo(sh) != 0;
+                g = &sh.geo[1];
+            }
+            for (int pass = 0; alive && pass < 2; ++pass) {
+                const int n_stages = g->n_stages;
+                const uint32_t slot_bytes = (uint32_t)g->slot_bytes, smB = base + (uint32_t)g->a_bytes;
+                int consumed = 0;
+                bool redo = false;
+                SmallIter it;
+                it.init(P, g->n_act, g->bn_down);
+                SmallTile t;
+                while (alive && !redo && it.next(P, g->active, g->n_act, t)) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.tempty[acc]), aph ^ 1u, &sh.abort_flag)) {
                         alive = false;
                         break;
                     }
-#ifdef DSMOE_TRACE
-                    if (sh.trace[4] == 0) TRACE(4);
-                    if (t.phase == 1 && sh.trace[8] == 0) TRACE(8);
-                    if (t.phase == 0 && i < 8) TRACE(16 + i);
-                    if (t.phase == 0 && i >= t.nk - 4) TRACE(24 + i - (t.nk - 4));
-#endif
                     ptx::tc_fence_after();
-                    // M = 128 although only t_pad rows were loaded: the rows beyond are whatever the ring holds,
-                    // they only reach TMEM lanes that nobody reads
-                    const uint32_t a0 = smA + s * slot_bytes, b0 = smB + s * slot_bytes;
+                    const uint32_t idesc = ptx::make_idesc_bf16(BM, (uint32_t)t.bn);
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                    for (int i = 0; i < t.nk; ++i) {
+                        const uint32_t fbar = ptx::smem_u32(&sh.full[s]), par = (phb >> s) & 1u;
+                        if (spec) {
+                            // like mbar_wait, but the slot may never be filled: the producer stops when the router
+                            // disagrees with the speculative geometry
+                            const uint64_t t0 = ptx::globaltimer_ns();
+                            for (uint32_t spin = 1; !ptx::mbar_try_wait(fbar, par); ++spin) {
+                                if (sh.spec_stop && consumed == sh.spec_issued) {
+                                    redo = true;
+                                    break;
+                                }
+                                if ((spin & 0xff) == 0 && (sh.abort_flag || ptx::globaltimer_ns() - t0 > ptx::kWaitLimitNs)) {
+                                    sh.abort_flag = 1;
+                                    alive = false;
+                                    break;
+                                }
+                            }
+                            if (redo || !alive) break;
+                        } else if (!ptx::mbar_wait(fbar, par, &sh.abort_flag)) {
+                            alive = false;
+                            break;
+                        }
+#ifdef DSMOE_TRACE
+                        if (sh.trace[4] == 0) TRACE(4);
+                        if (t.phase == 1 && sh.trace[8] == 0) TRACE(8);
+                        if (t.phase == 0 && i < 8) TRACE(16 + i);
+                        if (t.phase == 0 && i >= t.nk - 4) TRACE(24 + i - (t.nk - 4));
+#endif
+                        ptx::tc_fence_after();
+                        // M = 128 although only t_pad rows were loaded: the rows beyond are whatever the ring holds,
+                        // they only reach TMEM lanes that nobody reads
+                        const uint32_t a0 = smA + s * slot_bytes, b0 = smB + s * slot_bytes;
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        ptx::umma_bf16(d_tmem, ptx::make_desc_k_sw128(a0 + k * 32), ptx::make_desc_k_sw128(b0 + k * 32),
-                                       idesc, (uint32_t)((i | k) != 0));
-                    ptx::umma_commit(ptx::smem_u32(&sh.empty[s]));
-                    if (++s == n_stages) {
-                        s = 0;
-                        ph ^= 1u;
+                        for (int k = 0; k < BK / 16; ++k)
+                            ptx::umma_bf16(d_tmem, ptx::make_desc_k_sw128(a0 + k * 32), ptx::make_desc_k_sw128(b0 + k * 32),
+                                           idesc, (uint32_t)((i | k) != 0));
+                        ptx::umma_commit(ptx::smem_u32(&sh.empty[s]));
+                        phb ^= 1u << s;
+                        ++consumed;
+                        if (++s == n_stages) s = 0;
+                    }
+                    if (!alive || redo) break;
+                    if (spec) {
+                        // a finished tile goes to the epilogue only once the router has confirmed its geometry
+                        const int st = wait_geo(sh);
+                        if (st == 0) {
+                            alive = false;
+                            break;
+                        }
+                        if (st == 2) {
+                            redo = true;
+                            break;
+                        }
+                        spec = false;
+                    }
+                    ptx::umma_commit(ptx::smem_u32(&sh.tfull[acc]));
+                    if (++acc == 2) {
+                        acc = 0;
+                        aph ^= 1u;
                     }
                 }
-                if (!alive) break;
-                ptx::umma_commit(ptx::smem_u32(&sh.tfull[acc]));
-                if (++acc == 2) {
-                    acc = 0;
-                    aph ^= 1u;
+                if (alive && !redo && spec) {
+                    // a CTA without work under geo[0] may have some under geo[1]; the producer waits for this thread either way
+                    const int st = wait_geo(sh);
+                    if (st == 0) alive = false;
+                    else if (st == 2) redo = true;
+                    spec = false;
                 }
+                if (!(alive && redo)) break;
+                // take the remaining speculative loads off the ring, let the products issued so far retire, then
+                // tell the producer that the ring is idle
+                if (!wait_flag(&sh.spec_stop, sh)) break;
+                const int issued = sh.spec_issued;
+                while (alive && consumed < issued) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.full[s]), (phb >> s) & 1u, &sh.abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    ptx::mbar_arrive(ptx::smem_u32(&sh.empty[s]));
+                    phb ^= 1u << s;
+                    ++consumed;
+                    if (++s == n_stages) s = 0;
+                }
+                if (!alive) break;
+                ptx::umma_commit(ptx::smem_u32(&sh.drain));
+                if (!ptx::mbar_wait(ptx::smem_u32(&sh.drain), 0u, &sh.abort_flag)) break;
+                __threadfence_block();
+                sh.mma_drained = 1;
+                spec = false;
+                g = &sh.geo[1];
+                s = 0;
+                acc = 0;
+                aph = 0;
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (4 warps)
-        const int q = warp & 3;
+        // ------------------------------------------------------------ router, then epilogue (12 warps)
         const int etid = (int)threadIdx.x - 64;         // 0 .. kEpiThreads-1
+#define EPI_SYNC() asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory")
+        // ---- router, step 1
+        // The reduction over d of every token is cut into KS slices, one CTA per (token, slice).  A row of Wr
+        // (E floats) is covered by E/4 neighbouring threads with one 16-byte load each, so a warp reads whole
+        // rows, coalesced, and a thread keeps only its four experts' sums over every rpp-th row; all its loads are
+        // independent.  The threads' sums meet in shared memory.
+        const int KS = max(1, min(16, G / P.T));
+        if ((int)blockIdx.x < P.T * KS) {
+            const int t = blockIdx.x / KS, sl = blockIdx.x % KS, E = P.E;
+            const int klen = (P.d + KS - 1) / KS, kbeg = sl * klen, kend = min(P.d, kbeg + klen);
+            const __nv_bfloat16* __restrict__ xr = P.x + (size_t)t * P.d;
+            const float* __restrict__ Wr = P.Wr;
+            const int quads = (E + 3) / 4;                  // threads per row
+            const int rpp = kEpiThreads / quads;            // rows per pass
+            const int qd = etid % quads, r0 = etid / quads;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (etid == 0) TRACE(12);
+            if (r0 < rpp) {
+                if ((E & 3) == 0) {
+                    // batches of kRouterBatch rows: every load of a batch is issued before its first use
+                    for (int kb = kbeg + r0; kb < kend; kb += kRouterBatch * rpp) {
+                        float4 w[kRouterBatch];
+                        float xs[kRouterBatch];
+#pragma unroll
+                        for (int j = 0; j < kRouterBatch; ++j) {
+                            const int k = kb + j * rpp;
+                            const bool ok = k < kend;
+                            w[j] = ok ? __ldg(reinterpret_cast<const float4*>(Wr + (size_t)k * E) + qd) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            xs[j] = ok ? __bfloat162float(xr[k]) : 0.f;
+                        }
+#pragma unroll
+                        for (int j = 0; j < kRouterBatch; ++j) {
+                            acc.x = fmaf(xs[j], w[j].x, acc.x);
+                            acc.y = fmaf(xs[j], w[j].y, acc.y);
+                            acc.z = fmaf(xs[j], w[j].z, acc.z);
+                            acc.w = fmaf(xs[j], w[j].w, acc.w);
+                        }
+                    }
+                } else {
+                    const int e0 = qd * 4;
+                    for (int k = kbeg + r0; k < kend; k += rpp) {
+                        const float xv = __bfloat162float(xr[k]);
+                        const float* w = Wr + (size_t)k * E + e0;
+                        acc.x = fmaf(xv, __ldg(w), acc.x);
+                        if (e0 + 1 < E) acc.y = fmaf(xv, __ldg(w + 1), acc.y);
+                        if (e0 + 2 < E) acc.z = fmaf(xv, __ldg(w + 2), acc.z);
+                        if (e0 + 3 < E) acc.w = fmaf(xv, __ldg(w + 3), acc.w);
+                    }
+                }
+            }
+            if (etid == 0) TRACE(13);
+            reinterpret_cast<float4*>(stg)[etid] = acc;      // stg[(r0 * quads + qd) * 4 + j]
+            EPI_SYNC();
+            if (etid < E) {
+                const int e = etid;
+                float v = 0.f;
+                for (int r = 0; r < rpp; ++r) v += stg[(r * quads + (e >> 2)) * 4 + (e & 3)];
+                P.partial[((size_t)t * KS + sl) * kMaxExperts + e] = v;   // the partial-sum buffer is free until the down-projection
+            }
+        }
+        EPI_SYNC();
+        if (etid == 0) {
+            TRACE(1);
+            grid_arrive(P.sync, 0);
+            grid_wait(P.sync, 0, G, &sh.abort_flag);
+            TRACE(14);
+        }
+        EPI_SYNC();
+        // ---- router, step 2: CTA t adds the slices of token t in a fixed order; softmax and selection in one warp
+        if ((int)blockIdx.x < P.T && warp == 2 && !sh.abort_flag) {
+            const int t = blockIdx.x, E = P.E;
+            const bool v_lo = lane < E, v_hi = lane + 32 < E;
+            float l_lo = (P.br && v_lo) ? P.br[lane] : 0.f, l_hi = (P.br && v_hi) ? P.br[lane + 32] : 0.f;
+            for (int sl = 0; sl < KS; ++sl) {
+                const float* pl = P.partial + ((size_t)t * KS + sl) * kMaxExperts;
+                if (v_lo) l_lo += __ldcg(pl + lane);
+                if (v_hi) l_hi += __ldcg(pl + lane + 32);
+            }
+            softmax_select_store(l_lo, l_hi, t, P.sel, lane, P.scores, P.mask, P.k_t);
+        }
+        EPI_SYNC();
+        if (etid == 0) {
+            TRACE(15);
+            grid_arrive(P.sync, 3);
+            grid_wait(P.sync, 3, G, &sh.abort_flag);
+            TRACE(2);
+        }
+        EPI_SYNC();
+        // every CTA derives the set of selected experts from the T selection words
+        if (etid < P.T) {
+            unsigned long long m;
+            asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(m) : "l"(P.mask + etid) : "memory");
+            atomicOr(&sh.active_mask, m);
+        }
+        EPI_SYNC();
+        if (etid == 0) {
+            unsigned long long m = sh.active_mask;
+            if (P.E < 64) m &= (1ull << P.E) - 1ull;
+            SmallGeo& gr = sh.geo[1];
+            int n = 0;
+            for (int e = 0; e < P.E; ++e)
+                if ((m >> e) & 1ull) gr.active[n++] = e;
+            small_geometry(P, n, G, gr);
+            if (n != P.E) ptx::prefetch_tensormap(&tmW1.m[gr.up_rows / 16 - 1]);
+            __threadfence_block();
+            sh.geo_state = (n == P.E) ? 1 : 2;
+        }
+        EPI_SYNC();
+        const SmallGeo& ge = sh.geo[1];
+        const int n_act = ge.n_act;
+        const bool aborted_early = sh.abort_flag != 0;
+
+        // ---- epilogue
+        const int q = warp & 3;
         const bool tmem_warp = warp < 6;                 // warps 2..5 read TMEM; warps 6.. only share the arithmetic
         int acc = 0;
         uint32_t aph = 0;
         bool dead = aborted_early;     // a dead warp still takes part in every named barrier below
         bool up_done = false;
         SmallIter it;
-        it.init(P, n_act, sh.bn_down);
+        it.init(P, n_act, ge.bn_down);
         SmallTile t;
         const int row = q * 32 + lane;
         for (;;) {
-            const bool have = it.next(P, sh.active, n_act, t);
+            const bool have = it.next(P, ge.active, n_act, t);
             if (!up_done && (!have || t.phase == 1)) {
                 // this CTA's part of hg is complete: publish it (the arriving thread's fence, after the barrier,
                 // covers the other threads' stores), then signal the up/down grid barrier
                 asm volatile("fence.proxy.async;" ::: "memory");
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                EPI_SYNC();
                 if (etid == 0) {
                     grid_arrive(P.sync, 1);
                     TRACE(7);
@@ -901,7 +1072,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                             }
                         }
                     }
-                    asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                    EPI_SYNC();
 #ifdef DSMOE_TRACE
                     if (etid == 0) TRACE(29 + (c0 > 0));
 #endif
@@ -923,7 +1094,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                         hv[3] = __floats2bfloat162_rn(g * gelu_erf(b.z), g * gelu_erf(b.w));
                         *reinterpret_cast<uint4*>(P.hg + (long long)rr * ((long long)P.E * P.H) + ocol) = pk;
                     }
-                    asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                    EPI_SYNC();
                 }
             } else {
                 // fp32 partial sums of this CTA's share of the reduction: slot (cta, seg), row, 256 columns
@@ -953,18 +1124,18 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         // ---- last grid barrier, then the fix-up: out[t,c] = sum of the partial tiles covering column c in
         // ascending CTA order (the partition arithmetic mirrors SmallIter)
         __threadfence();
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+        EPI_SYNC();
         if (etid == 0) {
             TRACE(9);
             grid_arrive(P.sync, 2);
             if (!grid_wait(P.sync, 2, G, &sh.abort_flag)) sh.abort_flag = 1;
             TRACE(10);
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+        EPI_SYNC();
         if (!sh.abort_flag) {
             const int kbpe = P.H / BK;
             const int U = n_act * kbpe;
-            const int bnd = sh.bn_down;
+            const int bnd = ge.bn_down;
             const int nr = (P.d + bnd - 1) / bnd;
             const int total = nr * U;
             const int per = total > 0 ? (total + G - 1) / G : 1;
@@ -1252,6 +1423,9 @@ dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const 
     P.out_f32 = p.out_fp32 ? 1 : 0;
     P.sync = reinterpret_cast<int*>(ws + L.sync);
     P.dev_status = dev_status;
+    // With 16 tokens or more it is rare that an expert is selected by none of them, so the kernel starts the
+    // up-projection under that assumption while its router is still running; it starts over if the router disagrees.
+    P.spec = p.T >= kSpecMinT ? 1 : 0;
     DSMOE_CUDA_TRY(cudaMemsetAsync(P.sync, 0, 32, s));
     void* args[] = {&ms->mX, &ms->mW1, &ms->mHg, &ms->mW2, &P};
     const bool timed = g_timing.on && g_timing.n < kMaxTimed;
