@@ -30,7 +30,7 @@ constexpr int SMALL_THREADS = 448;    // small_layer_kernel: 2 + 4 warps as abov
 constexpr int kEpiThreads = SMALL_THREADS - 64;
 constexpr int TMEM_COLS = 512;
 constexpr int RING_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);   // operand ring: 4 x 48 KB, or more, smaller slots
-constexpr int SHARED_BYTES = 3072 + 256;                                     // barriers and small tables (struct Shared)
+constexpr int SHARED_BYTES = 4096 + 256;                                     // barriers and small tables (struct Shared)
 constexpr int STG_BYTES = BM * 36 * 4;                                 // epilogue staging tile: T rows x (32..256 + 4) floats
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)RING_BYTES + SHARED_BYTES + STG_BYTES;
 constexpr size_t SMEM_GEMM_BYTES = 1024 + (size_t)RING_BYTES + SHARED_BYTES;   // umma_gemm_kernel needs no staging tile
@@ -41,6 +41,14 @@ constexpr int kUpUnit = 16;          // small-T up-projection: weight rows per w
 constexpr int kUpTileUnits = 16;     // ... and units per tile (256 rows)
 constexpr int kRouterBatch = 12;     // rows of Wr a router thread loads at once
 constexpr int kFixBatch = 24;        // partial tiles a fix-up thread loads at once
+// small-T kernel: bytes of loads a CTA keeps in flight (<= RING_BYTES).  Four 36 KB slots per SM already cover the
+// bandwidth-delay product; a deeper ring only lengthens the queues that the router's loads, the grid barriers and
+// instruction fetches wait in.
+#ifndef DSMOE_SMALL_INFLIGHT
+#define DSMOE_SMALL_INFLIGHT (144 * 1024)
+#endif
+constexpr int kSmallInflightBytes = DSMOE_SMALL_INFLIGHT;
+static_assert(kSmallInflightBytes <= RING_BYTES, "in-flight bytes are ring bytes");
 constexpr int kSpecMinT = 16;        // tokens from which the small-T kernel streams ahead of its router
 
 struct GemmParams {
@@ -97,6 +105,7 @@ struct Shared {
     volatile int spec_issued, spec_stop;   // producer -> MMA issuer: ring slots filled under geo[0]; no more will be
     volatile int mma_drained;              // MMA issuer -> producer: those slots are consumed, the ring is idle
     float gate_s[BM], gate2_s[BM];
+    uint64_t mask_s[BM];                   // small_layer_kernel: every token's selection word
 #ifdef DSMOE_TRACE
     unsigned long long trace[32];
 #endif
@@ -415,7 +424,7 @@ struct SmallParams {
     float* partial;          // [grid][2][T][256]; doubles as the router's slice buffer
     void* out;
     int out_f32;
-    int* sync;               // 8 ints, zero at launch: four barrier counters [0..3] and an abort flag [4]
+    int* sync;               // 8 ints, zero at launch: barrier counters [0..2] and an abort flag [4]
     int spec;                // start streaming under "every expert selected" before the router has finished
     int32_t* dev_status;
 };
@@ -523,17 +532,19 @@ struct SmallIter {
     }
 };
 
-// One ring slot's loads.  what: bit 0 = the token operand (x or hg), bit 1 = the weight rows.
+// One ring slot's loads.  what: bit 0 = the token operand (x or hg), bit 1 = the weight rows.  The weights are read
+// once per call, so their copies carry the evict-first L2 policy `wpol`: the stream then leaves the router's operands,
+// hg, the partial sums and the kernel's own instructions in L2.
 __device__ __forceinline__ void small_issue(const SmallParams& P, const CUtensorMap* tmX, const BMaps16* tmW1,
                                             const CUtensorMap* tmHg, const BMaps* tmW2, const int* active,
                                             const SmallTile& t, int i, uint32_t slotA, uint32_t slotB, uint32_t bar,
-                                            int what) {
+                                            int what, uint64_t wpol) {
     if (t.phase == 0) {
         if (what & 1) ptx::tma_load_2d(slotA, tmX, bar, i * BK, 0);
         if (what & 2) {
-            ptx::tma_load_3d(slotB, &tmW1->m[t.bn1 / 16 - 1], bar, i * BK, t.n0, t.e);
+            ptx::tma_load_3d_hint(slotB, &tmW1->m[t.bn1 / 16 - 1], bar, i * BK, t.n0, t.e, wpol);
             if (t.bn > t.bn1)
-                ptx::tma_load_3d(slotB + t.bn1 * (BK * 2), &tmW1->m[(t.bn - t.bn1) / 16 - 1], bar, i * BK, 0, t.e2);
+                ptx::tma_load_3d_hint(slotB + t.bn1 * (BK * 2), &tmW1->m[(t.bn - t.bn1) / 16 - 1], bar, i * BK, 0, t.e2, wpol);
         }
     } else {
         const int kbpe = P.H / BK;
@@ -542,7 +553,7 @@ __device__ __forceinline__ void small_issue(const SmallParams& P, const CUtensor
         if (what & 1) ptx::tma_load_2d(slotA, tmHg, bar, e * P.H + kb * BK, 0);
         if (what & 2) {
             // column ranges are 64, 128 or 256 wide: one copy; only a ragged last range needs the decomposition
-            if ((t.bn & (t.bn - 1)) == 0) ptx::tma_load_3d(slotB, &tmW2->m[__ffs(t.bn) - 5], bar, kb * BK, t.n0, e);
+            if ((t.bn & (t.bn - 1)) == 0) ptx::tma_load_3d_hint(slotB, &tmW2->m[__ffs(t.bn) - 5], bar, kb * BK, t.n0, e, wpol);
             else load_weight_rows(tmW2, slotB, bar, kb * BK, t.n0, t.bn, e);
         }
     }
@@ -558,7 +569,69 @@ __device__ __forceinline__ void small_geometry(const SmallParams& P, int n, int 
     g.bn_down = g.up_rows <= 64 ? 64 : g.up_rows <= 128 ? 128 : BN;
     g.a_bytes = P.t_pad * BK * 2;
     g.slot_bytes = g.a_bytes + g.bn_down * BK * 2;
-    g.n_stages = min(MAX_STAGES, RING_BYTES / g.slot_bytes);
+    g.n_stages = max(2, min(MAX_STAGES, kSmallInflightBytes / g.slot_bytes));
+}
+
+// Second half of the router, run by the 12 epilogue warps of EVERY CTA: warp w owns tokens w, w + 12, ...; a lane
+// holds experts lane and lane + 32.  Logits = bias plus the KS slice sums in ascending slice order, then softmax.
+// The arithmetic is the same in every CTA, so are the results, and no grid barrier is needed to agree on them.
+//   mode 0: selection -- sh.mask_s[token], sh.active_mask; CTA t also writes token t's scores, mask and count out
+//   mode 1: router gates of experts e and e2 for every token (0 where not selected) -> sh.gate_s, sh.gate2_s
+// KS * (tokens per warp) <= 16 for every T this kernel takes, so a warp fetches all its slice sums in one batch
+// and waits for memory once.  One copy of this code serves both modes (not inlined): the second call finds its
+// instructions cached, which matters while the weight stream keeps the memory system busy.
+__device__ __noinline__ void small_router_pass(const SmallParams& P, Shared& sh, int KS, int w, int lane, int mode, int e,
+                                               int e2) {
+    constexpr int NW = kEpiThreads / 32;
+    const bool v_lo = lane < P.E, v_hi = lane + 32 < P.E;
+    const float b_lo = (P.br && v_lo) ? P.br[lane] : 0.f, b_hi = (P.br && v_hi) ? P.br[lane + 32] : 0.f;
+    const int ntok = w < P.T ? (P.T - w + NW - 1) / NW : 0;
+    const int lg = 31 - __clz(KS);
+    float vlo[16], vhi[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int tt = w + (j >> lg) * NW, sl = j & (KS - 1);      // KS is a power of two
+        const bool ok = j < ntok * KS;
+        const float* pl = P.partial + ((size_t)tt * KS + sl) * kMaxExperts;
+        vlo[j] = (ok && v_lo) ? __ldcg(pl + lane) : 0.f;
+        vhi[j] = (ok && v_hi) ? __ldcg(pl + lane + 32) : 0.f;
+    }
+#pragma unroll 1
+    for (int i = 0; i < ntok; ++i) {
+        const int tt = w + i * NW;
+        float l_lo = b_lo, l_hi = b_hi;
+#pragma unroll 1
+        for (int sl = 0; sl < KS; ++sl) {
+            l_lo += vlo[0];
+            l_hi += vhi[0];
+#pragma unroll
+            for (int j = 0; j < 15; ++j) {      // the next slice sum moves to the front
+                vlo[j] = vlo[j + 1];
+                vhi[j] = vhi[j + 1];
+            }
+        }
+        float s_lo, s_hi;
+        softmax_warp(l_lo, l_hi, P.E, lane, s_lo, s_hi);
+        if (mode == 0) {
+            const uint64_t m = select_warp(s_lo, s_hi, P.sel, lane);
+            if (lane == 0) {
+                sh.mask_s[tt] = m;
+                atomicOr(&sh.active_mask, (unsigned long long)m);
+            }
+            if (tt == (int)blockIdx.x) {
+                if (v_lo) P.scores[(size_t)tt * P.E + lane] = s_lo;
+                if (v_hi) P.scores[(size_t)tt * P.E + lane + 32] = s_hi;
+                if (lane == 0) {
+                    P.mask[tt] = m;
+                    if (P.k_t) P.k_t[tt] = __popcll(m);
+                }
+            }
+        } else {
+            const uint64_t mk = sh.mask_s[tt];
+            if (lane == (e & 31)) sh.gate_s[tt] = ((mk >> e) & 1ull) ? (e < 32 ? s_lo : s_hi) : 0.f;
+            if (lane == (e2 & 31)) sh.gate2_s[tt] = ((mk >> e2) & 1ull) ? (e2 < 32 ? s_lo : s_hi) : 0.f;
+        }
+    }
 }
 
 // Bounded wait for the router's verdict on the speculative geometry; 0 = gave up.
@@ -652,6 +725,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             int s = 0;
             uint32_t phb = 0;
             bool alive = true, spec = P.spec != 0;
+            const uint64_t wpol = ptx::policy_evict_first();
             const SmallGeo* g = &sh.geo[0];
             if (!spec) {
                 alive = wait_geo(sh) != 0;
@@ -697,7 +771,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                         }
                         const uint32_t bar = ptx::smem_u32(&sh.full[s]);
                         ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
-                        small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, t, i, smA + s * slot_bytes, smB + s * slot_bytes, bar, 3);
+                        small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, t, i, smA + s * slot_bytes, smB + s * slot_bytes, bar, 3, wpol);
                         phb ^= 1u << s;
                         ++issued;
                         if (++s == n_stages) s = 0;
@@ -733,7 +807,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 }
                 const uint32_t bar = ptx::smem_u32(&sh.full[s]);
                 ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
-                small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 2);
+                small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 2, wpol);
                 pend_t[npend] = t;
                 pend_i[npend] = i_cur;
                 pend_s[npend] = s;
@@ -751,7 +825,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             asm volatile("fence.proxy.async;" ::: "memory");   // hg was written through the generic proxy, TMA reads it
             for (int j = 0; alive && j < npend; ++j)
                 small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, pend_t[j], pend_i[j], smA + pend_s[j] * slot_bytes,
-                            smB + pend_s[j] * slot_bytes, ptx::smem_u32(&sh.full[pend_s[j]]), 1);
+                            smB + pend_s[j] * slot_bytes, ptx::smem_u32(&sh.full[pend_s[j]]), 1, wpol);
             while (alive && have) {
                 for (; i_cur < t.nk; ++i_cur) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ((phb >> s) & 1u) ^ 1u, &sh.abort_flag)) {
@@ -760,7 +834,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     }
                     const uint32_t bar = ptx::smem_u32(&sh.full[s]);
                     ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
-                    small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 3);
+                    small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 3, wpol);
                     phb ^= 1u << s;
                     if (++s == n_stages) s = 0;
                 }
@@ -905,7 +979,8 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         // (E floats) is covered by E/4 neighbouring threads with one 16-byte load each, so a warp reads whole
         // rows, coalesced, and a thread keeps only its four experts' sums over every rpp-th row; all its loads are
         // independent.  The threads' sums meet in shared memory.
-        const int KS = max(1, min(16, G / P.T));
+        int KS = 1;                                   // 1, 2, 4, 8 or 16 slices
+        while (KS < 16 && KS * 2 * P.T <= G) KS *= 2;
         if ((int)blockIdx.x < P.T * KS) {
             const int t = blockIdx.x / KS, sl = blockIdx.x % KS, E = P.E;
             const int klen = (P.d + KS - 1) / KS, kbeg = sl * klen, kend = min(P.d, kbeg + klen);
@@ -967,32 +1042,8 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             TRACE(14);
         }
         EPI_SYNC();
-        // ---- router, step 2: CTA t adds the slices of token t in a fixed order; softmax and selection in one warp
-        if ((int)blockIdx.x < P.T && warp == 2 && !sh.abort_flag) {
-            const int t = blockIdx.x, E = P.E;
-            const bool v_lo = lane < E, v_hi = lane + 32 < E;
-            float l_lo = (P.br && v_lo) ? P.br[lane] : 0.f, l_hi = (P.br && v_hi) ? P.br[lane + 32] : 0.f;
-            for (int sl = 0; sl < KS; ++sl) {
-                const float* pl = P.partial + ((size_t)t * KS + sl) * kMaxExperts;
-                if (v_lo) l_lo += __ldcg(pl + lane);
-                if (v_hi) l_hi += __ldcg(pl + lane + 32);
-            }
-            softmax_select_store(l_lo, l_hi, t, P.sel, lane, P.scores, P.mask, P.k_t);
-        }
-        EPI_SYNC();
-        if (etid == 0) {
-            TRACE(15);
-            grid_arrive(P.sync, 3);
-            grid_wait(P.sync, 3, G, &sh.abort_flag);
-            TRACE(2);
-        }
-        EPI_SYNC();
-        // every CTA derives the set of selected experts from the T selection words
-        if (etid < P.T) {
-            unsigned long long m;
-            asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(m) : "l"(P.mask + etid) : "memory");
-            atomicOr(&sh.active_mask, m);
-        }
+        // ---- router, step 2: softmax and selection of every token, in every CTA (see small_router_pass)
+        if (!sh.abort_flag) small_router_pass(P, sh, KS, warp - 2, lane, 0, 0, 0);
         EPI_SYNC();
         if (etid == 0) {
             unsigned long long m = sh.active_mask;
@@ -1005,6 +1056,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             if (n != P.E) ptx::prefetch_tensormap(&tmW1.m[gr.up_rows / 16 - 1]);
             __threadfence_block();
             sh.geo_state = (n == P.E) ? 1 : 2;
+            TRACE(2);
         }
         EPI_SYNC();
         const SmallGeo& ge = sh.geo[1];
@@ -1036,13 +1088,9 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 up_done = true;
             }
             if (!have) break;
-            if (t.phase == 0 && etid < P.T) {
-                // router gate of every token for this tile's expert(s), 0 where the token did not select it;
-                // fetched while the mainloop is still running (the previous tile ended on a barrier)
-                const uint64_t mk = P.mask[etid];
-                sh.gate_s[etid] = ((mk >> t.e) & 1ull) ? P.scores[(long long)etid * P.E + t.e] : 0.f;
-                sh.gate2_s[etid] = ((mk >> t.e2) & 1ull) ? P.scores[(long long)etid * P.E + t.e2] : 0.f;
-            }
+            // router gate of every token for this tile's expert(s), recomputed from the slice sums (other CTAs' copies
+            // of the scores are not visible yet) while the mainloop is still running
+            if (t.phase == 0 && !dead) small_router_pass(P, sh, KS, warp - 2, lane, 1, t.e, t.e2);
             if (tmem_warp && !dead && !ptx::mbar_wait(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag)) dead = true;
             dead = __any_sync(0xffffffffu, dead);     // the TMEM reads below are warp-collective
 #ifdef DSMOE_TRACE
@@ -1182,7 +1230,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             }
             if (P.counts_out && blockIdx.x == 0 && etid < P.E) {
                 int n = 0;
-                for (int tt = 0; tt < P.T; ++tt) n += (int)((P.mask[tt] >> etid) & 1ull);
+                for (int tt = 0; tt < P.T; ++tt) n += (int)((sh.mask_s[tt] >> etid) & 1ull);
                 P.counts_out[etid] = n;
             }
         }

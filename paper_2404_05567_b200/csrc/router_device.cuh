@@ -74,17 +74,25 @@ __device__ __forceinline__ uint64_t select_warp(float s_lo, float s_hi, const Se
     return m;
 }
 
-// Softmax over all E experts of one token (row maximum subtracted), then selection; the warp writes
-// scores[t,:], mask[t], k_t[t] (each optional).
-__device__ __forceinline__ void softmax_select_store(float l_lo, float l_hi, int t, const SelParams& q, int lane,
-                                                     float* __restrict__ scores, uint64_t* __restrict__ mask,
-                                                     int32_t* __restrict__ k_t) {
-    const bool v_lo = lane < q.E, v_hi = lane + 32 < q.E;
+// Softmax over all E experts of one token (row maximum subtracted), logits and scores of experts lane and
+// lane + 32 held by a full warp.
+__device__ __forceinline__ void softmax_warp(float l_lo, float l_hi, int E, int lane, float& s_lo, float& s_hi) {
+    const bool v_lo = lane < E, v_hi = lane + 32 < E;
     const float mx = warp_max(fmaxf(v_lo ? l_lo : -INFINITY, v_hi ? l_hi : -INFINITY));
     const float p_lo = v_lo ? expf(l_lo - mx) : 0.f;
     const float p_hi = v_hi ? expf(l_hi - mx) : 0.f;
     const float den = warp_sum(p_lo + p_hi);
-    const float s_lo = __fdiv_rn(p_lo, den), s_hi = __fdiv_rn(p_hi, den);
+    s_lo = __fdiv_rn(p_lo, den);
+    s_hi = __fdiv_rn(p_hi, den);
+}
+
+// Softmax, then selection; the warp writes scores[t,:], mask[t], k_t[t] (each optional).
+__device__ __forceinline__ void softmax_select_store(float l_lo, float l_hi, int t, const SelParams& q, int lane,
+                                                     float* __restrict__ scores, uint64_t* __restrict__ mask,
+                                                     int32_t* __restrict__ k_t) {
+    const bool v_lo = lane < q.E, v_hi = lane + 32 < q.E;
+    float s_lo, s_hi;
+    softmax_warp(l_lo, l_hi, q.E, lane, s_lo, s_hi);
     if (scores) {
         if (v_lo) scores[(size_t)t * q.E + lane] = s_lo;
         if (v_hi) scores[(size_t)t * q.E + lane + 32] = s_hi;
