@@ -49,7 +49,7 @@ constexpr int kFixBatch = 24;        // partial tiles a fix-up thread loads at o
 #endif
 constexpr int kSmallInflightBytes = DSMOE_SMALL_INFLIGHT;
 static_assert(kSmallInflightBytes <= RING_BYTES, "in-flight bytes are ring bytes");
-constexpr int kSpecMinT = 16;        // tokens from which the small-T kernel streams ahead of its router
+constexpr int kSpecMinT = 8;         // tokens from which the small-T kernel streams ahead of its router
 
 struct GemmParams {
     int mode, epi;
@@ -99,8 +99,11 @@ struct Shared {
     int seg0[kMaxExperts], seg1[kMaxExperts];
     unsigned long long active_mask;
     // small_layer_kernel: geo[0] assumes every expert selected (streaming starts under it while the router still
-    // runs), geo[1] is what the router found.  geo_state: 0 router pending, 1 geo[1] equals geo[0], 2 it differs.
+    // runs), geo[1] is what the router found.  geo_state: 0 router pending; 1 the up-projection started under geo[0] stands (geo[1]
+    // equals it, or misses only a few experts and has the same ring: their tiles are computed for nothing and gated
+    // to zero); 2 it is started over under geo[1].
     SmallGeo geo[2];
+    volatile int up_geo;                   // which of the two the up-projection follows (the down-projection: always geo[1])
     volatile int geo_state;
     volatile int spec_issued, spec_stop;   // producer -> MMA issuer: ring slots filled under geo[0]; no more will be
     volatile int mma_drained;              // MMA issuer -> producer: those slots are consumed, the ring is idle
@@ -464,24 +467,33 @@ struct SmallIter {
 
     int bn_down;
 
-    __device__ __forceinline__ void init(const SmallParams& P, int n_act, int bn_down_) {
+    // The two projections may be cut over different expert lists: the up-projection over n_up experts (all of
+    // them, when it was started before the router had finished), the down-projection over the n_down selected ones.
+    __device__ __forceinline__ void init(const SmallParams& P, int n_up, int n_down, int bn_down_) {
+        const int G = gridDim.x;
+        const int total = n_up * (P.H / kUpUnit);
+        const int per = (total + G - 1) / G;
+        u0 = min(total, (int)blockIdx.x * per);
+        u1 = min(total, u0 + per);
+        phase = 0;
+        set_down(P, n_down, bn_down_);
+    }
+    __device__ __forceinline__ void set_down(const SmallParams& P, int n_down, int bn_down_) {
         const int G = gridDim.x;
         bn_down = bn_down_;
-        {
-            const int total = n_act * (P.H / kUpUnit);
-            const int per = (total + G - 1) / G;
-            u0 = min(total, (int)blockIdx.x * per);
-            u1 = min(total, u0 + per);
-        }
-        {
-            const int U = n_act * (P.H / BK);
-            const int total = ((P.d + bn_down - 1) / bn_down) * U;
-            const int per = (total + G - 1) / G;
-            down_u0 = min(total, (int)blockIdx.x * per);
-            down_u1 = min(total, down_u0 + per);
-            r_first = U > 0 ? down_u0 / U : 0;
-        }
-        phase = 0;
+        const int U = n_down * (P.H / BK);
+        const int total = ((P.d + bn_down - 1) / bn_down) * U;
+        const int per = (total + G - 1) / G;
+        down_u0 = min(total, (int)blockIdx.x * per);
+        down_u1 = min(total, down_u0 + per);
+        r_first = U > 0 ? down_u0 / U : 0;
+    }
+    // (re)start the down-projection under another expert list
+    __device__ __forceinline__ void restart_down(const SmallParams& P, int n_down, int bn_down_) {
+        set_down(P, n_down, bn_down_);
+        phase = 1;
+        u0 = down_u0;
+        u1 = down_u1;
     }
 
     __device__ __forceinline__ bool next(const SmallParams& P, const int* active, int n_act, SmallTile& t) {
@@ -741,7 +753,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 slot_bytes = (uint32_t)g->slot_bytes;
                 a_bytes = (uint32_t)g->a_bytes;
                 smB = base + a_bytes;
-                it.init(P, g->n_act, g->bn_down);
+                it.init(P, g->n_act, g->n_act, g->bn_down);
                 have = it.next(P, g->active, g->n_act, t);
                 int issued = 0;
                 bool replaced = false;
@@ -784,6 +796,11 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     const int st = wait_geo(sh);
                     if (st == 0) alive = false;
                     else if (st == 2) replaced = true;
+                    else {
+                        g = &sh.geo[1];     // same ring; the down-projection runs over the selected experts
+                        it.restart_down(P, g->n_act, g->bn_down);
+                        have = it.next(P, g->active, g->n_act, t);
+                    }
                 }
                 if (!(alive && replaced)) break;
                 sh.spec_issued = issued;
@@ -865,9 +882,38 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 int consumed = 0;
                 bool redo = false;
                 SmallIter it;
-                it.init(P, g->n_act, g->bn_down);
+                const SmallGeo* gD = g;      // the down-projection's expert list: geo[1] once the router is done
+                it.init(P, g->n_act, g->n_act, g->bn_down);
                 SmallTile t;
-                while (alive && !redo && it.next(P, g->active, g->n_act, t)) {
+                for (;;) {
+                    if (!(alive && !redo && it.next(P, g->active, gD->n_act, t))) {
+                        if (alive && !redo && spec) {
+                            // nothing (left) to do under geo[0]; there may be under geo[1], and if the router
+                            // disagrees the producer waits for this thread
+                            const int st = wait_geo(sh);
+                            spec = false;
+                            if (st == 0) alive = false;
+                            else if (st == 2) redo = true;
+                            else {
+                                gD = &sh.geo[1];
+                                it.restart_down(P, gD->n_act, gD->bn_down);
+                                continue;
+                            }
+                        }
+                        break;
+                    }
+                    if (spec && t.phase == 1) {
+                        // no down-projection tile before the router has said over which experts it runs
+                        const int st = wait_geo(sh);
+                        if (st == 0) alive = false;
+                        else if (st == 2) redo = true;
+                        else {
+                            spec = false;
+                            gD = &sh.geo[1];
+                            it.restart_down(P, gD->n_act, gD->bn_down);
+                        }
+                        continue;
+                    }
                     if (!ptx::mbar_wait(ptx::smem_u32(&sh.tempty[acc]), aph ^ 1u, &sh.abort_flag)) {
                         alive = false;
                         break;
@@ -929,19 +975,16 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                             break;
                         }
                         spec = false;
+                        // the rest of the up-projection stays under geo[0]'s partition (and its identity expert list,
+                        // which this thread's iterator already holds); the down-projection follows geo[1]
+                        gD = &sh.geo[1];
+                        it.set_down(P, gD->n_act, gD->bn_down);
                     }
                     ptx::umma_commit(ptx::smem_u32(&sh.tfull[acc]));
                     if (++acc == 2) {
                         acc = 0;
                         aph ^= 1u;
                     }
-                }
-                if (alive && !redo && spec) {
-                    // a CTA without work under geo[0] may have some under geo[1]; the producer waits for this thread either way
-                    const int st = wait_geo(sh);
-                    if (st == 0) alive = false;
-                    else if (st == 2) redo = true;
-                    spec = false;
                 }
                 if (!(alive && redo)) break;
                 // take the remaining speculative loads off the ring, let the products issued so far retire, then
@@ -1053,13 +1096,20 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             for (int e = 0; e < P.E; ++e)
                 if ((m >> e) & 1ull) gr.active[n++] = e;
             small_geometry(P, n, G, gr);
-            if (n != P.E) ptx::prefetch_tensormap(&tmW1.m[gr.up_rows / 16 - 1]);
+            // an up-projection already under way stands if at most an eighth of the experts went unselected (and
+            // the ring keeps its geometry): starting over would cost more than their tiles do
+            const SmallGeo& g0 = sh.geo[0];
+            const bool keep = P.spec && (n == P.E || (n >= P.E - max(1, P.E / 8) && gr.a_bytes == g0.a_bytes &&
+                                                      gr.slot_bytes == g0.slot_bytes && gr.n_stages == g0.n_stages));
+            if (!keep) ptx::prefetch_tensormap(&tmW1.m[gr.up_rows / 16 - 1]);
+            sh.up_geo = keep ? 0 : 1;
             __threadfence_block();
-            sh.geo_state = (n == P.E) ? 1 : 2;
+            sh.geo_state = keep ? 1 : 2;
             TRACE(2);
         }
         EPI_SYNC();
         const SmallGeo& ge = sh.geo[1];
+        const SmallGeo& gu = sh.geo[sh.up_geo];
         const int n_act = ge.n_act;
         const bool aborted_early = sh.abort_flag != 0;
 
@@ -1071,11 +1121,11 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         bool dead = aborted_early;     // a dead warp still takes part in every named barrier below
         bool up_done = false;
         SmallIter it;
-        it.init(P, n_act, ge.bn_down);
+        it.init(P, gu.n_act, n_act, ge.bn_down);
         SmallTile t;
         const int row = q * 32 + lane;
         for (;;) {
-            const bool have = it.next(P, ge.active, n_act, t);
+            const bool have = it.next(P, gu.active, n_act, t);
             if (!up_done && (!have || t.phase == 1)) {
                 // this CTA's part of hg is complete: publish it (the arriving thread's fence, after the barrier,
                 // covers the other threads' stores), then signal the up/down grid barrier

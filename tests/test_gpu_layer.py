@@ -132,7 +132,15 @@ def test_c5_skewed_router_threshold_sweep(eps):
     dict(T=20, E=8, mode=gi.MODE_ALL, d=128, H=6144),
     dict(T=20, E=16, mode=gi.MODE_TOPK, K=1, d=128, H=3072),
     dict(T=32, E=16, mode=gi.MODE_TOPK, K=1, d=2048, H=128),         # ... and long reductions: it starts over mid-tile
-], ids=["topk1", "few", "none", "skew", "all", "wide_all", "wide_topk1", "deep_topk1"])
+    # nearly every expert selected: the up-projection started under "every expert" stands, the unselected experts'
+    # tiles are gated to zero and the down-projection runs over the selected ones only (15 and 14 of 16); with 12 of
+    # 16 it starts over
+    dict(T=12, E=16, mode=gi.MODE_TOPK, K=3),
+    dict(T=9, E=16, mode=gi.MODE_TOPK, K=3),
+    dict(T=9, E=16, mode=gi.MODE_TOPK, K=2),
+    dict(T=12, E=16, mode=gi.MODE_TOPK, K=3, d=128, H=3072),
+], ids=["topk1", "few", "none", "skew", "all", "wide_all", "wide_topk1", "deep_topk1", "near15", "near14", "far12",
+        "wide_near15"])
 def test_decode_path_when_some_experts_are_unselected(case):
     kw = dict(d=512, H=256)
     kw.update(case)
