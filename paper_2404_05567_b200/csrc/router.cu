@@ -73,64 +73,157 @@ __global__ void __launch_bounds__(256) router_small_kernel(const XT* __restrict_
     }
 }
 
-// Large T (prefill): a block owns 32 tokens and walks d in chunks staged through shared memory, so
-// each router weight is read from L2 once per 32 tokens.  Warp w keeps tokens 4w..4w+3.
-template <typename XT, int EP>
-__global__ void __launch_bounds__(256) router_tile_kernel(const XT* __restrict__ x, const float* __restrict__ Wr,
-                                                          const float* __restrict__ br, float* __restrict__ scores,
-                                                          uint64_t* __restrict__ mask, int32_t* __restrict__ k_t,
-                                                          int T, int d, SelParams q) {
-    constexpr int TB = 32, KC = 64, NE = EP / 32;
-    __shared__ __align__(16) float Xs[TB][KC + 4];
-    __shared__ float Ws[KC][EP];
+// Large T (prefill): an fp32 FMA GEMM [T,d] x [d,E] with the softmax and the selection as its epilogue.  A block
+// owns 64 tokens and walks d in chunks of 128 staged through shared memory (two buffers; the next chunk's global
+// loads are in flight while the current one is multiplied).  A thread keeps 2 tokens x EPL experts (EPL = 4 for
+// E <= 32, 8 for E <= 64): 8 neighbouring lanes cover all experts of a token with 16-byte shared-memory reads that
+// the lanes of a warp share, so the loop is bound by the FMA pipe, not by shared-memory traffic.
+//   warp w (of a group of 8): tokens 8w..8w+7; lane: tokens 8w + lane/8 + {0, 4}; experts 4 (lane % 8) + {0..3}
+//   (and 32 + the same when EPL = 8)
+template <typename XT>
+__device__ __forceinline__ void load8_as_f32(const XT* p, bool vec, int nvalid, float (&out)[8]);
+template <>
+__device__ __forceinline__ void load8_as_f32<__nv_bfloat16>(const __nv_bfloat16* p, bool vec, int nvalid, float (&out)[8]) {
+    if (vec && nvalid == 8) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __bfloat1622float2(h[i]);
+            out[2 * i] = f.x;
+            out[2 * i + 1] = f.y;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[i] = i < nvalid ? __bfloat162float(p[i]) : 0.f;
+    }
+}
+template <>
+__device__ __forceinline__ void load8_as_f32<float>(const float* p, bool vec, int nvalid, float (&out)[8]) {
+    if (vec && nvalid == 8) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(p)), b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+        out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+        out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[i] = i < nvalid ? p[i] : 0.f;
+    }
+}
+
+constexpr int kRtTB = 64, kRtKC = 128, kRtXS = kRtKC + 4, kRtSplit = 4, kRtThreads = 256 * kRtSplit;
+template <int EPL>
+constexpr size_t router_tile_smem() {
+    return (size_t)2 * kRtTB * kRtXS * sizeof(float) + (size_t)2 * kRtKC * (8 * EPL) * sizeof(float);
+}
+
+// 1024 threads: four groups of 8 warps; group g multiplies the g-th quarter of every 128-wide chunk (the same 2 x EPL
+// tile per thread in each group), so that every scheduler has 8 warps to hide the FMA and shared-memory latencies
+// behind.  The groups' partial sums meet in shared memory at the end and are added in group order.
+template <typename XT, int EPL>
+__global__ void __launch_bounds__(kRtThreads, 1) router_tile_kernel(const XT* __restrict__ x, const float* __restrict__ Wr,
+                                                                    const float* __restrict__ br, float* __restrict__ scores,
+                                                                    uint64_t* __restrict__ mask, int32_t* __restrict__ k_t,
+                                                                    int T, int d, SelParams q) {
+    constexpr int TB = kRtTB, KC = kRtKC, EP = 8 * EPL, XS = kRtXS, NT = kRtThreads;
+    constexpr int NW = KC * EP / NT, NX = TB * KC / 8 / NT, KQ = KC / kRtSplit;
+    static_assert(NX == 1 && NW >= 1, "staging: one 8-element group of x per thread");
+    extern __shared__ __align__(16) float rt_smem[];
+    float (*Xs)[TB][XS] = reinterpret_cast<float (*)[TB][XS]>(rt_smem);                      // [2][TB][XS]
+    float (*Ws)[KC][EP] = reinterpret_cast<float (*)[KC][EP]>(rt_smem + 2 * TB * XS);          // [2][KC][EP]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int t0 = blockIdx.x * TB, E = q.E;
-    float acc[4][NE];
+    const bool vec = (d & 7) == 0;                    // rows of x start 16-byte aligned
+    // staging: thread -> 8 consecutive k of one token (16 threads per token row), and NW router weights
+    const int xr = tid >> 4, xc = (tid & 15) * 8;
+    const XT* xrow = x + (size_t)min(t0 + xr, T - 1) * d;
+    const bool xrow_ok = t0 + xr < T;
+    float xreg[8], wreg[NW];
+    auto fetch = [&](int k0) {
+        const int nv = xrow_ok ? max(0, min(8, d - (k0 + xc))) : 0;
+        if (nv > 0) load8_as_f32<XT>(xrow + k0 + xc, vec, nv, xreg);
+        else {
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < 8; ++i) xreg[i] = 0.f;
+        }
 #pragma unroll
-        for (int u = 0; u < NE; ++u) acc[i][u] = 0.f;
+        for (int i = 0; i < NW; ++i) {
+            const int idx = tid + i * NT, kk = idx / EP, e = idx % EP;
+            wreg[i] = (e < E && k0 + kk < d) ? __ldg(Wr + (size_t)(k0 + kk) * E + e) : 0.f;
+        }
+    };
+    auto stash = [&](int b) {
+        *reinterpret_cast<float4*>(&Xs[b][xr][xc]) = make_float4(xreg[0], xreg[1], xreg[2], xreg[3]);
+        *reinterpret_cast<float4*>(&Xs[b][xr][xc + 4]) = make_float4(xreg[4], xreg[5], xreg[6], xreg[7]);
+#pragma unroll
+        for (int i = 0; i < NW; ++i) {
+            const int idx = tid + i * NT;
+            Ws[b][idx / EP][idx % EP] = wreg[i];
+        }
+    };
+    const int grp = warp >> 3, w8 = warp & 7;
+    const int tk = w8 * 8 + (lane >> 3), eo = (lane & 7) * 4;   // this thread's first token (in the block), first expert
+    float acc[2][EPL];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int u = 0; u < EPL; ++u) acc[i][u] = 0.f;
 
+    fetch(0);
+    stash(0);
+    __syncthreads();
+    int b = 0;
     for (int k0 = 0; k0 < d; k0 += KC) {
-        for (int idx = tid; idx < TB * KC; idx += 256) {
-            const int r = idx / KC, c = idx % KC;
-            const int t = t0 + r, k = k0 + c;
-            Xs[r][c] = (t < T && k < d) ? to_f32(x[(size_t)t * d + k]) : 0.f;
-        }
-        for (int idx = tid; idx < KC * EP; idx += 256) {
-            const int kk = idx / EP, e = idx % EP;
-            const int k = k0 + kk;
-            Ws[kk][e] = (e < E && k < d) ? __ldg(Wr + (size_t)k * E + e) : 0.f;
-        }
-        __syncthreads();
-#pragma unroll 4
-        for (int kk = 0; kk < KC; kk += 4) {
-            float4 xv[4];
+        const bool more = k0 + KC < d;
+        if (more) fetch(k0 + KC);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) xv[i] = *reinterpret_cast<const float4*>(&Xs[4 * warp + i][kk]);
+        for (int kq = 0; kq < KQ; kq += 4) {
+            const int kk = grp * KQ + kq;
+            const float4 xa = *reinterpret_cast<const float4*>(&Xs[b][tk][kk]);
+            const float4 xb = *reinterpret_cast<const float4*>(&Xs[b][tk + 4][kk]);
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                float w[NE];
+                const float xs0 = u == 0 ? xa.x : u == 1 ? xa.y : u == 2 ? xa.z : xa.w;
+                const float xs1 = u == 0 ? xb.x : u == 1 ? xb.y : u == 2 ? xb.z : xb.w;
 #pragma unroll
-                for (int v = 0; v < NE; ++v) w[v] = Ws[kk + u][lane + 32 * v];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float xs = u == 0 ? xv[i].x : u == 1 ? xv[i].y : u == 2 ? xv[i].z : xv[i].w;
-#pragma unroll
-                    for (int v = 0; v < NE; ++v) acc[i][v] = fmaf(xs, w[v], acc[i][v]);
+                for (int h = 0; h < EPL / 4; ++h) {
+                    const float4 w = *reinterpret_cast<const float4*>(&Ws[b][kk + u][eo + 32 * h]);
+                    acc[0][4 * h + 0] = fmaf(xs0, w.x, acc[0][4 * h + 0]);
+                    acc[0][4 * h + 1] = fmaf(xs0, w.y, acc[0][4 * h + 1]);
+                    acc[0][4 * h + 2] = fmaf(xs0, w.z, acc[0][4 * h + 2]);
+                    acc[0][4 * h + 3] = fmaf(xs0, w.w, acc[0][4 * h + 3]);
+                    acc[1][4 * h + 0] = fmaf(xs1, w.x, acc[1][4 * h + 0]);
+                    acc[1][4 * h + 1] = fmaf(xs1, w.y, acc[1][4 * h + 1]);
+                    acc[1][4 * h + 2] = fmaf(xs1, w.z, acc[1][4 * h + 2]);
+                    acc[1][4 * h + 3] = fmaf(xs1, w.w, acc[1][4 * h + 3]);
                 }
             }
         }
+        if (more) stash(b ^ 1);
         __syncthreads();
+        b ^= 1;
     }
-    const float b_lo = (br && lane < E) ? br[lane] : 0.f;
-    const float b_hi = (br && NE > 1 && lane + 32 < E) ? br[lane + 32] : 0.f;
+    // the groups' partial logits -> shared memory as [group][token][expert] (all staging buffers are free now), then
+    // one warp per token adds them in group order
+    float* Ls = rt_smem;                            // kRtSplit x TB x EP floats
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int t = t0 + 4 * warp + i;
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int h = 0; h < EPL / 4; ++h)
+            *reinterpret_cast<float4*>(&Ls[(grp * TB + tk + 4 * i) * EP + eo + 32 * h]) =
+                make_float4(acc[i][4 * h], acc[i][4 * h + 1], acc[i][4 * h + 2], acc[i][4 * h + 3]);
+    __syncthreads();
+    const float b_lo = (br && lane < E) ? br[lane] : 0.f;
+    const float b_hi = (br && lane + 32 < E) ? br[lane + 32] : 0.f;
+    for (int tl = warp; tl < TB; tl += NT / 32) {
+        const int t = t0 + tl;
         if (t < T) {   // uniform across the warp
-            const float l_hi = NE > 1 ? acc[i][NE - 1] + b_hi : 0.f;
-            softmax_select_store(acc[i][0] + b_lo, l_hi, t, q, lane, scores, mask, k_t);
+            float l_lo = b_lo, l_hi = b_hi;
+#pragma unroll
+            for (int g = 0; g < kRtSplit; ++g) {
+                l_lo += Ls[(g * TB + tl) * EP + lane];
+                if (EP > 32) l_hi += Ls[(g * TB + tl) * EP + (lane + 32) % EP];
+            }
+            softmax_select_store(l_lo, l_hi, t, q, lane, scores, mask, k_t);
         }
     }
 }
@@ -152,12 +245,15 @@ __global__ void __launch_bounds__(256) select_kernel(const float* __restrict__ s
 
 // counts[e], offsets[e] and, per chunk of 32 tokens, the number of earlier tokens that selected e
 // (chunk_prefix[c,e]).  One block; deterministic; no atomics, so grouped rows come out in token order.
+// The per-chunk counts wait for the scan in shared memory when they fit (in_smem), else in chunk_prefix itself.
 __global__ void __launch_bounds__(1024) finalize_kernel(const uint64_t* __restrict__ mask, int32_t* __restrict__ counts,
-                                                        int32_t* __restrict__ offsets, int32_t* __restrict__ chunk_prefix,
-                                                        int32_t* __restrict__ counts_out, int T, int E) {
+                                                        int32_t* __restrict__ offsets, int32_t* chunk_prefix,
+                                                        int32_t* __restrict__ counts_out, int T, int E, int in_smem) {
+    extern __shared__ int32_t cnt_dyn[];
     __shared__ int32_t cnt_s[kMaxExperts];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nchunks = (T + kChunk - 1) / kChunk;
+    int32_t* cc = in_smem ? cnt_dyn : chunk_prefix;      // per-chunk counts before the scan
     for (int c = warp; c < nchunks; c += 32) {
         const int t = c * kChunk + lane;
         const uint64_t m = t < T ? mask[t] : 0;
@@ -168,15 +264,15 @@ __global__ void __launch_bounds__(1024) finalize_kernel(const uint64_t* __restri
                 if (e < 32) c_lo = n; else c_hi = n;
             }
         }
-        if (lane < E) chunk_prefix[(size_t)c * E + lane] = c_lo;
-        if (lane + 32 < E) chunk_prefix[(size_t)c * E + lane + 32] = c_hi;
+        if (lane < E) cc[(size_t)c * E + lane] = c_lo;
+        if (lane + 32 < E) cc[(size_t)c * E + lane + 32] = c_hi;
     }
     __syncthreads();
     const int per = (nchunks + 31) / 32;
     for (int e = warp; e < E; e += 32) {
         const int c0 = min(nchunks, lane * per), c1 = min(nchunks, c0 + per);
         int sum = 0;
-        for (int c = c0; c < c1; ++c) sum += chunk_prefix[(size_t)c * E + e];
+        for (int c = c0; c < c1; ++c) sum += cc[(size_t)c * E + e];
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -185,7 +281,7 @@ __global__ void __launch_bounds__(1024) finalize_kernel(const uint64_t* __restri
         }
         int run = incl - sum;
         for (int c = c0; c < c1; ++c) {
-            const int v = chunk_prefix[(size_t)c * E + e];
+            const int v = cc[(size_t)c * E + e];
             chunk_prefix[(size_t)c * E + e] = run;
             run += v;
         }
@@ -232,9 +328,19 @@ static dsmoe_status launch_router_t(const dsmoe_layer_desc& p, const XT* x, cons
         else if (p.E <= 32) router_small_kernel<XT, 32><<<p.T, 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.d, q);
         else router_small_kernel<XT, 64><<<p.T, 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.d, q);
     } else {
-        const int grid = ceil_div(p.T, 32);
-        if (p.E <= 32) router_tile_kernel<XT, 32><<<grid, 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.T, p.d, q);
-        else router_tile_kernel<XT, 64><<<grid, 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.T, p.d, q);
+        const int grid = ceil_div(p.T, kRtTB);
+        static bool attr_set = false;     // per instantiation (XT)
+        if (!attr_set) {
+            DSMOE_CUDA_TRY(cudaFuncSetAttribute(router_tile_kernel<XT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)router_tile_smem<4>()));
+            DSMOE_CUDA_TRY(cudaFuncSetAttribute(router_tile_kernel<XT, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)router_tile_smem<8>()));
+            attr_set = true;
+        }
+        if (p.E <= 32)
+            router_tile_kernel<XT, 4><<<grid, kRtThreads, router_tile_smem<4>(), s>>>(x, Wr, br, scores, mask, k_t, p.T, p.d, q);
+        else
+            router_tile_kernel<XT, 8><<<grid, kRtThreads, router_tile_smem<8>(), s>>>(x, Wr, br, scores, mask, k_t, p.T, p.d, q);
     }
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
@@ -258,7 +364,15 @@ dsmoe_status launch_select(const dsmoe_layer_desc& p, const float* scores, uint6
 
 dsmoe_status launch_finalize(const dsmoe_layer_desc& p, const uint64_t* mask, int32_t* counts, int32_t* offsets,
                              int32_t* chunk_prefix, int32_t* counts_out, cudaStream_t s) {
-    finalize_kernel<<<1, 1024, 0, s>>>(mask, counts, offsets, chunk_prefix, counts_out, p.T, p.E);
+    constexpr size_t kMaxDyn = 160 * 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        DSMOE_CUDA_TRY(cudaFuncSetAttribute(finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDyn));
+        attr_set = true;
+    }
+    const size_t need = (size_t)ceil_div(p.T, kChunk) * p.E * sizeof(int32_t);
+    const int in_smem = need <= kMaxDyn ? 1 : 0;
+    finalize_kernel<<<1, 1024, in_smem ? need : 0, s>>>(mask, counts, offsets, chunk_prefix, counts_out, p.T, p.E, in_smem);
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
 }
