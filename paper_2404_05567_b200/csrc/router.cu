@@ -245,7 +245,10 @@ __global__ void __launch_bounds__(256) select_kernel(const float* __restrict__ s
 
 // counts[e], offsets[e] and, per chunk of 32 tokens, the number of earlier tokens that selected e
 // (chunk_prefix[c,e]).  One block; deterministic; no atomics, so grouped rows come out in token order.
-// The per-chunk counts wait for the scan in shared memory when they fit (in_smem), else in chunk_prefix itself.
+// Step 1: warp w counts chunks w, w+32, ... (lane = token, one ballot per expert), its mask words loaded in batches
+// of 8.  Step 2: warp e scans expert e's counts over the chunks, 32 chunks per warp-wide scan.  Between the steps the
+// counts sit in shared memory as [expert][chunk] (in_smem; row length odd, so both steps are free of bank
+// conflicts) when they fit, else in chunk_prefix itself.
 __global__ void __launch_bounds__(1024) finalize_kernel(const uint64_t* __restrict__ mask, int32_t* __restrict__ counts,
                                                         int32_t* __restrict__ offsets, int32_t* chunk_prefix,
                                                         int32_t* __restrict__ counts_out, int T, int E, int in_smem) {
@@ -253,40 +256,50 @@ __global__ void __launch_bounds__(1024) finalize_kernel(const uint64_t* __restri
     __shared__ int32_t cnt_s[kMaxExperts];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nchunks = (T + kChunk - 1) / kChunk;
-    int32_t* cc = in_smem ? cnt_dyn : chunk_prefix;      // per-chunk counts before the scan
-    for (int c = warp; c < nchunks; c += 32) {
-        const int t = c * kChunk + lane;
-        const uint64_t m = t < T ? mask[t] : 0;
-        int c_lo = 0, c_hi = 0;
-        for (int e = 0; e < E; ++e) {
-            const int n = __popc(__ballot_sync(0xffffffffu, (m >> e) & 1));
-            if (lane == (e & 31)) {
-                if (e < 32) c_lo = n; else c_hi = n;
+    const int S = nchunks | 1;                         // shared-memory row length
+    for (int cb = warp; cb < nchunks; cb += 32 * 8) {
+        uint64_t m[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int c = cb + 32 * j, t = c * kChunk + lane;
+            m[j] = (c < nchunks && t < T) ? mask[t] : 0;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int c = cb + 32 * j;
+            if (c >= nchunks) break;                   // the same for every lane
+            int c_lo = 0, c_hi = 0;
+            for (int e = 0; e < E; ++e) {
+                const int n = __popc(__ballot_sync(0xffffffffu, (m[j] >> e) & 1));
+                if (lane == (e & 31)) {
+                    if (e < 32) c_lo = n; else c_hi = n;
+                }
+            }
+            if (in_smem) {
+                if (lane < E) cnt_dyn[lane * S + c] = c_lo;
+                if (lane + 32 < E) cnt_dyn[(lane + 32) * S + c] = c_hi;
+            } else {
+                if (lane < E) chunk_prefix[(size_t)c * E + lane] = c_lo;
+                if (lane + 32 < E) chunk_prefix[(size_t)c * E + lane + 32] = c_hi;
             }
         }
-        if (lane < E) cc[(size_t)c * E + lane] = c_lo;
-        if (lane + 32 < E) cc[(size_t)c * E + lane + 32] = c_hi;
     }
     __syncthreads();
-    const int per = (nchunks + 31) / 32;
     for (int e = warp; e < E; e += 32) {
-        const int c0 = min(nchunks, lane * per), c1 = min(nchunks, c0 + per);
-        int sum = 0;
-        for (int c = c0; c < c1; ++c) sum += cc[(size_t)c * E + e];
-        int incl = sum;
+        int carry = 0;
+        for (int c0 = 0; c0 < nchunks; c0 += 32) {
+            const int c = c0 + lane;
+            const int v = c < nchunks ? (in_smem ? cnt_dyn[e * S + c] : chunk_prefix[(size_t)c * E + e]) : 0;
+            int incl = v;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += u;
+            }
+            if (c < nchunks) chunk_prefix[(size_t)c * E + e] = carry + incl - v;
+            carry += __shfl_sync(0xffffffffu, incl, 31);
         }
-        int run = incl - sum;
-        for (int c = c0; c < c1; ++c) {
-            const int v = cc[(size_t)c * E + e];
-            chunk_prefix[(size_t)c * E + e] = run;
-            run += v;
-        }
-        const int total = __shfl_sync(0xffffffffu, incl, 31);
-        if (lane == 0) cnt_s[e] = total;
+        if (lane == 0) cnt_s[e] = carry;
     }
     __syncthreads();
     if (warp == 0) {
@@ -370,7 +383,7 @@ dsmoe_status launch_finalize(const dsmoe_layer_desc& p, const uint64_t* mask, in
         DSMOE_CUDA_TRY(cudaFuncSetAttribute(finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDyn));
         attr_set = true;
     }
-    const size_t need = (size_t)ceil_div(p.T, kChunk) * p.E * sizeof(int32_t);
+    const size_t need = (size_t)(ceil_div(p.T, kChunk) | 1) * p.E * sizeof(int32_t);
     const int in_smem = need <= kMaxDyn ? 1 : 0;
     finalize_kernel<<<1, 1024, in_smem ? need : 0, s>>>(mask, counts, offsets, chunk_prefix, counts_out, p.T, p.E, in_smem);
     DSMOE_CUDA_TRY(cudaGetLastError());
