@@ -198,9 +198,11 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
 
     // grouped path: duplicate tokens per selected expert, run the experts, aggregate
     DSMOE_TRY(launch_finalize(p, mask, counts, offsets, chunk_prefix, counts_out, s));
-    DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, ws + L.xp, s));
+    // the tensor-core path needs no grouped copy of the tokens: its up-projection gathers rows of x by row_token
+    DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows,
+                             fast ? nullptr : ws + L.xp, s));
     if (fast)
-        DSMOE_TRY(launch_mlp_umma(p, ws + L.xp, packed, offsets, ws + L.h, ws + L.yp, dev_status, s));
+        DSMOE_TRY(launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, ws + L.yp, dev_status, s, x, row_token));
     else
         DSMOE_TRY(launch_mlp_generic(p, ws + L.xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h), ws + L.yp, s));
     return launch_combine(p, ws + L.yp, row_gate, token_rows, k_t, out, s);

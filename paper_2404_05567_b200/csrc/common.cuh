@@ -76,8 +76,10 @@ dsmoe_status timing_enable(int on);
 dsmoe_status timing_last(float* ms, int n_max, int* n);
 bool umma_supported(const dsmoe_layer_desc& p);   // bf16, d and H multiples of 64
 // Grouped expert MLPs on expert-sorted rows: h = GeLU(xp.W1[e]) (bf16, in `hbuf`), yp = h.W2[e].
+// With row_token (and x), the up-projection gathers its rows from x by index and xp is not read.
 dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,
-                             void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s);
+                             void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s, const void* x = nullptr,
+                             const int32_t* row_token = nullptr);
 // Whole-layer paths that need no grouping (all experts selected, or few tokens).  *done = false
 // means "not taken": the caller continues with the grouped path.
 // Whole layer for few tokens (T <= 128) in one cooperative launch, router included.

@@ -26,11 +26,13 @@ constexpr int BM = 128, BK = 64, BN = 256, STAGES = 4, MAX_STAGES = 16;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int NUM_THREADS = 192;
+constexpr int GATHER_WARPS = 8;
+constexpr int GATHER_THREADS = NUM_THREADS + 32 * GATHER_WARPS;   // umma_gemm_kernel with more warps that gather the rows of A
 constexpr int SMALL_THREADS = 448;    // small_layer_kernel: 2 + 4 warps as above, plus 8 warps that share the epilogue arithmetic
 constexpr int kEpiThreads = SMALL_THREADS - 64;
 constexpr int TMEM_COLS = 512;
 constexpr int RING_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);   // operand ring: 4 x 48 KB, or more, smaller slots
-constexpr int SHARED_BYTES = 4096 + 256;                                     // barriers and small tables (struct Shared)
+constexpr int SHARED_BYTES = 6144 + 256;                                     // barriers and small tables (struct Shared)
 constexpr int STG_BYTES = BM * 36 * 4;                                 // epilogue staging tile: T rows x (32..256 + 4) floats
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)RING_BYTES + SHARED_BYTES + STG_BYTES;
 constexpr size_t SMEM_GEMM_BYTES = 1024 + (size_t)RING_BYTES + SHARED_BYTES;   // umma_gemm_kernel needs no staging tile
@@ -63,6 +65,11 @@ struct GemmParams {
     long long ld_out;        // elements
     int out_f32;
     int32_t* dev_status;
+    // grouped, optional: row r of A is row gather[r] of the [gather_rows, k_per_expert] bf16 tensor gather_src; four
+    // extra warps then fetch the A tiles themselves (the kernel is launched with GATHER_THREADS) and tmA is unused
+    const int32_t* gather;
+    const void* gather_src;
+    int gather_rows;
 };
 
 // Tensor maps of one packed weight tensor [E, n, k] with boxes of 16, 32, 64, 128 and 256 rows: a tile of
@@ -95,6 +102,7 @@ struct Shared {
     uint32_t tmem_base;
     volatile int abort_flag;
     int bad_offsets;
+    int rowtok[GATHER_WARPS][BM / (GATHER_WARPS / STAGES)];                   // umma_gemm_kernel, gathered A: the source row of each tile row, per gathering warp
     int tile_prefix[kMaxExperts + 1];
     int seg0[kMaxExperts], seg1[kMaxExperts];
     unsigned long long active_mask;
@@ -183,7 +191,7 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& P, const Shared& s
     return t;
 }
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(GATHER_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ BMaps tmB, const GemmParams P) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -195,7 +203,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&sh.full[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh.full[s]), P.gather ? 1 + 32 * (GATHER_WARPS / STAGES) : 1);   // + one arrival per thread of the gathering warps
             ptx::mbar_init(ptx::smem_u32(&sh.empty[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -254,7 +262,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         break;
                     }
                     const uint32_t bar = ptx::smem_u32(&sh.full[s]);
-                    ptx::mbar_expect_tx(bar, A_STAGE_BYTES + (uint32_t)t.bn * BK * 2);
+                    ptx::mbar_expect_tx(bar, (P.gather ? 0u : (uint32_t)A_STAGE_BYTES) + (uint32_t)t.bn * BK * 2);
                     int a_col, b_e, b_k;
                     if (P.mode == GEMM_DENSE_DOWN) {
                         b_e = i / kbpe;
@@ -265,7 +273,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         b_k = i * BK;
                         a_col = b_k;
                     }
-                    ptx::tma_load_2d(smA + s * A_STAGE_BYTES, &tmA, bar, a_col, t.row0);
+                    if (!P.gather) ptx::tma_load_2d(smA + s * A_STAGE_BYTES, &tmA, bar, a_col, t.row0);
                     // full-width tiles take the one 256-row copy directly (measurably faster than walking the
                     // box sizes); only a ragged last column tile needs the decomposition
                     if (t.bn == BN) ptx::tma_load_3d(smB + s * B_STAGE_BYTES, &tmB.m[4], bar, b_k, t.n0, b_e);
@@ -318,6 +326,51 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     acc = 0;
                     aph ^= 1u;
                 }
+            }
+        }
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------ gather (8 warps, grouped up-projection only)
+        // Warps j and j + 4 bring the two halves of the A tiles of the ring stages j, j + 4, ... of this CTA's
+        // sequence: per stage, 16 cp.async instructions each, an instruction covering 4 rows x 128 bytes (8 lanes x 16 bytes per row), written in the
+        // 128-byte-swizzle order the MMA descriptors expect (chunk c of row r sits at chunk c ^ (r % 8)).  It then
+        // waits for its copies, makes them visible to the tensor core's proxy and arrives at the stage's barrier;
+        // while it waits, the other three warps' stages are in flight.
+        constexpr int PARTS = GATHER_WARPS / STAGES, ROWS = BM / PARTS;   // warps per stage, rows per warp
+        const int team = (warp - 6) % STAGES, part = (warp - 6) / STAGES;
+        int* rowtok = sh.rowtok[warp - 6];
+        const int lr = lane >> 3, lc = lane & 7;
+        int n = 0;                       // stages of the sequence seen so far
+        bool alive = true;
+        for (int id = blockIdx.x; id < ntiles && alive; id += gridDim.x) {
+            const Tile t = decode_tile(P, sh, id);
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < ROWS / 32; ++j) {
+                const int r = part * ROWS + lane + 32 * j;
+                const int tok = P.gather[t.row0 + (r < t.rows_valid ? r : 0)];   // rows past the segment: nobody reads them
+                rowtok[lane + 32 * j] = min(max(tok, 0), P.gather_rows - 1);
+            }
+            __syncwarp();
+            for (int i = 0; i < t.nk; ++i, ++n) {
+                if ((n & (STAGES - 1)) != team) continue;
+                const int s = n & (STAGES - 1);
+                const uint32_t ph = (uint32_t)(n / STAGES) & 1u;
+                if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
+                    alive = false;
+                    break;
+                }
+                const uint32_t dst0 = smA + s * A_STAGE_BYTES;
+                const char* src0 = static_cast<const char*>(P.gather_src) + (size_t)i * (BK * 2) + lc * 16;
+#pragma unroll 8
+                for (int jj = 0; jj < ROWS / 4; ++jj) {
+                    const int rl = jj * 4 + lr, r = part * ROWS + rl;
+                    ptx::cp_async16(dst0 + (uint32_t)r * (BK * 2) + (uint32_t)((lc ^ (r & 7)) << 4),
+                                    src0 + (size_t)rowtok[rl] * P.k_per_expert * 2);
+                }
+                ptx::cp_async_commit();
+                ptx::cp_async_wait<0>();
+                ptx::fence_proxy_async();
+                ptx::mbar_arrive(ptx::smem_u32(&sh.full[s]));
             }
         }
     } else {
@@ -1390,7 +1443,7 @@ dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams&
     }
     const bool timed = g_timing.on && g_timing.n < kMaxTimed;
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
-    umma_gemm_kernel<<<grid, NUM_THREADS, SMEM_GEMM_BYTES, s>>>(a, b, P);
+    umma_gemm_kernel<<<grid, P.gather ? GATHER_THREADS : NUM_THREADS, SMEM_GEMM_BYTES, s>>>(a, b, P);
     DSMOE_CUDA_TRY(cudaGetLastError());
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.stop[g_timing.n++], s));
     return DSMOE_OK;
@@ -1435,7 +1488,8 @@ bool umma_supported(const dsmoe_layer_desc& p) {
 }
 
 dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,
-                             void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s) {
+                             void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s, const void* x,
+                             const int32_t* row_token) {
     if (p.T == 0) return DSMOE_OK;
     if (!umma_supported(p)) return DSMOE_ERR_UNSUPPORTED;
     const size_t amax = amax_of(p);
@@ -1443,11 +1497,16 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
     const __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
     CUtensorMap mA1, mA2;
     BMaps mB1, mB2;
-    DSMOE_TRY(make_map_2d(&mA1, xp, amax, p.d, BM));
+    // with row_token, the up-projection fetches its rows straight from x (no grouped copy of the tokens); its A
+    // tensor map is then unused, any valid one will do
+    DSMOE_TRY(make_map_2d(&mA1, row_token ? hbuf : xp, amax, row_token ? p.H : p.d, BM));
     DSMOE_TRY(make_bmaps(&mB1, w1t, p.E, p.H, p.d));
     DSMOE_TRY(make_map_2d(&mA2, hbuf, amax, p.H, BM));
     DSMOE_TRY(make_bmaps(&mB2, w2t, p.E, p.d, p.H));
     GemmParams up{GEMM_GROUPED, EPI_GELU, p.E, p.H, p.d, (int)amax, offsets, nullptr, hbuf, p.H, 0, dev_status};
+    up.gather = row_token;
+    up.gather_src = x;
+    up.gather_rows = p.T;
     GemmParams down{GEMM_GROUPED, EPI_STORE, p.E, p.d, p.H, (int)amax, offsets, nullptr, yp, p.d, 0, dev_status};
     DSMOE_TRY(launch_gemm(mA1, mB1, up, sm_count(), s));
     DSMOE_TRY(launch_gemm(mA2, mB2, down, sm_count(), s));

@@ -79,6 +79,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, 
         : "memory");
 }
 
+// ---------------------------------------------------------------- cp.async (16-byte copies issued by ordinary threads)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // L2 policy for data that is read once: its lines are the first to be replaced, so a long stream does not push
 // everything else (small operands, instructions) out of L2.
 __device__ __forceinline__ uint64_t policy_evict_first() {
