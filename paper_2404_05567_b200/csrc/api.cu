@@ -51,6 +51,7 @@ WsLayout ws_layout(const dsmoe_layer_desc& p) {
     // fp32 partial sums of the small-T path: (CTA, 2 column ranges, T, 256)
     L.partial = take(p.T <= kSmallMaxT ? (size_t)kSmallMaxCtas * 2 * T * 256 * 4 : 0);
     L.sync = take(64);                   // grid-barrier counters of the small-T kernel
+    L.router = take(router_umma_supported(p) ? router_umma_scratch(p) : 0);   // tensor-core router: split Wr, partial logits
     L.total = off;
     return L;
 }
@@ -189,7 +190,10 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     if (fast && small_supported(p))
         return launch_layer_small(p, x, Wr, br, packed, scores, mask, k_t, counts_out, out, ws, L, dev_status, s);
 
-    DSMOE_TRY(launch_router(p, x, Wr, br, scores, mask, k_t, s));
+    if (fast && router_umma_supported(p))
+        DSMOE_TRY(launch_router_umma(p, x, Wr, br, scores, mask, k_t, ws + L.router, dev_status, s));
+    else
+        DSMOE_TRY(launch_router(p, x, Wr, br, scores, mask, k_t, s));
     if (fast) {
         bool done = false;
         DSMOE_TRY(launch_layer_umma(p, x, packed, scores, mask, k_t, counts_out, out, ws, L, dev_status, s, &done));

@@ -43,7 +43,7 @@ static inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; 
 // Byte offsets of every internal buffer inside the caller's workspace.
 struct WsLayout {
     size_t scores, mask, k_t, counts, offsets, chunk_prefix, row_token, row_gate, token_rows;
-    size_t xp, h, yp, partial, sync, total;
+    size_t xp, h, yp, partial, sync, router, total;
 };
 WsLayout ws_layout(const dsmoe_layer_desc& p);
 
@@ -75,6 +75,13 @@ void timing_reset();
 dsmoe_status timing_enable(int on);
 dsmoe_status timing_last(float* ms, int n_max, int* n);
 bool umma_supported(const dsmoe_layer_desc& p);   // bf16, d and H multiples of 64
+// Router for many tokens with the logits on the tensor cores (bf16 x; Wr split exactly into three bf16 terms, fp32
+// accumulation), then softmax and selection.  `scratch` holds router_umma_scratch(p) bytes.
+bool router_umma_supported(const dsmoe_layer_desc& p);
+size_t router_umma_scratch(const dsmoe_layer_desc& p, size_t* split_bytes = nullptr);
+dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
+                                float* scores, uint64_t* mask, int32_t* k_t, char* scratch, int32_t* dev_status,
+                                cudaStream_t s);
 // Grouped expert MLPs on expert-sorted rows: h = GeLU(xp.W1[e]) (bf16, in `hbuf`), yp = h.W2[e].
 // With row_token (and x), the up-projection gathers its rows from x by index and xp is not read.
 dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,

@@ -1435,13 +1435,14 @@ struct Timing {
     cudaEvent_t start[kMaxTimed], stop[kMaxTimed];
 } g_timing;
 
-dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams& P, int grid, cudaStream_t s) {
+dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams& P, int grid, cudaStream_t s,
+                         bool may_time = true) {
     static bool attr_set = false;
     if (!attr_set) {
         DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_BYTES));
         attr_set = true;
     }
-    const bool timed = g_timing.on && g_timing.n < kMaxTimed;
+    const bool timed = may_time && g_timing.on && g_timing.n < kMaxTimed;
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
     umma_gemm_kernel<<<grid, P.gather ? GATHER_THREADS : NUM_THREADS, SMEM_GEMM_BYTES, s>>>(a, b, P);
     DSMOE_CUDA_TRY(cudaGetLastError());
@@ -1449,7 +1450,74 @@ dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams&
     return DSMOE_OK;
 }
 
+// ---------------------------------------------------------------- router logits on the tensor cores
+// Wr (fp32) is written as the exact sum of three bf16 terms, w = w1 + w2 + w3 (w1 = bf16(w), w2 = bf16(w - w1),
+// w3 = bf16(w - w1 - w2): 3 x 8 significant bits cover fp32's 24).  x is bf16, so every product x.w_i is exact in
+// fp32 and the three sums accumulate in fp32: the logits are as accurate as an fp32 dot product, at tensor-core
+// speed.  The three terms sit side by side along N: B = [3 * EP, d] bf16, K-major, EP = E rounded up to 32 or 64.
+__global__ void __launch_bounds__(256) router_split_kernel(const float* __restrict__ Wr, __nv_bfloat16* __restrict__ out,
+                                                           int d, int E, int EP) {
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= (long long)EP * d) return;
+    const int e = (int)(idx / d), k = (int)(idx % d);
+    const float w = e < E ? Wr[(size_t)k * E + e] : 0.f;
+    const __nv_bfloat16 w1 = __float2bfloat16_rn(w);
+    const float r1 = w - __bfloat162float(w1);
+    const __nv_bfloat16 w2 = __float2bfloat16_rn(r1);
+    const float r2 = r1 - __bfloat162float(w2);
+    out[idx] = w1;
+    out[idx + (long long)EP * d] = w2;
+    out[idx + 2ll * EP * d] = __float2bfloat16_rn(r2);
+}
+
+// logits = (s1 + s2) + s3 + bias per expert, then softmax and selection: one warp per token
+__global__ void __launch_bounds__(256) router_finish_kernel(const float* __restrict__ sums, const float* __restrict__ br,
+                                                            float* __restrict__ scores, uint64_t* __restrict__ mask,
+                                                            int32_t* __restrict__ k_t, int T, int EP, SelParams q) {
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const float* row = sums + (size_t)t * 3 * EP;
+    const bool v_lo = lane < q.E, v_hi = lane + 32 < q.E;
+    float l_lo = 0.f, l_hi = 0.f;
+    if (v_lo) l_lo = ((row[lane] + row[EP + lane]) + row[2 * EP + lane]) + (br ? br[lane] : 0.f);
+    if (v_hi) l_hi = ((row[lane + 32] + row[EP + lane + 32]) + row[2 * EP + lane + 32]) + (br ? br[lane + 32] : 0.f);
+    softmax_select_store(l_lo, l_hi, t, q, lane, scores, mask, k_t);
+}
+
 }  // namespace
+
+size_t router_umma_scratch(const dsmoe_layer_desc& p, size_t* split_bytes) {
+    const size_t EP = p.E <= 32 ? 32 : 64;
+    const size_t a = align_up(3 * EP * (size_t)p.d * 2, 256);
+    if (split_bytes) *split_bytes = a;
+    return a + align_up((size_t)p.T * 3 * EP * 4, 256);
+}
+
+bool router_umma_supported(const dsmoe_layer_desc& p) { return umma_supported(p) && p.T > 256; }
+
+dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
+                                float* scores, uint64_t* mask, int32_t* k_t, char* scratch, int32_t* dev_status,
+                                cudaStream_t s) {
+    const int EP = p.E <= 32 ? 32 : 64;
+    size_t split_bytes = 0;
+    router_umma_scratch(p, &split_bytes);
+    __nv_bfloat16* wsplit = reinterpret_cast<__nv_bfloat16*>(scratch);
+    float* sums = reinterpret_cast<float*>(scratch + split_bytes);
+    router_split_kernel<<<ceil_div(EP * p.d, 256), 256, 0, s>>>(Wr, wsplit, p.d, p.E, EP);
+    DSMOE_CUDA_TRY(cudaGetLastError());
+    CUtensorMap mA;
+    BMaps mB;
+    DSMOE_TRY(make_map_2d(&mA, x, p.T, p.d, BM));
+    DSMOE_TRY(make_bmaps(&mB, wsplit, 1, 3 * EP, p.d));
+    GemmParams g{GEMM_DENSE_DOWN, EPI_STORE, 1, 3 * EP, p.d, p.T, nullptr, nullptr, sums, 3 * EP, 1, dev_status};
+    const int tiles = ceil_div(p.T, BM);
+    DSMOE_TRY(launch_gemm(mA, mB, g, tiles < sm_count() ? tiles : sm_count(), s, false));
+    router_finish_kernel<<<ceil_div(p.T, 8), 256, 0, s>>>(sums, br, scores, mask, k_t, p.T, EP,
+                                                         SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k});
+    DSMOE_CUDA_TRY(cudaGetLastError());
+    return DSMOE_OK;
+}
 
 #ifdef DSMOE_TRACE
 extern "C" __attribute__((visibility("default"))) int dsmoe_trace_read(unsigned long long* out) {

@@ -86,7 +86,15 @@ __global__ void __launch_bounds__(128) combine_bf16_kernel(const uint4* __restri
         float acc[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-        for (int i = 0; i < k; ++i) fma8(acc, __ldg(yp + (size_t)rows_s[i] * nvec + v), gate_s[i]);
+        // four rows' loads are issued before their first use (past the k-th row, row 0 is fetched again and not used)
+        for (int i = 0; i < k; i += 4) {
+            uint4 y[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) y[j] = __ldg(yp + (size_t)rows_s[i + j < k ? i + j : 0] * nvec + v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (i + j < k) fma8(acc, y[j], gate_s[i + j]);
+        }
         if (OUT_F32) {
             float4* o = reinterpret_cast<float4*>(out) + ((size_t)t * nvec + v) * 2;
             o[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
