@@ -244,60 +244,56 @@ __global__ void __launch_bounds__(256) select_kernel(const float* __restrict__ s
 }
 
 // counts[e], offsets[e] and, per chunk of 32 tokens, the number of earlier tokens that selected e
-// (chunk_prefix[c,e]).  One block; deterministic; no atomics, so grouped rows come out in token order.
-// Step 1: warp w counts chunks w, w+32, ... (lane = token, one ballot per expert), its mask words loaded in batches
-// of 8.  Step 2: warp e scans expert e's counts over the chunks, 32 chunks per warp-wide scan.  Between the steps the
-// counts sit in shared memory as [expert][chunk] (in_smem; row length odd, so both steps are free of bank
-// conflicts) when they fit, else in chunk_prefix itself.
-__global__ void __launch_bounds__(1024) finalize_kernel(const uint64_t* __restrict__ mask, int32_t* __restrict__ counts,
-                                                        int32_t* __restrict__ offsets, int32_t* chunk_prefix,
-                                                        int32_t* __restrict__ counts_out, int T, int E, int in_smem) {
-    extern __shared__ int32_t cnt_dyn[];
+// (chunk_prefix[c,e]).  Deterministic; no atomics, so grouped rows come out in token order.  Two kernels:
+// chunk_count_kernel, one warp per chunk (lane = token, one ballot per expert), leaves the chunk's counts in
+// chunk_prefix[c,:]; finalize_kernel, one block, turns them into exclusive prefixes over the chunks (warp e scans
+// expert e, 32 chunks per warp-wide scan) and writes the totals and their offsets.
+__global__ void __launch_bounds__(256) chunk_count_kernel(const uint64_t* __restrict__ mask, int32_t* __restrict__ chunk_prefix,
+                                                          int T, int E) {
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (c * kChunk >= T) return;
+    const int t = c * kChunk + lane;
+    const uint64_t m = t < T ? mask[t] : 0;
+    int c_lo = 0, c_hi = 0;
+    for (int e = 0; e < E; ++e) {
+        const int n = __popc(__ballot_sync(0xffffffffu, (m >> e) & 1));
+        if (lane == (e & 31)) {
+            if (e < 32) c_lo = n; else c_hi = n;
+        }
+    }
+    if (lane < E) chunk_prefix[(size_t)c * E + lane] = c_lo;
+    if (lane + 32 < E) chunk_prefix[(size_t)c * E + lane + 32] = c_hi;
+}
+
+__global__ void __launch_bounds__(1024) finalize_kernel(int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+                                                        int32_t* __restrict__ chunk_prefix, int32_t* __restrict__ counts_out,
+                                                        int T, int E) {
     __shared__ int32_t cnt_s[kMaxExperts];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nchunks = (T + kChunk - 1) / kChunk;
-    const int S = nchunks | 1;                         // shared-memory row length
-    for (int cb = warp; cb < nchunks; cb += 32 * 8) {
-        uint64_t m[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int c = cb + 32 * j, t = c * kChunk + lane;
-            m[j] = (c < nchunks && t < T) ? mask[t] : 0;
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int c = cb + 32 * j;
-            if (c >= nchunks) break;                   // the same for every lane
-            int c_lo = 0, c_hi = 0;
-            for (int e = 0; e < E; ++e) {
-                const int n = __popc(__ballot_sync(0xffffffffu, (m[j] >> e) & 1));
-                if (lane == (e & 31)) {
-                    if (e < 32) c_lo = n; else c_hi = n;
-                }
-            }
-            if (in_smem) {
-                if (lane < E) cnt_dyn[lane * S + c] = c_lo;
-                if (lane + 32 < E) cnt_dyn[(lane + 32) * S + c] = c_hi;
-            } else {
-                if (lane < E) chunk_prefix[(size_t)c * E + lane] = c_lo;
-                if (lane + 32 < E) chunk_prefix[(size_t)c * E + lane + 32] = c_hi;
-            }
-        }
-    }
-    __syncthreads();
     for (int e = warp; e < E; e += 32) {
         int carry = 0;
-        for (int c0 = 0; c0 < nchunks; c0 += 32) {
-            const int c = c0 + lane;
-            const int v = c < nchunks ? (in_smem ? cnt_dyn[e * S + c] : chunk_prefix[(size_t)c * E + e]) : 0;
-            int incl = v;
+        for (int c0 = 0; c0 < nchunks; c0 += 32 * 4) {
+            // four scans' worth of loads are issued together
+            int v[4];
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int u = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += u;
+            for (int j = 0; j < 4; ++j) {
+                const int c = c0 + 32 * j + lane;
+                v[j] = c < nchunks ? chunk_prefix[(size_t)c * E + e] : 0;
             }
-            if (c < nchunks) chunk_prefix[(size_t)c * E + e] = carry + incl - v;
-            carry += __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int c = c0 + 32 * j + lane;
+                int incl = v[j];
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int u = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += u;
+                }
+                if (c < nchunks) chunk_prefix[(size_t)c * E + e] = carry + incl - v[j];
+                carry += __shfl_sync(0xffffffffu, incl, 31);
+            }
         }
         if (lane == 0) cnt_s[e] = carry;
     }
@@ -377,15 +373,12 @@ dsmoe_status launch_select(const dsmoe_layer_desc& p, const float* scores, uint6
 
 dsmoe_status launch_finalize(const dsmoe_layer_desc& p, const uint64_t* mask, int32_t* counts, int32_t* offsets,
                              int32_t* chunk_prefix, int32_t* counts_out, cudaStream_t s) {
-    constexpr size_t kMaxDyn = 160 * 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
-        DSMOE_CUDA_TRY(cudaFuncSetAttribute(finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDyn));
-        attr_set = true;
+    const int nchunks = ceil_div(p.T, kChunk);
+    if (nchunks > 0) {
+        chunk_count_kernel<<<ceil_div(nchunks, 8), 256, 0, s>>>(mask, chunk_prefix, p.T, p.E);
+        DSMOE_CUDA_TRY(cudaGetLastError());
     }
-    const size_t need = (size_t)(ceil_div(p.T, kChunk) | 1) * p.E * sizeof(int32_t);
-    const int in_smem = need <= kMaxDyn ? 1 : 0;
-    finalize_kernel<<<1, 1024, in_smem ? need : 0, s>>>(mask, counts, offsets, chunk_prefix, counts_out, p.T, p.E, in_smem);
+    finalize_kernel<<<1, 1024, 0, s>>>(counts, offsets, chunk_prefix, counts_out, p.T, p.E);
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
 }
