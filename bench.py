@@ -29,6 +29,7 @@ WORKLOADS = {
     "c2_t1": ("c2", dict(T=1)), "c2_t8": ("c2", dict(T=8)), "c2_t32": ("c2", dict(T=32)),
     "c3": ("c3", {}), "c4": ("c4", {}), "c5": ("c5", dict(eps=0.01)),
 }
+NCU_TRAFFIC_BYTES = {"c2_t32": 276.4e6, "c3": 1023.2e6}
 DEFAULT_STEPS = {"c2_t1": 1000, "c2_t8": 1000, "c2_t32": 1000, "c3": 100, "c4": 50, "c5": 50}
 METRIC = "moe_layer_tokens_per_s"
 
@@ -277,7 +278,9 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
         roof = dict(bound="tensor", achieved=algo / (launch_ms * 1e-3) / 1e12, peak=P["tf_sustained"],
                     unit="TFLOP/s", peak_source=P["source"] + " (sustained bf16)", kernel="umma_gemm_kernel")
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = None
+    # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
+    # summarised under profiles/ (c3: mean of the up- and down-projection launches); null where no capture was taken
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(name)
     roof["launch_ms"] = launch_ms / per_step_launches
     roof["launch_ms_each"] = [float(v) for v in durs.mean(axis=0)]
     roof["launches_per_step"] = per_step_launches
@@ -287,7 +290,7 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
     roof["step_frac"] = ((algo / step_s / 1e9) if decode else (algo / step_s / 1e12)) / roof["peak"]
 
     res = dict(value=value, ms_per_step=ms_total / steps, clocks=clocks, roofline=roof, A=A, active_experts=n_act,
-               launches_per_step=(1 if decode else (3 if s.mode == gi.MODE_ALL else 7)), spec=s)
+               launches_per_step=(1 if decode else (5 if s.mode == gi.MODE_ALL else 9)), spec=s)
 
     # ---- end to end through the host-buffer entry point
     if with_e2e:
