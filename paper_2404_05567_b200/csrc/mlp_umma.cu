@@ -51,6 +51,10 @@ constexpr int kFixBatch = 24;        // partial tiles a fix-up thread loads at o
 #endif
 constexpr int kSmallInflightBytes = DSMOE_SMALL_INFLIGHT;
 static_assert(kSmallInflightBytes <= RING_BYTES, "in-flight bytes are ring bytes");
+#ifndef DSMOE_SMALL_L2_PREFETCH
+#define DSMOE_SMALL_L2_PREFETCH (384 * 1024)
+#endif
+constexpr int kSmallL2PrefetchBytes = DSMOE_SMALL_L2_PREFETCH;   // small-T kernel: W2 bytes a CTA asks into L2 before the middle barrier
 constexpr int kSpecMinT = 8;         // tokens from which the small-T kernel streams ahead of its router
 
 struct GemmParams {
@@ -887,6 +891,29 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 if (++i_cur == t.nk) {
                     i_cur = 0;
                     have = it.next(P, g->active, g->n_act, t);
+                }
+            }
+            // Between the two projections HBM has nothing to do for several microseconds (epilogues, the slowest
+            // CTA, the barrier), and the ring is full.  So the next weight tiles of this CTA's sequence are asked
+            // into L2 meanwhile: the down-projection then finds them there instead of in DRAM.  All CTAs together
+            // ask for well under half of L2.  (Not for the fewest tokens: there the gap is short and the requests only
+            // compete with the ring's own.)
+            if (alive && have && P.spec) {
+                SmallIter pit = it;
+                SmallTile pt = t;
+                int pi = i_cur;
+                bool phave = have;
+                const int kbpe = P.H / BK;
+                for (int bytes = 0; phave && bytes < kSmallL2PrefetchBytes;) {
+                    if ((pt.bn & (pt.bn - 1)) == 0) {
+                        const int gb = pt.kstart + pi;
+                        ptx::tma_prefetch_3d(&tmW2.m[__ffs(pt.bn) - 5], (gb % kbpe) * BK, pt.n0, g->active[gb / kbpe]);
+                    }
+                    bytes += pt.bn * BK * 2;
+                    if (++pi == pt.nk) {
+                        pi = 0;
+                        phave = pit.next(P, g->active, g->n_act, pt);
+                    }
                 }
             }
             TRACE(5);
