@@ -32,9 +32,15 @@ constexpr int SMALL_THREADS = 448;    // small_layer_kernel: 2 + 4 warps as abov
 constexpr int kEpiThreads = SMALL_THREADS - 64;
 constexpr int TMEM_COLS = 512;
 constexpr int RING_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);   // operand ring: 4 x 48 KB, or more, smaller slots
+#ifndef DSMOE_SMALL_INFLIGHT
+#define DSMOE_SMALL_INFLIGHT (144 * 1024)
+#endif
+constexpr int SMALL_RING_BYTES = DSMOE_SMALL_INFLIGHT;                 // small_layer_kernel's ring
 constexpr int SHARED_BYTES = 6144 + 256;                                     // barriers and small tables (struct Shared)
 constexpr int STG_BYTES = BM * 36 * 4;                                 // epilogue staging tile: T rows x (32..256 + 4) floats
-constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)RING_BYTES + SHARED_BYTES + STG_BYTES;
+// small_layer_kernel asks only for the ring bytes it keeps in flight: what it leaves stays with the SM's L1, which
+// serves the kernel's many small loads (its parameters' copy, the router's operands)
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)SMALL_RING_BYTES + SHARED_BYTES + STG_BYTES;
 constexpr size_t SMEM_GEMM_BYTES = 1024 + (size_t)RING_BYTES + SHARED_BYTES;   // umma_gemm_kernel needs no staging tile
 
 enum { GEMM_GROUPED = 0, GEMM_DENSE_UP = 1, GEMM_DENSE_DOWN = 2 };
@@ -46,10 +52,7 @@ constexpr int kFixBatch = 24;        // partial tiles a fix-up thread loads at o
 // small-T kernel: bytes of loads a CTA keeps in flight (<= RING_BYTES).  Four 36 KB slots per SM already cover the
 // bandwidth-delay product; a deeper ring only lengthens the queues that the router's loads, the grid barriers and
 // instruction fetches wait in.
-#ifndef DSMOE_SMALL_INFLIGHT
-#define DSMOE_SMALL_INFLIGHT (144 * 1024)
-#endif
-constexpr int kSmallInflightBytes = DSMOE_SMALL_INFLIGHT;
+constexpr int kSmallInflightBytes = SMALL_RING_BYTES;
 static_assert(kSmallInflightBytes <= RING_BYTES, "in-flight bytes are ring bytes");
 #ifndef DSMOE_SMALL_L2_PREFETCH
 #define DSMOE_SMALL_L2_PREFETCH (384 * 1024)
@@ -738,8 +741,8 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
-    Shared& sh = *reinterpret_cast<Shared*>(smem_raw + (base - raw) + RING_BYTES);
-    float* stg = reinterpret_cast<float*>(smem_raw + (base - raw) + RING_BYTES + SHARED_BYTES);
+    Shared& sh = *reinterpret_cast<Shared*>(smem_raw + (base - raw) + SMALL_RING_BYTES);
+    float* stg = reinterpret_cast<float*>(smem_raw + (base - raw) + SMALL_RING_BYTES + SHARED_BYTES);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x;
 
