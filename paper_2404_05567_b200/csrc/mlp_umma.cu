@@ -1615,7 +1615,11 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
 // fix-up.
 bool small_supported(const dsmoe_layer_desc& p) {
     const int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
-    return umma_supported(p) && p.T >= 1 && p.T <= kSmallMaxT && p.T <= G && ceil_div(p.d, 64) <= G;
+    if (!(umma_supported(p) && p.T >= 1 && p.T <= kSmallMaxT && p.T <= G && ceil_div(p.d, 64) <= G)) return false;
+    // the router's second half fetches all slice sums of a warp's tokens in one batch of 16 (small_router_pass)
+    int KS = 1;
+    while (KS < 16 && KS * 2 * p.T <= G) KS *= 2;
+    return KS * ceil_div(p.T, kEpiThreads / 32) <= 16;
 }
 
 dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
