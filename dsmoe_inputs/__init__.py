@@ -116,7 +116,7 @@ def as_f32(a: np.ndarray) -> np.ndarray:
 # Workload recipes
 # --------------------------------------------------------------------------
 
-MODE_THRESHOLD, MODE_TOPK, MODE_ALL = 0, 1, 2
+MODE_THRESHOLD, MODE_TOPK, MODE_ALL, MODE_THRESHOLD_TOPK = 0, 1, 2, 3
 
 
 @dataclass

@@ -66,12 +66,36 @@ void oracle_router_scores(const void *x, int dtype, const float *Wr, const float
 /*
  * Selection on fp32 scores ("Sparse Inference" paragraph; footnote on normalised
  * probability).  mode 0: threshold, S > eps, or S*N > eps with one fp32 multiply when
- * eps_normalized; mode 1: the K highest scores, ties to the lower index; mode 2: all.
+ * eps_normalized; mode 1: the K highest scores, ties to the lower index; mode 2: all;
+ * mode 3: threshold, batch average of the counts as K, then mode 1 (see below).
  * min_k = 1 keeps the lowest-index argmax of a token that selected nothing.
  * mask[t] has bit e set iff expert e is selected; k_t[t] = popcount.
  */
 void oracle_select(const float *scores, int64_t T, int64_t E, int mode, float eps,
                    int eps_normalized, int K, int min_k, uint64_t *mask, int32_t *k_t) {
+    if (mode == 3) {
+        /* Threshold-TopK ("Expert Sampling Strategy" paragraph): threshold the normalised
+         * probability, count the experts this activates per token, take the average over
+         * the batch as K, then select the K highest scores of every token.  The paper does
+         * not say how a fractional average becomes K: here it is rounded half up and kept
+         * within [1, E]. */
+        int64_t total = 0;
+        for (int64_t t = 0; t < T; ++t)
+            for (int64_t e = 0; e < E; ++e) {
+                const float *s = scores + t * E;
+                if (eps_normalized) {
+                    volatile float v = s[e] * (float)E;
+                    total += v > eps;
+                } else {
+                    total += s[e] > eps;
+                }
+            }
+        int64_t k = T > 0 ? (2 * total + T) / (2 * T) : 1; /* floor(total / T + 1/2) */
+        if (k < 1) k = 1;
+        if (k > E) k = E;
+        oracle_select(scores, T, E, 1, eps, eps_normalized, (int)k, min_k, mask, k_t);
+        return;
+    }
     for (int64_t t = 0; t < T; ++t) {
         const float *s = scores + t * E;
         uint64_t m = 0;

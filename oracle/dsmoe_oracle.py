@@ -18,11 +18,11 @@ _SRC = os.path.join(_HERE, "dsmoe_oracle.c")
 _LIB = os.path.join(_HERE, "libdsmoe_oracle.so")
 _lib = None
 
-MODE_THRESHOLD, MODE_TOPK, MODE_ALL = 0, 1, 2
+MODE_THRESHOLD, MODE_TOPK, MODE_ALL, MODE_THRESHOLD_TOPK = 0, 1, 2, 3
 
 __all__ = [
     "build", "router_scores", "select", "group", "layer", "expert_rows", "combine",
-    "num_threads", "MODE_THRESHOLD", "MODE_TOPK", "MODE_ALL",
+    "num_threads", "MODE_THRESHOLD", "MODE_TOPK", "MODE_ALL", "MODE_THRESHOLD_TOPK",
 ]
 
 

@@ -358,3 +358,67 @@ def test_stage_functions_agree_with_independent_numpy():
         ref[g["row_token"][r]] += float(g["row_gate"][r]) * yp[r].astype(np.float32).astype(np.float64)
     np.testing.assert_allclose(out, ref, rtol=1e-12, atol=1e-18)
     np.testing.assert_allclose(oracle.layer(xb, W1b, W2b, S, mask), out, rtol=1e-5, atol=1e-7)
+
+
+# ---------------------------------------------------------------- Threshold-TopK ("Expert Sampling Strategy" paragraph)
+
+def _bits(*experts):
+    m = 0
+    for e in experts:
+        m |= 1 << e
+    return m
+
+
+def test_threshold_topk_worked_example_typed_by_hand():
+    # 4 tokens x 4 experts.  Raw threshold 0.2 activates 4, 1, 2 and 2 experts: 9 in all, 2.25 per token on
+    # average, so K = 2 and every token keeps its two highest scores (ties go to the lower index).
+    S = np.array([[0.30, 0.25, 0.24, 0.21],
+                  [0.70, 0.10, 0.10, 0.10],
+                  [0.40, 0.40, 0.10, 0.10],
+                  [0.15, 0.35, 0.15, 0.35]], dtype=np.float32)
+    thr_mask, thr_k = oracle.select(S, oracle.MODE_THRESHOLD, eps=0.2)
+    assert list(thr_k) == [4, 1, 2, 2]
+    mask, k_t = oracle.select(S, oracle.MODE_THRESHOLD_TOPK, eps=0.2)
+    assert list(k_t) == [2, 2, 2, 2]
+    assert [int(m) for m in mask] == [_bits(0, 1), _bits(0, 1), _bits(0, 1), _bits(1, 3)]
+
+
+def test_threshold_topk_rounds_the_average_half_up_and_stays_within_1_and_E():
+    # counts (1, 2): average 1.5 -> K = 2;  counts (1, 1, 2): 4/3 -> K = 1
+    S2 = np.array([[0.7, 0.2, 0.1], [0.45, 0.45, 0.10]], dtype=np.float32)
+    _, k = oracle.select(S2, oracle.MODE_THRESHOLD_TOPK, eps=0.3)
+    assert list(k) == [2, 2]
+    S3 = np.array([[0.7, 0.2, 0.1], [0.6, 0.25, 0.15], [0.45, 0.45, 0.10]], dtype=np.float32)
+    m, k = oracle.select(S3, oracle.MODE_THRESHOLD_TOPK, eps=0.3)
+    assert list(k) == [1, 1, 1] and [int(v) for v in m] == [1, 1, 1]      # expert 0 everywhere (tie -> lower index)
+    # nothing passes the threshold: K is kept at 1 (top-1); everything passes: K = E (select-all)
+    S = gi_scores(T=11, E=6)
+    m1, k1 = oracle.select(S, oracle.MODE_THRESHOLD_TOPK, eps=2.0)
+    mt, kt = oracle.select(S, oracle.MODE_TOPK, K=1)
+    assert np.array_equal(m1, mt) and np.all(k1 == 1)
+    ma, ka = oracle.select(S, oracle.MODE_THRESHOLD_TOPK, eps=0.0)
+    assert np.all(ma == np.uint64(2 ** 6 - 1)) and np.all(ka == 6)
+
+
+def gi_scores(T, E, seed_layer=0):
+    s = gi.LayerSpec("tt", T=T, d=64, H=64, E=E, dtype="bf16", router_gain=4.0)
+    x, (Wr, br) = gi.tokens(s), gi.router(s)
+    return oracle.router_scores(x, Wr, br)
+
+
+@pytest.mark.parametrize("normalized", [0, 1])
+def test_threshold_topk_K_is_the_rounded_mean_of_the_threshold_counts(normalized):
+    S = gi_scores(T=57, E=16)
+    for eps in (0.02, 0.05, 0.1, 0.3):
+        eps_use = eps * 16 if normalized else eps
+        v = (S * np.float32(16)) if normalized else S
+        counts = (v > np.float32(eps_use)).sum(axis=1)              # independent numpy thresholding
+        K = int(min(16, max(1, math.floor(counts.sum() / 57 + 0.5))))
+        mask, k_t = oracle.select(S, oracle.MODE_THRESHOLD_TOPK, eps=eps_use, eps_normalized=normalized)
+        assert np.all(k_t == K)
+        order = np.argsort(-S, axis=1, kind="stable")[:, :K]          # K highest, ties to the lower index
+        want = np.zeros(57, dtype=np.uint64)
+        for t in range(57):
+            for e in order[t]:
+                want[t] |= np.uint64(1) << np.uint64(e)
+        assert np.array_equal(mask, want)
