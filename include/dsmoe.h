@@ -57,7 +57,13 @@ typedef enum { DSMOE_F32 = 0, DSMOE_BF16 = 1 } dsmoe_dtype;
 typedef enum {
     DSMOE_SELECT_THRESHOLD = 0,  /* expert e active iff score exceeds eps                  */
     DSMOE_SELECT_TOPK = 1,       /* the K highest scores; ties go to the lower index       */
-    DSMOE_SELECT_ALL = 2         /* every expert: the dense-training forward               */
+    DSMOE_SELECT_ALL = 2,        /* every expert: the dense-training forward               */
+    /* "Expert Sampling Strategy" paragraph, Threshold-TopK: the threshold rule gives each token a count of
+     * active experts; the average count over the T tokens of the call, rounded half up and kept within
+     * [1, E] (the paper leaves the rounding open), is the K of a top-K selection applied to every token.
+     * eps and eps_normalized as for DSMOE_SELECT_THRESHOLD; K is ignored.  dsmoe_select_static does not
+     * offer this mode (DSMOE_ERR_UNSUPPORTED). */
+    DSMOE_SELECT_THRESHOLD_TOPK = 3
 } dsmoe_mode;
 
 typedef struct {

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdsmoe.so")
 
 F32, BF16 = 0, 1
-SELECT_THRESHOLD, SELECT_TOPK, SELECT_ALL = 0, 1, 2
+SELECT_THRESHOLD, SELECT_TOPK, SELECT_ALL, SELECT_THRESHOLD_TOPK = 0, 1, 2, 3
 
 EXPORTS = (
     "dsmoe_status_string", "dsmoe_workspace_size", "dsmoe_router", "dsmoe_select", "dsmoe_permute",

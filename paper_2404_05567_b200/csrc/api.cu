@@ -8,13 +8,15 @@ dsmoe_status check_desc(const dsmoe_layer_desc* p) {
     if (!p) return DSMOE_ERR_INVALID_ARG;
     if (p->T < 0 || p->d <= 0 || p->H <= 0 || p->E <= 0) return DSMOE_ERR_INVALID_ARG;
     if (p->dtype != DSMOE_F32 && p->dtype != DSMOE_BF16) return DSMOE_ERR_INVALID_ARG;
-    if (p->mode != DSMOE_SELECT_THRESHOLD && p->mode != DSMOE_SELECT_TOPK && p->mode != DSMOE_SELECT_ALL)
+    if (p->mode != DSMOE_SELECT_THRESHOLD && p->mode != DSMOE_SELECT_TOPK && p->mode != DSMOE_SELECT_ALL &&
+        p->mode != DSMOE_SELECT_THRESHOLD_TOPK)
         return DSMOE_ERR_INVALID_ARG;
     if (p->mode == DSMOE_SELECT_TOPK && p->K < 1) return DSMOE_ERR_INVALID_ARG;
     if (p->min_k != 0 && p->min_k != 1) return DSMOE_ERR_INVALID_ARG;
     if (p->eps_normalized != 0 && p->eps_normalized != 1) return DSMOE_ERR_INVALID_ARG;
     if (p->out_fp32 != 0 && p->out_fp32 != 1) return DSMOE_ERR_INVALID_ARG;
-    if (p->mode == DSMOE_SELECT_THRESHOLD && !(p->eps == p->eps)) return DSMOE_ERR_INVALID_ARG;   // NaN
+    if ((p->mode == DSMOE_SELECT_THRESHOLD || p->mode == DSMOE_SELECT_THRESHOLD_TOPK) && !(p->eps == p->eps))
+        return DSMOE_ERR_INVALID_ARG;   // NaN
     if ((p->d & 7) || (p->H & 7)) return DSMOE_ERR_INVALID_ARG;
     if (p->E > kMaxExperts) return DSMOE_ERR_UNSUPPORTED;
     // every per-assignment index is an int32
@@ -52,6 +54,7 @@ WsLayout ws_layout(const dsmoe_layer_desc& p) {
     L.partial = take(p.T <= kSmallMaxT ? (size_t)kSmallMaxCtas * 2 * T * 256 * 4 : 0);
     L.sync = take(64);                   // grid-barrier counters of the small-T kernel
     L.router = take(router_umma_supported(p) ? router_umma_scratch(p) : 0);   // tensor-core router: split Wr, partial logits
+    L.batch_k = take(256);               // Threshold-TopK: the batch's K
     L.total = off;
     return L;
 }
@@ -95,7 +98,7 @@ dsmoe_status dsmoe_select(const dsmoe_layer_desc* desc, const float* scores, uin
     if (!workspace || ws_bytes < L.total) return DSMOE_ERR_WORKSPACE;
     char* ws = static_cast<char*>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
-    DSMOE_TRY(launch_select(*desc, scores, mask, k_t, s));
+    DSMOE_TRY(launch_select(*desc, scores, mask, k_t, s, reinterpret_cast<int*>(ws + L.batch_k)));
     return launch_finalize(*desc, mask, counts, offsets, reinterpret_cast<int32_t*>(ws + L.chunk_prefix), nullptr, s);
 }
 
@@ -190,10 +193,16 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     if (fast && small_supported(p))
         return launch_layer_small(p, x, Wr, br, packed, scores, mask, k_t, counts_out, out, ws, L, dev_status, s);
 
+    // Threshold-TopK needs the whole batch's threshold counts before any token can be selected: the router runs
+    // with the threshold rule, then the selection is redone with the batch's K
+    dsmoe_layer_desc pr = p;
+    if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK) pr.mode = DSMOE_SELECT_THRESHOLD;
     if (fast && router_umma_supported(p))
-        DSMOE_TRY(launch_router_umma(p, x, Wr, br, scores, mask, k_t, ws + L.router, dev_status, s));
+        DSMOE_TRY(launch_router_umma(pr, x, Wr, br, scores, mask, k_t, ws + L.router, dev_status, s));
     else
-        DSMOE_TRY(launch_router(p, x, Wr, br, scores, mask, k_t, s));
+        DSMOE_TRY(launch_router(pr, x, Wr, br, scores, mask, k_t, s));
+    if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK)
+        DSMOE_TRY(launch_select(p, scores, mask, k_t, s, reinterpret_cast<int*>(ws + L.batch_k)));
     if (fast) {
         bool done = false;
         DSMOE_TRY(launch_layer_umma(p, x, packed, scores, mask, k_t, counts_out, out, ws, L, dev_status, s, &done));

@@ -43,15 +43,16 @@ static inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; 
 // Byte offsets of every internal buffer inside the caller's workspace.
 struct WsLayout {
     size_t scores, mask, k_t, counts, offsets, chunk_prefix, row_token, row_gate, token_rows;
-    size_t xp, h, yp, partial, sync, router, total;
+    size_t xp, h, yp, partial, sync, router, batch_k, total;
 };
 WsLayout ws_layout(const dsmoe_layer_desc& p);
 
 // ---- router.cu
 dsmoe_status launch_router(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
                            float* scores, uint64_t* mask, int32_t* k_t, cudaStream_t s);
+// k_scratch: one int of device memory, needed by DSMOE_SELECT_THRESHOLD_TOPK only (the batch's K)
 dsmoe_status launch_select(const dsmoe_layer_desc& p, const float* scores, uint64_t* mask, int32_t* k_t,
-                           cudaStream_t s);
+                           cudaStream_t s, int* k_scratch = nullptr);
 dsmoe_status launch_finalize(const dsmoe_layer_desc& p, const uint64_t* mask, int32_t* counts,
                              int32_t* offsets, int32_t* chunk_prefix, int32_t* counts_out, cudaStream_t s);
 

@@ -1544,7 +1544,7 @@ dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const 
     const int tiles = ceil_div(p.T, BM);
     DSMOE_TRY(launch_gemm(mA, mB, g, tiles < sm_count() ? tiles : sm_count(), s, false));
     router_finish_kernel<<<ceil_div(p.T, 8), 256, 0, s>>>(sums, br, scores, mask, k_t, p.T, EP,
-                                                         SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k});
+                                                         SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k, nullptr});
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
 }
@@ -1616,6 +1616,7 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
 bool small_supported(const dsmoe_layer_desc& p) {
     const int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
     if (!(umma_supported(p) && p.T >= 1 && p.T <= kSmallMaxT && p.T <= G && ceil_div(p.d, 64) <= G)) return false;
+    if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK) return false;   // its K needs a pass over the batch first: grouped path
     // the router's second half fetches all slice sums of a warp's tokens in one batch of 16 (small_router_pass)
     int KS = 1;
     while (KS < 16 && KS * 2 * p.T <= G) KS *= 2;
@@ -1671,7 +1672,7 @@ dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const 
     P.x = static_cast<const __nv_bfloat16*>(x);
     P.Wr = Wr;
     P.br = br;
-    P.sel = SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k};
+    P.sel = SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k, nullptr};
     P.scores = scores;
     P.mask = mask;
     P.k_t = k_t;

@@ -11,7 +11,7 @@
 namespace dsmoe {
 
 static SelParams sel_params(const dsmoe_layer_desc& p) {
-    return SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k};
+    return SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k, nullptr};
 }
 
 // Small T (decode): one block per token, the reduction over d split across all 256 threads.
@@ -363,10 +363,42 @@ dsmoe_status launch_router(const dsmoe_layer_desc& p, const void* x, const float
     return launch_router_t(p, static_cast<const float*>(x), Wr, br, scores, mask, k_t, s);
 }
 
+// Threshold-TopK ("Expert Sampling Strategy" paragraph): K = the batch average of the per-token counts that the
+// threshold gave, rounded half up and kept within [1, E].  One block; integer sums, so the result does not depend
+// on the order of the additions.
+__global__ void __launch_bounds__(1024) batch_k_kernel(const int32_t* __restrict__ k_t, int T, int E, int* __restrict__ K_out) {
+    __shared__ long long part[32];
+    long long sum = 0;
+    for (int t = threadIdx.x; t < T; t += 1024) sum += k_t[t];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long total = 0;
+        for (int w = 0; w < 32; ++w) total += part[w];
+        long long k = (2 * total + T) / (2ll * T);
+        *K_out = (int)(k < 1 ? 1 : (k > E ? E : k));
+    }
+}
+
 dsmoe_status launch_select(const dsmoe_layer_desc& p, const float* scores, uint64_t* mask, int32_t* k_t,
-                           cudaStream_t s) {
+                           cudaStream_t s, int* k_scratch) {
     if (p.T == 0) return DSMOE_OK;
-    select_kernel<<<ceil_div(p.T, 8), 256, 0, s>>>(scores, mask, k_t, p.T, sel_params(p));
+    SelParams q = sel_params(p);
+    if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK) {
+        if (!k_scratch) return DSMOE_ERR_UNSUPPORTED;
+        q.mode = DSMOE_SELECT_THRESHOLD;
+        q.min_k = 0;                     // the counts are the threshold's own
+        select_kernel<<<ceil_div(p.T, 8), 256, 0, s>>>(scores, mask, k_t, p.T, q);
+        DSMOE_CUDA_TRY(cudaGetLastError());
+        batch_k_kernel<<<1, 1024, 0, s>>>(k_t, p.T, p.E, k_scratch);
+        DSMOE_CUDA_TRY(cudaGetLastError());
+        q.mode = DSMOE_SELECT_TOPK;
+        q.min_k = p.min_k;
+        q.K_dev = k_scratch;
+    }
+    select_kernel<<<ceil_div(p.T, 8), 256, 0, s>>>(scores, mask, k_t, p.T, q);
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
 }

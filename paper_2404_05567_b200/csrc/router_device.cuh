@@ -11,6 +11,7 @@ struct SelParams {
     int E, mode;
     float eps;
     int eps_normalized, K, min_k;
+    const int* K_dev;    // when set, the K of the top-K rule is read from here (Threshold-TopK: K comes from the batch)
 };
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -40,14 +41,15 @@ __device__ __forceinline__ uint64_t select_warp(float s_lo, float s_hi, const Se
         sel_hi = v_hi && a_hi > q.eps;
     } else if (q.mode == DSMOE_SELECT_TOPK) {
         // rank = number of experts that beat this one (higher score, or equal score and lower index)
+        const int K = q.K_dev ? *q.K_dev : q.K;
         int better_lo = 0, better_hi = 0;
         for (int j = 0; j < q.E; ++j) {
             const float o = j < 32 ? __shfl_sync(0xffffffffu, s_lo, j) : __shfl_sync(0xffffffffu, s_hi, j - 32);
             better_lo += (o > s_lo) || (o == s_lo && j < lane);
             better_hi += (o > s_hi) || (o == s_hi && j < lane + 32);
         }
-        sel_lo = v_lo && better_lo < q.K;
-        sel_hi = v_hi && better_hi < q.K;
+        sel_lo = v_lo && better_lo < K;
+        sel_hi = v_hi && better_hi < K;
     } else {
         sel_lo = v_lo;
         sel_hi = v_hi;

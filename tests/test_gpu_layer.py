@@ -151,3 +151,26 @@ def test_decode_path_when_some_experts_are_unselected(case):
         assert r["A"] == 0 and np.all(np_f32(r["layer"].out) == 0.0)
     if case["mode"] == gi.MODE_TOPK and case["K"] == 1:
         assert r["empty_experts"] >= (8 if case["E"] == 32 else 1)
+
+
+# ---------------------------------------------------------------- Threshold-TopK ("Expert Sampling Strategy" paragraph)
+
+@pytest.mark.parametrize("case", [
+    dict(T=40, d=128, H=128, E=8, eps=0.06),                  # few tokens: not the one-launch decode kernel (K needs the batch)
+    dict(T=300, d=128, H=64, E=16, eps=0.03),
+    dict(T=1000, d=256, H=128, E=32, eps=0.7, eps_normalized=1, zipf_s=1.1),
+    dict(T=513, d=64, H=72, E=5, eps=0.16),                   # plain fp32-FMA path (H % 64 != 0)
+], ids=["t40", "t300", "t1000_skew", "plain"])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_threshold_topk_layer(case, dtype):
+    s = gi.LayerSpec("tt_" + str(case["T"]), dtype=dtype, mode=gi.MODE_THRESHOLD_TOPK, router_gain=4.0, **case)
+    r = layer_parity(s)
+    k = np_popcounts(r["layer"].mask, s.T)
+    assert len(set(k.tolist())) == 1 and 1 <= int(k[0]) <= s.E        # every token got the same K
+    assert r["A"] == s.T * int(k[0])
+    assert r["err_rows"] <= (TOL_BF16 if dtype == "bf16" else TOL_F32), (r["err_rows"], r["err"])
+
+
+def np_popcounts(mask_t, T):
+    m = mask_t.cpu().numpy()[:T].view(np.uint64)
+    return np.array([bin(int(v)).count("1") for v in m])

@@ -44,6 +44,9 @@ MODES = [
     dict(mode=gi.MODE_TOPK, K=5),
     dict(mode=gi.MODE_TOPK, K=100),
     dict(mode=gi.MODE_ALL),
+    dict(mode=gi.MODE_THRESHOLD_TOPK, eps=0.02),                          # Threshold-TopK: K from the batch
+    dict(mode=gi.MODE_THRESHOLD_TOPK, eps=0.9, eps_normalized=1),
+    dict(mode=gi.MODE_THRESHOLD_TOPK, eps=2.0),                           # nothing passes: K = 1
 ]
 
 
