@@ -121,6 +121,7 @@ struct Shared {
     volatile int up_geo;                   // which of the two the up-projection follows (the down-projection: always geo[1])
     volatile int geo_state;
     volatile int spec_issued, spec_stop;   // producer -> MMA issuer: ring slots filled under geo[0]; no more will be
+    volatile int up_arrived;               // epilogue -> producer: this CTA has arrived at the barrier between the projections
     volatile int mma_drained;              // MMA issuer -> producer: those slots are consumed, the ring is idle
     float gate_s[BM], gate2_s[BM];
     uint64_t mask_s[BM];                   // small_layer_kernel: every token's selection word
@@ -762,6 +763,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         sh.spec_issued = 0;
         sh.spec_stop = 0;
         sh.mma_drained = 0;
+        sh.up_arrived = 0;
         small_geometry(P, P.E, G, sh.geo[0]);
 #ifdef DSMOE_TRACE
         for (int i = 0; i < 32; ++i) sh.trace[i] = 0;
@@ -901,7 +903,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             // into L2 meanwhile: the down-projection then finds them there instead of in DRAM.  All CTAs together
             // ask for well under half of L2.  (Not for the fewest tokens: there the gap is short and the requests only
             // compete with the ring's own.)
-            if (alive && have && P.spec) {
+            if (alive && have && P.spec && wait_flag(&sh.up_arrived, sh)) {     // ... once this CTA's own hg is out
                 SmallIter pit = it;
                 SmallTile pt = t;
                 int pi = i_cur;
@@ -1216,6 +1218,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 EPI_SYNC();
                 if (etid == 0) {
                     grid_arrive(P.sync, 1);
+                    sh.up_arrived = 1;
                     TRACE(7);
                 }
                 up_done = true;
