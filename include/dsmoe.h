@@ -165,9 +165,10 @@ dsmoe_status dsmoe_combine(const dsmoe_layer_desc* desc, const void* yp, const f
                            dsmoe_stream stream);
 
 /*
- * Kernel-preferred copy of the (static, post-training) expert weights: W1 transposed to
- * [E,H,d] followed by W2 transposed to [E,d,H], both bf16, so that every tensor-core
- * operand is contiguous along the reduction.  dtype must be DSMOE_BF16.
+ * Kernel-preferred copy of the (static, post-training) expert weights, bf16: W1 as
+ * [E][d/64][H][64] followed by W2 as [E][H/64][d][64] (block-major along the reduction), so
+ * that every tensor-core operand is contiguous along the reduction and every tile a kernel
+ * fetches is one contiguous piece of memory.  dtype must be DSMOE_BF16; d and H multiples of 64.
  * dsmoe_packed_size reports the bytes `packed` must hold.
  */
 dsmoe_status dsmoe_packed_size(const dsmoe_layer_desc* desc, size_t* bytes);

@@ -158,6 +158,7 @@ dsmoe_status dsmoe_pack_weights(const dsmoe_layer_desc* desc, const void* W1, co
                                 dsmoe_stream stream) {
     DSMOE_TRY(check_desc(desc));
     if (desc->dtype != DSMOE_BF16 || !W1 || !W2 || !packed || !aligned16(packed)) return DSMOE_ERR_INVALID_ARG;
+    if ((desc->d % 64) || (desc->H % 64)) return DSMOE_ERR_UNSUPPORTED;   // the packed layout is in blocks of 64
     return launch_pack(*desc, W1, W2, packed, (cudaStream_t)stream);
 }
 

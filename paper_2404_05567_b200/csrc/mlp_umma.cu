@@ -141,14 +141,19 @@ __device__ unsigned long long g_trace[192][32];
 
 __device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f)); }
 
-// Weight rows [n0, n0 + rows) of expert e, reduction block starting at k: power-of-two boxes, largest first.
-__device__ __forceinline__ void load_weight_rows(const BMaps* maps, uint32_t dst, uint32_t bar, int k, int n0, int rows,
+// The packed weights are block-major along the reduction: [E][k / 64][n][64], so the tile (64 k, rows n0..) of
+// reduction block kb is the `rows` consecutive 128-byte rows starting at wrow(kb, n0, N) of a [E][(K/64)*N][64]
+// tensor: one contiguous piece of memory.
+__device__ __forceinline__ int wrow(int kb, int n0, int N) { return kb * N + n0; }
+
+// Weight rows [row0, row0 + rows) of expert e (see wrow): power-of-two boxes, largest first.
+__device__ __forceinline__ void load_weight_rows(const BMaps* maps, uint32_t dst, uint32_t bar, int row0, int rows,
                                                  int e) {
     int done = 0;
 #pragma unroll
     for (int lvl = 4; lvl >= 0; --lvl) {
         if ((rows - done) >= (16 << lvl)) {
-            ptx::tma_load_3d(dst + done * (BK * 2), &maps->m[lvl], bar, k, n0 + done, e);
+            ptx::tma_load_3d(dst + done * (BK * 2), &maps->m[lvl], bar, 0, row0 + done, e);
             done += 16 << lvl;
         }
     }
@@ -284,8 +289,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (!P.gather) ptx::tma_load_2d(smA + s * A_STAGE_BYTES, &tmA, bar, a_col, t.row0);
                     // full-width tiles take the one 256-row copy directly (measurably faster than walking the
                     // box sizes); only a ragged last column tile needs the decomposition
-                    if (t.bn == BN) ptx::tma_load_3d(smB + s * B_STAGE_BYTES, &tmB.m[4], bar, b_k, t.n0, b_e);
-                    else load_weight_rows(&tmB, smB + s * B_STAGE_BYTES, bar, b_k, t.n0, t.bn, b_e);
+                    const int b_row = wrow(b_k / BK, t.n0, P.n_per_expert);
+                    if (t.bn == BN) ptx::tma_load_3d(smB + s * B_STAGE_BYTES, &tmB.m[4], bar, 0, b_row, b_e);
+                    else load_weight_rows(&tmB, smB + s * B_STAGE_BYTES, bar, b_row, t.bn, b_e);
                     if (++s == STAGES) {
                         s = 0;
                         ph ^= 1u;
@@ -615,9 +621,9 @@ __device__ __forceinline__ void small_issue(const SmallParams& P, const CUtensor
     if (t.phase == 0) {
         if (what & 1) ptx::tma_load_2d(slotA, tmX, bar, i * BK, 0);
         if (what & 2) {
-            ptx::tma_load_3d_hint(slotB, &tmW1->m[t.bn1 / 16 - 1], bar, i * BK, t.n0, t.e, wpol);
+            ptx::tma_load_3d_hint(slotB, &tmW1->m[t.bn1 / 16 - 1], bar, 0, wrow(i, t.n0, P.H), t.e, wpol);
             if (t.bn > t.bn1)
-                ptx::tma_load_3d_hint(slotB + t.bn1 * (BK * 2), &tmW1->m[(t.bn - t.bn1) / 16 - 1], bar, i * BK, 0, t.e2, wpol);
+                ptx::tma_load_3d_hint(slotB + t.bn1 * (BK * 2), &tmW1->m[(t.bn - t.bn1) / 16 - 1], bar, 0, wrow(i, 0, P.H), t.e2, wpol);
         }
     } else {
         const int kbpe = P.H / BK;
@@ -626,8 +632,8 @@ __device__ __forceinline__ void small_issue(const SmallParams& P, const CUtensor
         if (what & 1) ptx::tma_load_2d(slotA, tmHg, bar, e * P.H + kb * BK, 0);
         if (what & 2) {
             // column ranges are 64, 128 or 256 wide: one copy; only a ragged last range needs the decomposition
-            if ((t.bn & (t.bn - 1)) == 0) ptx::tma_load_3d_hint(slotB, &tmW2->m[__ffs(t.bn) - 5], bar, kb * BK, t.n0, e, wpol);
-            else load_weight_rows(tmW2, slotB, bar, kb * BK, t.n0, t.bn, e);
+            if ((t.bn & (t.bn - 1)) == 0) ptx::tma_load_3d_hint(slotB, &tmW2->m[__ffs(t.bn) - 5], bar, 0, wrow(kb, t.n0, P.d), e, wpol);
+            else load_weight_rows(tmW2, slotB, bar, wrow(kb, t.n0, P.d), t.bn, e);
         }
     }
 }
@@ -912,7 +918,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 for (int bytes = 0; phave && bytes < kSmallL2PrefetchBytes;) {
                     if ((pt.bn & (pt.bn - 1)) == 0) {
                         const int gb = pt.kstart + pi;
-                        ptx::tma_prefetch_3d(&tmW2.m[__ffs(pt.bn) - 5], (gb % kbpe) * BK, pt.n0, g->active[gb / kbpe]);
+                        ptx::tma_prefetch_3d(&tmW2.m[__ffs(pt.bn) - 5], 0, wrow(gb % kbpe, pt.n0, P.d), g->active[gb / kbpe]);
                     }
                     bytes += pt.bn * BK * 2;
                     if (++pi == pt.nk) {
@@ -1424,12 +1430,13 @@ dsmoe_status make_map_2d(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_
     return r == CUDA_SUCCESS ? DSMOE_OK : DSMOE_ERR_CUDA;
 }
 
-// bf16 [E, n, k] row-major, box {64 k, box_n, 1}, 128-byte swizzle
+// packed weights of E experts, n output columns, reduction length k: bf16 [E][k / 64][n][64], seen as
+// [E][(k / 64) * n][64]; box {64, box_n, 1}, 128-byte swizzle
 dsmoe_status make_map_3d(CUtensorMap* m, const void* ptr, uint64_t E, uint64_t n, uint64_t k, uint32_t box_n) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return DSMOE_ERR_CUDA;
-    const cuuint64_t dims[3] = {k, n, E};
-    const cuuint64_t strides[2] = {k * 2, n * k * 2};
+    const cuuint64_t dims[3] = {BK, (k / BK) * n, E};
+    const cuuint64_t strides[2] = {BK * 2, n * k * 2};
     const cuuint32_t box[3] = {BK, box_n, 1};
     const cuuint32_t es[3] = {1, 1, 1};
     const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
@@ -1487,7 +1494,7 @@ dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams&
 // Wr (fp32) is written as the exact sum of three bf16 terms, w = w1 + w2 + w3 (w1 = bf16(w), w2 = bf16(w - w1),
 // w3 = bf16(w - w1 - w2): 3 x 8 significant bits cover fp32's 24).  x is bf16, so every product x.w_i is exact in
 // fp32 and the three sums accumulate in fp32: the logits are as accurate as an fp32 dot product, at tensor-core
-// speed.  The three terms sit side by side along N: B = [3 * EP, d] bf16, K-major, EP = E rounded up to 32 or 64.
+// speed.  The three terms sit side by side along N: B = [3 * EP, d] bf16 in the packed weights' layout, EP = E rounded up to 32 or 64.
 __global__ void __launch_bounds__(256) router_split_kernel(const float* __restrict__ Wr, __nv_bfloat16* __restrict__ out,
                                                            int d, int E, int EP) {
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
@@ -1498,9 +1505,11 @@ __global__ void __launch_bounds__(256) router_split_kernel(const float* __restri
     const float r1 = w - __bfloat162float(w1);
     const __nv_bfloat16 w2 = __float2bfloat16_rn(r1);
     const float r2 = r1 - __bfloat162float(w2);
-    out[idx] = w1;
-    out[idx + (long long)EP * d] = w2;
-    out[idx + 2ll * EP * d] = __float2bfloat16_rn(r2);
+    // block-major like the packed expert weights: [k / 64][3 * EP][64], term g in rows g * EP .. of every block
+    const long long o = ((long long)(k / BK) * (3 * EP) + e) * BK + k % BK;
+    out[o] = w1;
+    out[o + (long long)EP * BK] = w2;
+    out[o + 2ll * EP * BK] = __float2bfloat16_rn(r2);
 }
 
 // logits = (s1 + s2) + s3 + bias per expert, then softmax and selection: one warp per token

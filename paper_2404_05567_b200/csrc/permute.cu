@@ -139,7 +139,8 @@ __global__ void __launch_bounds__(128) combine_f32_kernel(const float4* __restri
     }
 }
 
-// dst[b][c][r] = src[b][r][c] for a batch of [rows, cols] bf16 matrices (32x32 tiles through smem).
+// Packing of a batch of [rows = reduction, cols = outputs] bf16 matrices: dst[b][r / 64][c][r % 64] = src[b][r][c]
+// (32x32 tiles through smem; rows is a multiple of 64 where this layout is used).
 __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src,
                                                              __nv_bfloat16* __restrict__ dst, int rows, int cols) {
     __shared__ __nv_bfloat16 tile[32][33];
@@ -153,7 +154,7 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
     __syncthreads();
     for (int i = ty; i < 32; i += 8) {
         const int c = c0 + i, r = r0 + tx;
-        if (r < rows && c < cols) dst[base + (size_t)c * rows + r] = tile[tx][i];
+        if (r < rows && c < cols) dst[base + ((size_t)(r / 64) * cols + c) * 64 + (r % 64)] = tile[tx][i];
     }
 }
 
@@ -201,7 +202,7 @@ dsmoe_status launch_pack(const dsmoe_layer_desc& p, const void* W1, const void* 
     const __nv_bfloat16* w2 = static_cast<const __nv_bfloat16*>(W2);
     __nv_bfloat16* w1t = static_cast<__nv_bfloat16*>(packed);
     __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
-    // W1[e]: [d,H] -> [H,d];  W2[e]: [H,d] -> [d,H]
+    // W1[e]: [d,H] -> [d/64][H][64];  W2[e]: [H,d] -> [H/64][d][64]
     transpose_bf16_kernel<<<dim3(ceil_div(p.H, 32), ceil_div(p.d, 32), p.E), 256, 0, s>>>(w1, w1t, p.d, p.H);
     DSMOE_CUDA_TRY(cudaGetLastError());
     transpose_bf16_kernel<<<dim3(ceil_div(p.d, 32), ceil_div(p.H, 32), p.E), 256, 0, s>>>(w2, w2t, p.H, p.d);

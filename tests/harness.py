@@ -57,7 +57,7 @@ class Layer:
         self.W1_d, self.W2_d = to_dev(self.W1), to_dev(self.W2)
         self.ws = torch.empty(dm.dsmoe_workspace_size(self.desc), dtype=torch.uint8, device="cuda")
         self.packed = None
-        if pack and s.dtype == "bf16":
+        if pack and s.dtype == "bf16" and s.d % 64 == 0 and s.H % 64 == 0:      # the packed layout is in blocks of 64
             self.packed = torch.empty(dm.dsmoe_packed_size(self.desc), dtype=torch.uint8, device="cuda")
             dm.dsmoe_pack_weights(self.desc, self.W1_d, self.W2_d, self.packed)
         self.dev_status = torch.zeros(1, dtype=torch.int32, device="cuda")
