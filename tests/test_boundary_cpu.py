@@ -72,3 +72,18 @@ def test_null_pointers_and_short_workspace_are_rejected_before_any_launch():
     assert L.dsmoe_packed_size(ctypes.byref(desc), ctypes.byref(ctypes.c_size_t(0))) == 1
     empty = dm.make_desc(0, 64, 64, 4, dm.F32)
     assert L.dsmoe_layer_forward(ctypes.byref(empty), z, z, z, z, z, z, z, z, z, z, ctypes.c_size_t(0), z, z) == 0
+
+
+def test_pack_rejects_shapes_that_are_not_multiples_of_64_and_the_new_selection_mode_is_accepted():
+    L = dm.lib()
+    fake = ctypes.c_void_p(4096)
+    z = ctypes.c_void_p(0)
+    odd = dm.make_desc(16, 128, 72, 4, dm.BF16)          # H = 72: the packed layout is in blocks of 64
+    assert L.dsmoe_pack_weights(ctypes.byref(odd), fake, fake, fake, z) == 2
+    # Threshold-TopK is a valid mode of the descriptor (sizes as for the threshold rule: up to E experts per token) ...
+    tt = dm.make_desc(128, 64, 64, 32, dm.BF16, mode=dm.SELECT_THRESHOLD_TOPK, eps=0.1)
+    thr = dm.make_desc(128, 64, 64, 32, dm.BF16, mode=dm.SELECT_THRESHOLD, eps=0.1)
+    assert dm.dsmoe_workspace_size(tt) >= dm.dsmoe_workspace_size(thr) - 4096 and dm.amax(tt) == 128 * 32
+    # ... a mode beyond it is not
+    bad = dm.make_desc(128, 64, 64, 32, dm.BF16, mode=4)
+    assert L.dsmoe_workspace_size(ctypes.byref(bad), ctypes.byref(ctypes.c_size_t(0))) == 1
