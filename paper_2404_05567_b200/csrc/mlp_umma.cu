@@ -659,7 +659,18 @@ __device__ __forceinline__ void small_geometry(const SmallParams& P, int n, int 
 // KS * (tokens per warp) <= 16 for every T this kernel takes, so a warp fetches all its slice sums in one batch
 // and waits for memory once.  One copy of this code serves both modes (not inlined): the second call finds its
 // instructions cached, which matters while the weight stream keeps the memory system busy.
-__device__ __noinline__ void small_router_pass(const SmallParams& P, Shared& sh, int KS, int w, int lane, int mode, int e,
+// What small_router_pass needs of the kernel's parameters, passed by value: a reference to the parameter block would
+// make every thread copy all of it into local memory for the call.
+struct RouterArgs {
+    int T, E;
+    const float* br;
+    const float* partial;
+    float* scores;
+    uint64_t* mask;
+    int32_t* k_t;
+    SelParams sel;
+};
+__device__ __noinline__ void small_router_pass(const RouterArgs P, Shared& sh, int KS, int w, int lane, int mode, int e,
                                                int e2) {
     constexpr int NW = kEpiThreads / 32;
     const bool v_lo = lane < P.E, v_hi = lane + 32 < P.E;
@@ -1177,7 +1188,8 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         }
         EPI_SYNC();
         // ---- router, step 2: softmax and selection of every token, in every CTA (see small_router_pass)
-        if (!sh.abort_flag) small_router_pass(P, sh, KS, warp - 2, lane, 0, 0, 0);
+        const RouterArgs RA{P.T, P.E, P.br, P.partial, P.scores, P.mask, P.k_t, P.sel};
+        if (!sh.abort_flag) small_router_pass(RA, sh, KS, warp - 2, lane, 0, 0, 0);
         EPI_SYNC();
         if (etid == 0) {
             unsigned long long m = sh.active_mask;
@@ -1232,7 +1244,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             if (!have) break;
             // router gate of every token for this tile's expert(s), recomputed from the slice sums (other CTAs' copies
             // of the scores are not visible yet) while the mainloop is still running
-            if (t.phase == 0 && !dead) small_router_pass(P, sh, KS, warp - 2, lane, 1, t.e, t.e2);
+            if (t.phase == 0 && !dead) small_router_pass(RA, sh, KS, warp - 2, lane, 1, t.e, t.e2);
             if (tmem_warp && !dead && !ptx::mbar_wait(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag)) dead = true;
             dead = __any_sync(0xffffffffu, dead);     // the TMEM reads below are warp-collective
 #ifdef DSMOE_TRACE
