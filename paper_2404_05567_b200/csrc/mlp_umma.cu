@@ -893,8 +893,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             TRACE(3);
             // down-projection: weight tiles first, for as many slots as the ring has; their hg tiles follow
             // once every CTA has finished writing hg
-            SmallTile pend_t[MAX_STAGES];
-            int pend_i[MAX_STAGES], pend_s[MAX_STAGES];
+            int pend_g[MAX_STAGES], pend_s[MAX_STAGES];      // reduction block and ring slot of each weight tile under way
             int npend = 0, i_cur = 0;
             while (alive && have && npend < n_stages) {
                 if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ((phb >> s) & 1u) ^ 1u, &sh.abort_flag)) {
@@ -904,8 +903,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 const uint32_t bar = ptx::smem_u32(&sh.full[s]);
                 ptx::mbar_expect_tx(bar, a_bytes + (uint32_t)t.bn * BK * 2);
                 small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, t, i_cur, smA + s * slot_bytes, smB + s * slot_bytes, bar, 2, wpol);
-                pend_t[npend] = t;
-                pend_i[npend] = i_cur;
+                pend_g[npend] = t.kstart + i_cur;
                 pend_s[npend] = s;
                 ++npend;
                 phb ^= 1u << s;
@@ -942,9 +940,11 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             if (alive && !grid_wait(P.sync, 1, G, &sh.abort_flag)) alive = false;
             TRACE(6);
             asm volatile("fence.proxy.async;" ::: "memory");   // hg was written through the generic proxy, TMA reads it
-            for (int j = 0; alive && j < npend; ++j)
-                small_issue(P, &tmX, &tmW1, &tmHg, &tmW2, g->active, pend_t[j], pend_i[j], smA + pend_s[j] * slot_bytes,
-                            smB + pend_s[j] * slot_bytes, ptx::smem_u32(&sh.full[pend_s[j]]), 1, wpol);
+            for (int j = 0; alive && j < npend; ++j) {
+                const int kbpe = P.H / BK, gb = pend_g[j];
+                ptx::tma_load_2d(smA + pend_s[j] * slot_bytes, &tmHg, ptx::smem_u32(&sh.full[pend_s[j]]),
+                                 g->active[gb / kbpe] * P.H + (gb % kbpe) * BK, 0);
+            }
             while (alive && have) {
                 for (; i_cur < t.nk; ++i_cur) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ((phb >> s) & 1u) ^ 1u, &sh.abort_flag)) {
