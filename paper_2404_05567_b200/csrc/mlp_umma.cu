@@ -1344,22 +1344,25 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             // a thread owns 4 consecutive columns of one token; its partial loads are issued in batches before
             // the additions, which run in ascending CTA order
             const int d4 = P.d / 4;
-            const long long n_out4 = (long long)P.T * d4;
-            const long long per_cta = (n_out4 + G - 1) / G;     // an equal share for every CTA
-            for (long long j = etid; j < per_cta; j += kEpiThreads) {
-                const long long idx = (long long)blockIdx.x * per_cta + j;
+            const int n_out4 = P.T * d4;                        // T <= 128 and d < 2^16: an int
+            const int per_cta = (n_out4 + G - 1) / G;           // an equal share for every CTA
+            for (int j = etid; j < per_cta; j += kEpiThreads) {
+                const int idx = (int)blockIdx.x * per_cta + j;
                 if (idx >= n_out4) break;
-                const int tt = (int)(idx / d4), col = (int)(idx % d4) * 4;
+                const int tt = idx / d4, col = (idx % d4) * 4;
                 const int r = col / bnd, cc = col % bnd;
                 float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (U > 0) {
                     const int i0 = (r * U) / per, i1 = ((r + 1) * U - 1) / per;
+                    // CTA i0 may have started in the range before (then range r is its second one); every later
+                    // contributor starts inside range r
+                    const int seg_first = i0 * per < r * U ? 1 : 0;
                     for (int ib = i0; ib <= i1; ib += kFixBatch) {
                         float4 v[kFixBatch];
 #pragma unroll
                         for (int j = 0; j < kFixBatch; ++j) {
                             const int i = ib + j;
-                            const int seg = r - (i * per) / U;
+                            const int seg = i == i0 ? seg_first : 0;
                             v[j] = i <= i1 ? __ldcg(reinterpret_cast<const float4*>(
                                                  P.partial + (((long long)i * 2 + seg) * P.T + tt) * BN + cc))
                                            : make_float4(0.f, 0.f, 0.f, 0.f);
