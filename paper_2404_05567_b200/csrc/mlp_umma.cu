@@ -1324,8 +1324,8 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             }
         }
         // ---- last grid barrier, then the fix-up: out[t,c] = sum of the partial tiles covering column c in
-        // ascending CTA order (the partition arithmetic mirrors SmallIter)
-        __threadfence();
+        // ascending CTA order (the partition arithmetic mirrors SmallIter).  The arriving thread's fence, after
+        // the CTA barrier, covers the other threads' partial-sum stores.
         EPI_SYNC();
         if (etid == 0) {
             TRACE(9);
