@@ -29,7 +29,7 @@ WORKLOADS = {
     "c2_t1": ("c2", dict(T=1)), "c2_t8": ("c2", dict(T=8)), "c2_t32": ("c2", dict(T=32)),
     "c3": ("c3", {}), "c4": ("c4", {}), "c5": ("c5", dict(eps=0.01)),
 }
-NCU_TRAFFIC_BYTES = {"c2_t32": 277.9e6, "c3": 1023.2e6}
+NCU_TRAFFIC_BYTES = {"c2_t32": 272.7e6, "c3": 1017.6e6}
 DEFAULT_STEPS = {"c2_t1": 1000, "c2_t8": 1000, "c2_t32": 1000, "c3": 100, "c4": 50, "c5": 50}
 METRIC = "moe_layer_tokens_per_s"
 
