@@ -469,16 +469,18 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // the experts that at least one token selected -- no grouping, no aggregation pass:
 //
 //   router   the reduction over d of every token cut into slices, one CTA each  -> grid barrier
-//            CTA t adds token t's slices: softmax, selection                    -> grid barrier
+//            every CTA adds every token's slices itself: softmax, selection (same arithmetic, same result
+//            everywhere, so no second barrier); runs on the epilogue warps, underneath the up-projection
 //   up       hg[t,(e,j)] = [e in sel(t)] S[t,e] GeLU(x[t].W1[e][:,j]); a CTA takes a contiguous run of
 //            16-row units of the selected experts' W1 (a tile may cross one expert boundary) -> grid barrier
 //   down     out = hg . W2cat as stream-K: units of (256 output columns, expert, 64-wide reduction
 //            block); fp32 partial tiles, at most two per CTA                    -> grid barrier
 //   fix-up   every CTA adds the partial tiles of its share of out[T,d] in ascending-CTA order
 //
-// The operand ring keeps running across the up/down barrier: the producer prefetches the first W2
-// tiles (which do not depend on hg) while other CTAs finish, and adds the hg tiles once the barrier
-// has passed.  Every wait, on an mbarrier or on a grid barrier, is bounded.
+// From 8 tokens on the up-projection starts before the router has finished, under "every expert selected"
+// (see the kernel).  The operand ring keeps running across the up/down barrier: the producer prefetches the
+// first W2 tiles (which do not depend on hg) while other CTAs finish, asks the next ones into L2, and adds
+// the hg tiles once the barrier has passed.  Every wait, on an mbarrier or on a grid barrier, is bounded.
 
 struct SmallParams {
     int T, d, H, E, t_pad;
@@ -803,7 +805,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     const uint32_t tmem_base = sh.tmem_base;
     const uint32_t smA = base;
 
-    // From here the three roles run side by side.  Warps 2.. compute the router (two grid barriers) and publish the
+    // From here the three roles run side by side.  Warps 2.. compute the router (one grid barrier) and publish the
     // geometry it implies in geo[1]; warps 0 and 1 either wait for that, or (P.spec) start streaming and multiplying
     // the up-projection at once under geo[0], "every expert selected" -- the products x.W1 do not depend on the
     // router, only the partition of the work does.  If the router confirms geo[0] they simply carry on; if not,
