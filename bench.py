@@ -28,9 +28,13 @@ import dsmoe_inputs as gi  # noqa: E402
 WORKLOADS = {
     "c2_t1": ("c2", dict(T=1)), "c2_t8": ("c2", dict(T=8)), "c2_t32": ("c2", dict(T=32)),
     "c3": ("c3", {}), "c4": ("c4", {}), "c5": ("c5", dict(eps=0.01)),
+    # the paper's own DS-MoE-6B layer shape (Table tab:model_arch: width 4096, 32 experts of width 512), not part
+    # of the default run: narrower experts than the benchmark configurations
+    "paper6b_t32": ("c2", dict(T=32, d=4096, H=512)), "paper6b_topk6": ("c3", dict(T=8192, d=4096, H=512, K=6)),
 }
 NCU_TRAFFIC_BYTES = {"c2_t32": 272.7e6, "c3": 1017.6e6}
-DEFAULT_STEPS = {"c2_t1": 1000, "c2_t8": 1000, "c2_t32": 1000, "c3": 100, "c4": 50, "c5": 50}
+DEFAULT_STEPS = {"c2_t1": 1000, "c2_t8": 1000, "c2_t32": 1000, "c3": 100, "c4": 50, "c5": 50, "paper6b_t32": 1000,
+                 "paper6b_topk6": 100}
 METRIC = "moe_layer_tokens_per_s"
 
 
