@@ -1,19 +1,24 @@
 """Benchmark of the DS-MoE layer forward on B200: MoE-layer tokens/s plus the roofline fraction of
 the dominant kernel, with the CPU oracle timed beside it.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2_t32|c2_t1|c2_t8|c3|c4|c5]
-                    [--impl ours|reference] [--no-extra]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference] [--no-extra]
 
 A step is one dsmoe_layer_forward over one batch of synthetic tokens.  The decode-shaped workloads
-cycle through several distinct sets of expert weights (> L2 in total) so that every step reads its
-weights from HBM, as consecutive layers of a real model do; the prefill-shaped and dense workloads
+cycle through many distinct sets of expert weights (far more than L2 in total) so that every step reads
+its weights from HBM, as consecutive layers of a real model do; the prefill-shaped and dense workloads
 touch far more than L2 per step by themselves.  One JSON line goes to stdout.
+
+--gpus N > 1 without a torchrun environment starts N ranks itself (one process per GPU); under
+torchrun the ranks are already there.  The layer shards by token with no exchange, so the ranks are
+replicas and the only collective is the reduction of the timing.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -25,17 +30,43 @@ import numpy as np  # noqa: E402
 
 import dsmoe_inputs as gi  # noqa: E402
 
+# name -> (recipe, overrides).  c1..c5 are the benchmark configurations; paper_* are the layer shapes of the paper's
+# own models (Table tab:model_arch: DS-MoE-1B/3B/6B; Table tab:scaled: DS-MoE-10B/14B/19B), 32 experts each, top-K as
+# the paper's speed tests use it (Table tab:latency: 6 for 3B, 4 for 6B; Table tab:scaled: 4).
+PAPER_SHAPES = {"1b": (2048, 256, 6), "3b": (3072, 384, 6), "6b": (4096, 512, 4),
+                "10b": (5120, 640, 4), "14b": (6144, 768, 4), "19b": (7168, 896, 4)}
 WORKLOADS = {
     "c2_t1": ("c2", dict(T=1)), "c2_t8": ("c2", dict(T=8)), "c2_t32": ("c2", dict(T=32)),
-    "c3": ("c3", {}), "c4": ("c4", {}), "c5": ("c5", dict(eps=0.01)),
-    # the paper's own DS-MoE-6B layer shape (Table tab:model_arch: width 4096, 32 experts of width 512), not part
-    # of the default run: narrower experts than the benchmark configurations
-    "paper6b_t32": ("c2", dict(T=32, d=4096, H=512)), "paper6b_topk6": ("c3", dict(T=8192, d=4096, H=512, K=6)),
+    "c3": ("c3", {}), "c4": ("c4", {}),
+    "c5": ("c5", dict(eps=0.01)),
+    # output-token throughput as the paper measures it ("GPU Inference Analysis"): a decode loop in which layer i's
+    # output is layer i+1's input, 24 distinct layers (Table tab:model_arch: N_layer = 24 .. 36); W2 is drawn 16 times
+    # larger so that the activations keep their scale from layer to layer without the model's normalisation layers
+    "decode_loop_t8": ("c2", dict(T=8, w2_gain=16.0)), "decode_loop_t32": ("c2", dict(T=32, w2_gain=16.0)),
 }
-NCU_TRAFFIC_BYTES = {"c2_t32": 272.7e6, "c3": 1017.6e6}
-DEFAULT_STEPS = {"c2_t1": 1000, "c2_t8": 1000, "c2_t32": 1000, "c3": 100, "c4": 50, "c5": 50, "paper6b_t32": 1000,
-                 "paper6b_topk6": 100}
+for _e in (0.0, 0.01, 0.05, 0.1, 0.2):
+    WORKLOADS[f"c5_eps{_e}"] = ("c5", dict(eps=_e))
+for _n, (_d, _H, _K) in PAPER_SHAPES.items():
+    WORKLOADS[f"paper{_n}_prefill"] = ("c3", dict(T=8192, d=_d, H=_H, K=_K))
+    WORKLOADS[f"paper{_n}_t32"] = ("c2", dict(T=32, d=_d, H=_H))
+NCU_TRAFFIC_BYTES = {}     # dram bytes per launch of the dominant kernel from the ncu captures under profiles/
+DEFAULT_STEPS = {"c3": 100, "c4": 50}
+ALSO = [("c2_t1", 500), ("c2_t8", 500), ("c3", 30), ("c4", 15)] + [(f"c5_eps{e}", 15) for e in (0.0, 0.01, 0.05, 0.1, 0.2)] + \
+       [(f"paper{n}_prefill", 30) for n in PAPER_SHAPES] + [(f"paper{n}_t32", 300) for n in ("1b", "3b", "6b", "19b")] + \
+       [("decode_loop_t8", 20), ("decode_loop_t32", 20)]
 METRIC = "moe_layer_tokens_per_s"
+NOMINAL = dict(hbm=8000.0, tf=2250.0)     # datasheet: HBM3e GB/s, dense bf16 TFLOP/s
+LOOP_LAYERS = 24
+
+
+def default_steps(name):
+    if name in DEFAULT_STEPS:
+        return DEFAULT_STEPS[name]
+    if name.startswith("decode_loop"):
+        return 40                                   # x 24 layers per step
+    if name.startswith("c5") or name.endswith("_prefill"):
+        return 50
+    return 1000
 
 
 def peaks():
@@ -189,7 +220,40 @@ def job_throughput(dist, ms_local: float, tokens_local: int, device="cuda"):
     return float(n.item()) / (ms * 1e-3), ms, dist.get_world_size()
 
 
-def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, sampler_index=0):
+_PACKED = {}      # (d, H, E, recipe name, w2_gain, layer) -> packed weights on the device, shared between workloads
+
+
+def packed_weights(dm, torch, s, desc, layer):
+    key = (s.d, s.H, s.E, s.name, s.w2_gain, layer)
+    if key not in _PACKED:
+        W1, W2 = gi.experts(s, layer)
+        W1_d = torch.from_numpy(W1.view(np.int16)).cuda().view(torch.bfloat16)
+        W2_d = torch.from_numpy(W2.view(np.int16)).cuda().view(torch.bfloat16)
+        pk = torch.empty(dm.dsmoe_packed_size(desc), dtype=torch.uint8, device="cuda")
+        dm.dsmoe_pack_weights(desc, W1_d, W2_d, pk)      # one-off, outside every timed region
+        torch.cuda.synchronize()
+        _PACKED[key] = pk
+    return _PACKED[key]
+
+
+def drop_weights(torch, keep_shape=None):
+    for k in list(_PACKED):
+        if keep_shape is None or k[:3] != keep_shape:
+            del _PACKED[k]
+    torch.cuda.empty_cache()
+
+
+def kernels_per_step(s, decode):
+    """Launches of this library's kernels in one dsmoe_layer_forward (memsets are not kernels)."""
+    if decode:
+        return 1                                   # small_layer_kernel
+    router = 3 if s.T > 256 else 1                 # split Wr, logits GEMM, softmax+select | one router kernel
+    if s.mode == gi.MODE_ALL:
+        return router + 2                          # up, down
+    return router + 3 + 2                          # chunk count, finalize, permute index, up, down (aggregation inside)
+
+
+def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, sampler_index=0, graph=False):
     import torch
     import paper_2404_05567_b200 as dm
 
@@ -200,38 +264,42 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
             return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
         return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
-    def desc_of(s):
-        return dm.make_desc(s.T, s.d, s.H, s.E, dm.BF16 if s.dtype == "bf16" else dm.F32, s.mode, s.eps,
-                            s.eps_normalized, s.K, s.min_k, s.out_fp32)
-
     cfg, kw = WORKLOADS[name]
     s = gi.spec(cfg, **kw)
-    desc = desc_of(s)
+    desc = dm.make_desc(s.T, s.d, s.H, s.E, dm.BF16, s.mode, s.eps, s.eps_normalized, s.K, s.min_k, s.out_fp32)
     P = peaks()
     decode = s.T <= 128
-    n_layers = 8 if decode else 1          # 8 x 268 MB of packed weights > 126 MB of L2
+    loop = name.startswith("decode_loop")
+    # decode: distinct weight sets, at least 2 GB in all (L2 holds 126 MB), cycled; the loop workloads chain 24 of them
+    per_layer = 4.0 * s.E * s.d * s.H
+    n_layers = LOOP_LAYERS if loop else (max(3, min(8, int(np.ceil(2.1e9 / per_layer)))) if decode else 1)
     Wr, br = gi.router(s)
     Wr_d, br_d = to_dev(Wr), to_dev(br)
-    packed = []
-    for layer in range(n_layers):
-        W1, W2 = gi.experts(s, layer)
-        W1_d, W2_d = to_dev(W1), to_dev(W2)
-        pk = torch.empty(dm.dsmoe_packed_size(desc), dtype=torch.uint8, device="cuda")
-        dm.dsmoe_pack_weights(desc, W1_d, W2_d, pk)      # one-off, outside every timed region
-        torch.cuda.synchronize()
-        packed.append(pk)
-        del W1_d, W2_d, W1, W2
+    packed = [packed_weights(dm, torch, s, desc, layer) for layer in range(n_layers)]
     x = gi.tokens(s)
     x_d = to_dev(x)
-    ws = torch.empty(dm.dsmoe_workspace_size(desc), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(dm.dsmoe_workspace_size_packed(desc), dtype=torch.uint8, device="cuda")
     out = torch.empty((s.T, s.d), dtype=torch.bfloat16, device="cuda")
+    act = [x_d, out, torch.empty_like(out)]           # loop workloads: layer i reads act[..] and writes the other
     mask = torch.zeros(s.T, dtype=torch.int64, device="cuda")
     counts = torch.zeros(64, dtype=torch.int32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
 
-    def step(i, want=False):
-        dm.dsmoe_layer_forward(desc, x_d, Wr_d, br_d, None, None, packed[i % n_layers], out,
+    def layer_call(i, src, dst, want=False):
+        dm.dsmoe_layer_forward(desc, src, Wr_d, br_d, None, None, packed[i % n_layers], dst,
                                mask if want else None, counts if want else None, ws, status)
+
+    if loop:
+        def step(i, want=False):
+            # one decoding step of a 24-layer stack: x -> layer 0 -> layer 1 -> ... (each layer its own weights)
+            src = x_d
+            for layer in range(n_layers):
+                dst = act[1 + layer % 2]
+                layer_call(layer, src, dst, want and layer == 0)
+                src = dst
+    else:
+        def step(i, want=False):
+            layer_call(i, x_d, out, want)
 
     step(0, want=True)
     torch.cuda.synchronize()
@@ -239,65 +307,103 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
     cnt = counts[:s.E].cpu().numpy()
     A = int(cnt.sum())
     n_act = int((cnt > 0).sum())
+    # selection statistics of this batch (stage calls, outside the timed region)
+    scores = torch.empty((s.T, s.E), dtype=torch.float32, device="cuda")
+    dm.dsmoe_router(desc, x_d, Wr_d, br_d, scores)
+    st_d = torch.zeros(288, dtype=torch.uint8, device="cuda")
+    dm.dsmoe_stats(desc, scores, mask, st_d)
+    stats = dm.read_stats(st_d)
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timed region
+    calls_per_step = n_layers if loop else 1
+    timed_per_call = 1 if decode else 2
+    run_step = step
+    if graph:
+        # the whole step as one CUDA graph (launch overhead out of the way)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(3):
+                step(i)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step(0)
+        run_step = lambda i, want=False: g.replay()     # noqa: E731
+
+    # ---- device-resident timed region.  The library's event pairs around the dominant kernel's launches sit in this
+    # same loop: the kernel times are those of the steps that make up `value`.
     for i in range(max(warmup, 3)):
-        step(i)
+        run_step(i)
+    n_pairs = 0 if graph else steps * calls_per_step * timed_per_call
+    dm.dsmoe_timing_enable(n_pairs)
     sampler = ClockSampler(sampler_index)
     barrier()
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(steps):
-        step(i)
+        run_step(i)
     e1.record()
     barrier()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.finish()
+    durs = np.array(dm.dsmoe_timing_read(n_pairs)) if n_pairs else np.zeros(0)
+    dm.dsmoe_timing_enable(0)
     value, ms_total, world = job_throughput(dist, ms_total, s.T * steps)
+    assert int(status.item()) == 0
 
-    # ---- per-launch time of the dominant kernel (the tcgen05 expert GEMM), CUDA events inside the library
-    dm.dsmoe_timing_enable(True)
-    n_timed = min(steps, 200)
-    durs = []
-    for i in range(n_timed):
-        step(i)
-        durs.append(dm.dsmoe_timing_last())
-    dm.dsmoe_timing_enable(False)
-    durs = np.array(durs)                        # [n_timed, timed launches per step]
-    per_step_launches = durs.shape[1]
-    launch_ms = float(durs.sum(axis=1).mean())   # time inside the dominant kernel per step
-    if decode:
-        # selected experts' weights (W1 and W2), each byte once, all inside one launch of small_layer_kernel
-        algo = 2.0 * n_act * s.d * s.H * 2.0
-        roof = dict(bound="hbm", achieved=algo / (launch_ms * 1e-3) / 1e9, peak=P["hbm"], unit="GB/s",
-                    peak_source=P["source"] + " (copy bandwidth)", kernel="small_layer_kernel")
-    else:
-        algo = 4.0 * A * s.d * s.H             # both projections: two launches of umma_gemm_kernel per step
-        roof = dict(bound="tensor", achieved=algo / (launch_ms * 1e-3) / 1e12, peak=P["tf_sustained"],
-                    unit="TFLOP/s", peak_source=P["source"] + " (sustained bf16)", kernel="umma_gemm_kernel")
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
-    # summarised under profiles/ (c3: mean of the up- and down-projection launches); null where no capture was taken
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get(name)
-    roof["launch_ms"] = launch_ms / per_step_launches
-    roof["launch_ms_each"] = [float(v) for v in durs.mean(axis=0)]
-    roof["launches_per_step"] = per_step_launches
-    roof["algorithmic_per_launch"] = algo / per_step_launches
-    # whole-step figure against the same roofline (what the layer as a whole achieves)
     step_s = ms_total * 1e-3 / steps
-    roof["step_frac"] = ((algo / step_s / 1e9) if decode else (algo / step_s / 1e12)) / roof["peak"]
-
-    res = dict(value=value, ms_per_step=ms_total / steps, clocks=clocks, roofline=roof, A=A, active_experts=n_act,
-               launches_per_step=(1 if decode else (5 if s.mode == gi.MODE_ALL else 9)), spec=s)
+    res = dict(value=value, ms_per_step=ms_total / steps, clocks=clocks, A=A, active_experts=n_act, stats=stats,
+               launches_per_step=kernels_per_step(s, decode) * calls_per_step, spec=s)
+    if len(durs):
+        durs = durs.reshape(steps, calls_per_step * timed_per_call)
+        kernel_ms = float(durs.sum(axis=1).mean())        # time inside the dominant kernel per step
+        capped = "sw_power_cap" in clocks["reasons"] or (clocks["sm_mhz"] and clocks["sm_max_mhz"] and
+                                                          clocks["sm_mhz"] < 0.9 * clocks["sm_max_mhz"])
+        weight_bytes = 2.0 * n_act * s.d * s.H * 2.0 * calls_per_step
+        flops = 4.0 * A * s.d * s.H * calls_per_step
+        if decode:
+            # selected experts' weights (W1 and W2), each byte once, all inside one launch of small_layer_kernel
+            roof = dict(bound="hbm", achieved=weight_bytes / (kernel_ms * 1e-3) / 1e9, peak=P["hbm"], unit="GB/s",
+                        peak_source=P["source"] + " (copy bandwidth)", kernel="small_layer_kernel")
+            roof["frac"] = roof["achieved"] / roof["peak"]
+            roof["frac_nominal"] = roof["achieved"] / NOMINAL["hbm"]
+            roof["step_frac"] = weight_bytes / step_s / 1e9 / roof["peak"]
+            roof["algorithmic_per_launch"] = weight_bytes / calls_per_step
+        else:
+            # both projections: two launches of umma_gemm_kernel per step.  Peak: the burst figure unless the clock
+            # samples of this very region show the power cap (then the sustained one applies)
+            kind = "sustained" if capped else "burst"
+            peak = P["tf_sustained"] if capped else P["tf_burst"]
+            ach = flops / (kernel_ms * 1e-3) / 1e12
+            roof = dict(bound="tensor", achieved=ach, peak=peak, unit="TFLOP/s",
+                        peak_source=f"{P['source']} ({kind} bf16: clocks of this region {'show' if capped else 'show no'} power cap)",
+                        kernel="umma_gemm_kernel", frac=ach / peak, frac_burst=ach / P["tf_burst"],
+                        frac_sustained=ach / P["tf_sustained"], frac_nominal=ach / NOMINAL["tf"],
+                        step_frac=flops / step_s / 1e12 / peak, algorithmic_per_launch=flops / 2)
+            # where few assignments are left the weights' bytes bound the step, not the flops: the roofline time is
+            # the larger of the two
+            t_flop, t_byte = flops / (peak * 1e12), weight_bytes / (P["hbm"] * 1e9)
+            roof["roofline_ms"] = max(t_flop, t_byte) * 1e3
+            roof["roofline_bound"] = "tensor" if t_flop >= t_byte else "hbm"
+            roof["frac_of_roofline_time"] = max(t_flop, t_byte) / (kernel_ms * 1e-3)
+            roof["step_frac_of_roofline_time"] = max(t_flop, t_byte) / step_s
+        # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
+        # summarised under profiles/; null where no capture of the current kernel exists
+        roof["traffic"] = NCU_TRAFFIC_BYTES.get(name)
+        roof["kernel_ms_per_step"] = kernel_ms
+        roof["launch_ms_each"] = [float(v) for v in durs.mean(axis=0)[:timed_per_call]]
+        roof["launches_per_step"] = calls_per_step * timed_per_call
+        res["roofline"] = roof
 
     # ---- end to end through the host-buffer entry point
-    if with_e2e:
+    if with_e2e and not loop:
         x_host = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory()
         out_host = torch.empty((s.T, s.d), dtype=torch.bfloat16).pin_memory()
 
@@ -319,15 +425,56 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
         res["e2e"] = {"value": e2e_value, "unit": "tokens/s",
                       "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes}
     del packed, ws
-    torch.cuda.empty_cache()
     return res
 
 
 def workload_config(name, s):
-    mode = {0: "threshold", 1: "topk", 2: "all"}[s.mode]
+    mode = {0: "threshold", 1: "topk", 2: "all", 3: "threshold_topk"}[s.mode]
     return {"workload": name, "T": s.T, "d": s.d, "E": s.E, "H": s.H, "select": mode, "eps": s.eps, "K": s.K,
-            "l2": "decode: 8 weight sets cycled (2.1 GB > L2); prefill/dense: > L2 touched per step",
+            "l2": "decode: distinct weight sets cycled (>= 2 GB in all > L2; 24 chained in the loop workloads); prefill/dense: > L2 touched per step",
             "weights": "packed once outside the timed region"}
+
+
+def free_port() -> int:
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        return so.getsockname()[1]
+
+
+def launch_ranks(n: int, argv) -> int:
+    """Starts n copies of this script, one per GPU, with the rendezvous variables torchrun would set.
+    Rank 0 inherits stdout (it prints the JSON line); the exit code is the worst of the ranks'."""
+    port = free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=env,
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    rc = 0
+    for p in procs:
+        rc = max(rc, abs(p.wait()))
+    return rc
+
+
+def rendezvous_only(rank, world):
+    """Everything of the N-rank run but the GPU work: process group (NCCL on GPUs, gloo without), barrier, and
+    the reduction of a per-rank timing into the whole-job figure.  Used to check the launch path on CPU."""
+    import torch
+    import torch.distributed as td
+    cuda = torch.cuda.is_available() and torch.cuda.device_count() >= world
+    if cuda:
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if world > 1:
+        td.init_process_group("nccl" if cuda else "gloo")
+        td.barrier()
+    value, ms, n = job_throughput(td if world > 1 else None, 10.0 * (rank + 1), 1000, device="cuda" if cuda else "cpu")
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "rendezvous_only": True, "n_gpus": n, "value": value, "ms_per_step": ms,
+                          "backend": "nccl" if cuda else "gloo"}))
+    if world > 1:
+        td.barrier()
+        td.destroy_process_group()
 
 
 def main():
@@ -338,16 +485,25 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_t32", choices=sorted(WORKLOADS))
     ap.add_argument("--no-extra", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="replay each step as one CUDA graph")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--rendezvous-only", action="store_true",
+                    help="start the ranks, reduce a stand-in timing and print n_gpus; no GPU work")
     args = ap.parse_args()
     name = args.workload
-    steps = args.steps if args.steps is not None else DEFAULT_STEPS[name]
+    steps = args.steps if args.steps is not None else default_steps(name)
     warmup = args.warmup if args.warmup is not None else 20
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     cfg, kw = WORKLOADS[name]
     s = gi.spec(cfg, **kw)
+
+    if args.rendezvous_only:
+        rendezvous_only(rank, world)
+        return
 
     if args.impl == "reference":
         if rank != 0:
@@ -379,30 +535,39 @@ def main():
     if dist is not None:
         dist.barrier()
 
-    res = run_workload(name, steps, warmup, dist=dist, sampler_index=physical_gpu_index(local_rank))
+    res = run_workload(name, steps, warmup, dist=dist, sampler_index=physical_gpu_index(local_rank), graph=args.graph)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
     s = res["spec"]
+    st = res["stats"]
     line = {"metric": METRIC, "value": res["value"], "unit": "tokens/s", "n_gpus": world, "steps": steps,
             "warmup": max(warmup, 3), "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(name, s),
             "clocks": res["clocks"], "e2e": res.get("e2e"), "gpu_launches": res["launches_per_step"] * steps,
-            "roofline": res["roofline"], "assignments": res["A"], "active_experts": res["active_experts"]}
+            "roofline": res.get("roofline"), "assignments": res["A"], "active_experts": res["active_experts"],
+            "selection": {"near_threshold_1e-6": st["near_threshold"], "zero_tokens": st["zero_tokens"],
+                          "empty_experts": st["empty_experts"]}}
     if world == 1:
         cb = oracle_tokens_per_s(s, budget_s=args.cpu_budget)
         line["cpu_baseline"] = {"value": cb["value"], "unit": "tokens/s", "cores": cb["cores"], "kind": "oracle",
                                 "sample": cb["sample"]}
         if not args.no_extra:
             also = []
-            for other, k in (("c2_t1", 500), ("c2_t8", 500), ("c3", 30), ("c4", 15)):
+            shape = None
+            for other, k in ALSO:
                 if other == name:
                     continue
+                so = gi.spec(WORKLOADS[other][0], **WORKLOADS[other][1])
+                if shape is not None and (so.d, so.H, so.E) != shape:
+                    drop_weights(torch, keep_shape=(so.d, so.H, so.E))   # keep the device's memory use bounded
+                shape = (so.d, so.H, so.E)
                 r = run_workload(other, k, 5, with_e2e=False, sampler_index=physical_gpu_index(local_rank))
                 also.append({"workload": other, "value": r["value"], "unit": "tokens/s", "ms_per_step": r["ms_per_step"],
-                             "steps": k, "roofline": r["roofline"], "clocks": r["clocks"], "assignments": r["A"],
-                             "active_experts": r["active_experts"]})
+                             "steps": k, "roofline": r.get("roofline"), "clocks": r["clocks"], "assignments": r["A"],
+                             "active_experts": r["active_experts"],
+                             "near_threshold_1e-6": r["stats"]["near_threshold"]})
             line["also"] = also
     print(json.dumps(line))
     if dist is not None:

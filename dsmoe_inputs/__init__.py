@@ -137,6 +137,7 @@ class LayerSpec:
     router_gain: float = 1.0       # scalar applied to the drawn Wr
     zipf_s: float = 0.0            # > 0: router bias b[e] = ln p, p ~ Zipf(s) over a seeded permutation
     seed: int = 0
+    w2_gain: float = 1.0           # scalar applied to the drawn W2 (layer stacks: keeps the activations' scale)
 
     def replace(self, **kw) -> "LayerSpec":
         d = asdict(self)
@@ -196,7 +197,7 @@ def router(s: LayerSpec, layer: int = 0):
 def experts(s: LayerSpec, layer: int = 0):
     """(W1[E,d,H], W2[E,H,d]) ~ N(0,0.02^2) in the layer's storage type."""
     W1 = normal(s.seed, f"{s.name}.W1.{layer}", (s.E, s.d, s.H), 0.02, s.dtype)
-    W2 = normal(s.seed, f"{s.name}.W2.{layer}", (s.E, s.H, s.d), 0.02, s.dtype)
+    W2 = normal(s.seed, f"{s.name}.W2.{layer}", (s.E, s.H, s.d), 0.02 * s.w2_gain, s.dtype)
     return W1, W2
 
 

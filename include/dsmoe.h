@@ -32,6 +32,9 @@
  *   - Amax = T*E for THRESHOLD and ALL, T*min(K,E) for TOPK: the capacity of every
  *     per-assignment buffer, so the data-dependent A never has to reach the host.
  *   - W = E for THRESHOLD and ALL, min(K,E) for TOPK: row stride of token_rows.
+ *   - Host side: one thread at a time may call into the library (it keeps small per-device and
+ *     per-buffer caches without locks).  Any number of devices may be used from that thread; a call
+ *     works on the current device, which must own every pointer passed.
  */
 #ifndef DSMOE_H_
 #define DSMOE_H_
@@ -84,9 +87,18 @@ typedef void* dsmoe_stream;
 
 const char* dsmoe_status_string(dsmoe_status s);
 
-/* Bytes of scratch that dsmoe_permute, dsmoe_expert_mlp and dsmoe_layer_forward need for
- * this desc (one figure, the maximum over the three and over the internal paths). */
+/* Bytes of scratch for this desc.  A call takes one of two kinds of path, and their buffers overlap:
+ * the plain path (fp32 layers, or no packed weights: grouped copy of the tokens, fp32 hidden
+ * activations, expert outputs) and the tensor-core paths (packed bf16 weights: bf16 hidden activations
+ * and an fp32 running sum of [T,d]).
+ *   dsmoe_workspace_size         enough for any call with this desc (the larger of the two)
+ *   dsmoe_workspace_size_packed  enough for dsmoe_expert_mlp / dsmoe_layer_forward when `packed` is
+ *                                given (DSMOE_ERR_UNSUPPORTED if this desc has no tensor-core path)
+ *   dsmoe_workspace_size_stages  enough for dsmoe_select and dsmoe_permute (index scratch only)
+ * Every entry point checks ws_bytes against the figure of the path it takes. */
 dsmoe_status dsmoe_workspace_size(const dsmoe_layer_desc* desc, size_t* bytes);
+dsmoe_status dsmoe_workspace_size_packed(const dsmoe_layer_desc* desc, size_t* bytes);
+dsmoe_status dsmoe_workspace_size_stages(const dsmoe_layer_desc* desc, size_t* bytes);
 
 /*
  * Router scores, Eq. 1 (first half): scores[t,:] = softmax(x[t,:].Wr + br) over all E
@@ -102,7 +114,7 @@ dsmoe_status dsmoe_router(const dsmoe_layer_desc* desc, const void* x, const flo
  *   scores [T,E] fp32 (read); mask [T] uint64, bit e set iff expert e is selected;
  *   k_t [T] int32 = popcount(mask); counts [E] int32 = tokens per expert;
  *   offsets [E+1] int32 = exclusive prefix sum of counts, offsets[E] = A.
- * All four outputs are written in full.  workspace as reported by dsmoe_workspace_size.
+ * All four outputs are written in full.  workspace: at least dsmoe_workspace_size_stages bytes.
  */
 dsmoe_status dsmoe_select(const dsmoe_layer_desc* desc, const float* scores, uint64_t* mask,
                           int32_t* k_t, int32_t* counts, int32_t* offsets, void* workspace,
@@ -133,6 +145,8 @@ dsmoe_status dsmoe_select_static(const dsmoe_layer_desc* desc, const float* scor
  *   row_token [Amax] int32: token of row r;  row_gate [Amax] fp32: scores[token,e];
  *   token_rows [T,W] int32: rows of token t in ascending expert order, -1 beyond k_t;
  *   xp [Amax,d] dtype: xp[r,:] = x[row_token[r],:].  Entries at r >= A are not written.
+ *   workspace: at least dsmoe_workspace_size_stages bytes.  A row index that falls outside
+ *   [0, Amax) because the given offsets do not belong to the given mask is skipped, never stored to.
  */
 dsmoe_status dsmoe_permute(const dsmoe_layer_desc* desc, const void* x, const float* scores,
                            const uint64_t* mask, const int32_t* offsets, int32_t* row_token,
@@ -146,6 +160,10 @@ dsmoe_status dsmoe_permute(const dsmoe_layer_desc* desc, const void* x, const fl
  *   yp [Amax,d] dtype (written for r < A).
  *   packed: NULL, or the buffer dsmoe_pack_weights filled from these W1, W2 (bf16 only);
  *   with it the tensor-core kernels run, without it a plain fp32-FMA kernel does.
+ *   dev_status: optional device int32.  The tensor-core kernels check the segments first: an expert
+ *   whose [offsets[e], offsets[e+1]) is negative, decreasing or ends beyond Amax is treated as empty
+ *   (none of its rows is written) and DSMOE_ERR_INVALID_ARG is stored there; DSMOE_ERR_TIMEOUT if a
+ *   bounded wait ran out.
  */
 dsmoe_status dsmoe_expert_mlp(const dsmoe_layer_desc* desc, const void* xp, const void* W1,
                               const void* W2, const void* packed, const int32_t* offsets,
@@ -183,6 +201,10 @@ dsmoe_status dsmoe_pack_weights(const dsmoe_layer_desc* desc, const void* W1, co
  *   mask_out [T] uint64 and counts_out [E] int32: optional copies of the selection.
  *   dev_status: optional device int32; kernels write a dsmoe_status there if a bounded
  *   wait runs out or an index check fails (they then exit cleanly); untouched otherwise.
+ *   With packed weights and a sparse selection the aggregation runs inside the down-projection:
+ *   each expert's output is multiplied by its gate in fp32 and added to the token's fp32 sum in
+ *   ascending expert order (the order dsmoe_combine uses), and rounded once when the token's last
+ *   expert is done; results are bit-identical from run to run.
  */
 dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, const float* Wr,
                                  const float* br, const void* W1, const void* W2,
@@ -202,15 +224,37 @@ dsmoe_status dsmoe_layer_forward_host(const dsmoe_layer_desc* desc, const void* 
                                       size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream);
 
 /*
- * Measurement aid (no counterpart in the paper): with timing enabled, every tensor-core expert
- * GEMM launch of dsmoe_expert_mlp / dsmoe_layer_forward is bracketed by a pair of CUDA events on
- * the caller's stream.  dsmoe_timing_enable(1) creates the events once (call it outside any timed
- * region); dsmoe_timing_last waits for the most recent call's launches and writes their durations
- * in milliseconds, in launch order (up-projection, then down-projection), to the HOST array ms
- * (at most n_max), setting *n to the number written.  Not thread-safe; off by default.
+ * Selection statistics for logging ("Layer Utilization" paragraph: active experts per layer and per
+ * token; Section 4.2 footnote for the threshold).  Written to the DEVICE struct `stats`:
+ *   assignments     A = sum_t k_t                          zero_tokens    tokens that selected no expert
+ *   counts[e]       tokens that selected expert e          empty_experts  experts selected by no token
+ *   near_threshold  threshold rules only: how many scores lie within 1e-6 of eps (in the quantity the
+ *                   rule compares: S, or fl32(S*E) when eps_normalized) -- decisions that a different
+ *                   rounding of the softmax could flip; 0 for the other rules
+ *   scores [T,E], mask [T]: read.  The caller copies the struct back when it wants the figures.
  */
-dsmoe_status dsmoe_timing_enable(int on);
-dsmoe_status dsmoe_timing_last(float* ms, int n_max, int* n);
+typedef struct {
+    int64_t assignments;
+    int64_t near_threshold;
+    int32_t zero_tokens;
+    int32_t empty_experts;
+    int32_t counts[64];
+} dsmoe_selection_stats;
+
+dsmoe_status dsmoe_stats(const dsmoe_layer_desc* desc, const float* scores, const uint64_t* mask,
+                         dsmoe_selection_stats* stats, dsmoe_stream stream);
+
+/*
+ * Measurement aid (no counterpart in the paper): a ring of CUDA event pairs on the caller's stream.
+ * After dsmoe_timing_enable(n_pairs) (n_pairs > 0; events are created here, so call it outside any
+ * timed region), every launch of an expert-MLP tensor-core kernel (the two grouped or dense GEMMs of
+ * a prefill call, the one kernel of a decode call) is bracketed by the next pair until n_pairs are
+ * used.  dsmoe_timing_read waits for the recorded pairs, writes their durations in milliseconds, in
+ * launch order, to the HOST array ms (at most n_max), sets *n and empties the ring.
+ * dsmoe_timing_enable(0) switches it off.  Off by default.
+ */
+dsmoe_status dsmoe_timing_enable(int n_pairs);
+dsmoe_status dsmoe_timing_read(float* ms, int n_max, int* n);
 
 #ifdef __cplusplus
 }

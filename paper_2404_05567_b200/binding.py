@@ -22,8 +22,8 @@ SELECT_THRESHOLD, SELECT_TOPK, SELECT_ALL, SELECT_THRESHOLD_TOPK = 0, 1, 2, 3
 EXPORTS = (
     "dsmoe_status_string", "dsmoe_workspace_size", "dsmoe_router", "dsmoe_select", "dsmoe_permute",
     "dsmoe_expert_mlp", "dsmoe_combine", "dsmoe_packed_size", "dsmoe_pack_weights",
-    "dsmoe_layer_forward", "dsmoe_layer_forward_host", "dsmoe_timing_enable", "dsmoe_timing_last",
-    "dsmoe_select_static",
+    "dsmoe_layer_forward", "dsmoe_layer_forward_host", "dsmoe_timing_enable", "dsmoe_timing_read",
+    "dsmoe_select_static", "dsmoe_workspace_size_packed", "dsmoe_workspace_size_stages", "dsmoe_stats",
 )
 
 
@@ -101,6 +101,36 @@ def dsmoe_workspace_size(desc: LayerDesc) -> int:
     return n.value
 
 
+def dsmoe_workspace_size_packed(desc: LayerDesc) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().dsmoe_workspace_size_packed(ctypes.byref(desc), ctypes.byref(n)), "dsmoe_workspace_size_packed")
+    return n.value
+
+
+def dsmoe_workspace_size_stages(desc: LayerDesc) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().dsmoe_workspace_size_stages(ctypes.byref(desc), ctypes.byref(n)), "dsmoe_workspace_size_stages")
+    return n.value
+
+
+class SelectionStats(ctypes.Structure):
+    _fields_ = [("assignments", ctypes.c_int64), ("near_threshold", ctypes.c_int64), ("zero_tokens", ctypes.c_int32),
+                ("empty_experts", ctypes.c_int32), ("counts", ctypes.c_int32 * 64)]
+
+
+def dsmoe_stats(desc, scores, mask, stats, stream=None):
+    """``stats``: a CUDA uint8 tensor of ``ctypes.sizeof(SelectionStats)`` bytes; see ``read_stats``."""
+    _check(lib().dsmoe_stats(ctypes.byref(desc), _ptr(scores), _ptr(mask), _ptr(stats), _stream(stream)), "dsmoe_stats")
+
+
+def read_stats(stats) -> dict:
+    """Copies the device struct back (synchronises) and returns it as a dict."""
+    raw = bytes(stats.cpu().numpy().tobytes())
+    st = SelectionStats.from_buffer_copy(raw)
+    return dict(assignments=int(st.assignments), near_threshold=int(st.near_threshold), zero_tokens=int(st.zero_tokens),
+                empty_experts=int(st.empty_experts), counts=[int(c) for c in st.counts])
+
+
 def dsmoe_packed_size(desc: LayerDesc) -> int:
     n = ctypes.c_size_t(0)
     _check(lib().dsmoe_packed_size(ctypes.byref(desc), ctypes.byref(n)), "dsmoe_packed_size")
@@ -161,15 +191,15 @@ def dsmoe_layer_forward_host(desc, x_host, x_dev, Wr, br, W1, W2, packed, out_de
                                           _ptr(dev_status), _stream(stream)), "dsmoe_layer_forward_host")
 
 
-def dsmoe_timing_enable(on: bool):
-    _check(lib().dsmoe_timing_enable(ctypes.c_int(1 if on else 0)), "dsmoe_timing_enable")
+def dsmoe_timing_enable(n_pairs: int):
+    _check(lib().dsmoe_timing_enable(ctypes.c_int(int(n_pairs))), "dsmoe_timing_enable")
 
 
-def dsmoe_timing_last(n_max: int = 8):
-    """Durations (ms) of the expert-GEMM launches of the most recent call, in launch order."""
-    buf = (ctypes.c_float * n_max)()
+def dsmoe_timing_read(n_max: int):
+    """Durations (ms) of the timed launches since the ring was enabled or last read, in launch order."""
+    buf = (ctypes.c_float * max(n_max, 1))()
     n = ctypes.c_int(0)
-    _check(lib().dsmoe_timing_last(buf, ctypes.c_int(n_max), ctypes.byref(n)), "dsmoe_timing_last")
+    _check(lib().dsmoe_timing_read(buf, ctypes.c_int(n_max), ctypes.byref(n)), "dsmoe_timing_read")
     return [float(buf[i]) for i in range(n.value)]
 
 

@@ -40,23 +40,55 @@ WsLayout ws_layout(const dsmoe_layer_desc& p) {
     L.counts = take(kMaxExperts * 4);
     L.offsets = take((kMaxExperts + 1) * 4);
     L.chunk_prefix = take((size_t)ceil_div(p.T, kChunk) * E * 4);
+    L.batch_k = take(256);               // Threshold-TopK: the batch's K
+    L.sync = take(64);                   // grid-barrier counters of the small-T kernel
+    L.tile_done = take((size_t)kMaxExperts * ceil_div(p.d, 256) * 4);   // grouped down-projection: finished tiles per (expert, column range)
     L.row_token = take(amax * 4);
     L.row_gate = take(amax * 4);
     L.token_rows = take(T * (size_t)width_of(p) * 4);
+    L.stage_total = off;
+    const size_t big0 = off;
+    // plain path: grouped copy of the tokens, fp32 hidden activations, expert outputs
     L.xp = take(amax * p.d * es);
-    // h: fp32 [Amax,H] in the plain path, bf16 [Amax,H] in the grouped tensor-core path, bf16 [T,E*H] in
-    // the dense and small-T paths
-    size_t h_bytes = amax * p.H * 4;
-    if (p.T <= kSmallMaxT && T * E * p.H * 2 > h_bytes) h_bytes = T * E * p.H * 2;
-    L.h = take(h_bytes);
+    L.h_plain = take(amax * p.H * 4);
     L.yp = take(amax * p.d * es);
+    L.total_plain = off;
+    // tensor-core paths (bf16, packed weights); they start where the plain path's buffers start
+    off = big0;
+    size_t h_bytes = 0;
+    if (umma_supported(p)) {
+        h_bytes = amax * p.H * 2;                                   // grouped: [Amax, H]
+        if (T * E * p.H * 2 > h_bytes && (p.mode == DSMOE_SELECT_ALL || p.T <= kSmallMaxT))
+            h_bytes = T * E * p.H * 2;                              // dense forward, small-T: [T, E*H]
+    }
+    L.h = take(h_bytes);
+    L.acc = take(umma_supported(p) ? T * p.d * 4 : 0);
     // fp32 partial sums of the small-T path: (CTA, 2 column ranges, T, 256)
-    L.partial = take(p.T <= kSmallMaxT ? (size_t)kSmallMaxCtas * 2 * T * 256 * 4 : 0);
-    L.sync = take(64);                   // grid-barrier counters of the small-T kernel
+    L.partial = take(umma_supported(p) && p.T <= kSmallMaxT ? (size_t)kSmallMaxCtas * 2 * T * 256 * 4 : 0);
     L.router = take(router_umma_supported(p) ? router_umma_scratch(p) : 0);   // tensor-core router: split Wr, partial logits
-    L.batch_k = take(256);               // Threshold-TopK: the batch's K
-    L.total = off;
+    L.total_packed = off;
+    L.total = L.total_plain > L.total_packed ? L.total_plain : L.total_packed;
     return L;
+}
+
+namespace {
+DeviceState g_dev_state[kMaxDeviceSlots];
+}
+
+dsmoe_status device_state(DeviceState** out, int* device) {
+    int dev = -1;
+    DSMOE_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDeviceSlots) return DSMOE_ERR_UNSUPPORTED;
+    DeviceState& st = g_dev_state[dev];
+    if (!st.sm_count) {
+        int n = 0;
+        DSMOE_CUDA_TRY(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
+        if (n <= 0) return DSMOE_ERR_CUDA;
+        st.sm_count = n;
+    }
+    *out = &st;
+    if (device) *device = dev;
+    return DSMOE_OK;
 }
 
 static const char* const kStatusText[] = {
@@ -80,6 +112,21 @@ dsmoe_status dsmoe_workspace_size(const dsmoe_layer_desc* desc, size_t* bytes) {
     return DSMOE_OK;
 }
 
+dsmoe_status dsmoe_workspace_size_packed(const dsmoe_layer_desc* desc, size_t* bytes) {
+    DSMOE_TRY(check_desc(desc));
+    if (!bytes) return DSMOE_ERR_INVALID_ARG;
+    if (!umma_supported(*desc)) return DSMOE_ERR_UNSUPPORTED;
+    *bytes = ws_layout(*desc).total_packed;
+    return DSMOE_OK;
+}
+
+dsmoe_status dsmoe_workspace_size_stages(const dsmoe_layer_desc* desc, size_t* bytes) {
+    DSMOE_TRY(check_desc(desc));
+    if (!bytes) return DSMOE_ERR_INVALID_ARG;
+    *bytes = ws_layout(*desc).stage_total;
+    return DSMOE_OK;
+}
+
 dsmoe_status dsmoe_router(const dsmoe_layer_desc* desc, const void* x, const float* Wr, const float* br,
                           float* scores, dsmoe_stream stream) {
     DSMOE_TRY(check_desc(desc));
@@ -95,7 +142,7 @@ dsmoe_status dsmoe_select(const dsmoe_layer_desc* desc, const float* scores, uin
     if (!mask && desc->T > 0) return DSMOE_ERR_INVALID_ARG;
     if (!counts || !offsets || (!scores && desc->T > 0) || (!k_t && desc->T > 0)) return DSMOE_ERR_INVALID_ARG;
     const WsLayout L = ws_layout(*desc);
-    if (!workspace || ws_bytes < L.total) return DSMOE_ERR_WORKSPACE;
+    if (!workspace || ws_bytes < L.stage_total) return DSMOE_ERR_WORKSPACE;
     char* ws = static_cast<char*>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
     DSMOE_TRY(launch_select(*desc, scores, mask, k_t, s, reinterpret_cast<int*>(ws + L.batch_k)));
@@ -110,7 +157,7 @@ dsmoe_status dsmoe_permute(const dsmoe_layer_desc* desc, const void* x, const fl
     if (!x || !scores || !mask || !offsets || !row_token || !row_gate || !token_rows || !xp) return DSMOE_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(xp)) return DSMOE_ERR_INVALID_ARG;
     const WsLayout L = ws_layout(*desc);
-    if (!workspace || ws_bytes < L.total) return DSMOE_ERR_WORKSPACE;
+    if (!workspace || ws_bytes < L.stage_total) return DSMOE_ERR_WORKSPACE;
     char* ws = static_cast<char*>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
     // recompute the per-chunk ranks from the mask (the caller's offsets are used as given)
@@ -130,13 +177,13 @@ dsmoe_status dsmoe_expert_mlp(const dsmoe_layer_desc* desc, const void* xp, cons
     if (packed && desc->dtype != DSMOE_BF16) return DSMOE_ERR_INVALID_ARG;
     if (!packed && (!W1 || !W2 || !aligned16(W1) || !aligned16(W2))) return DSMOE_ERR_INVALID_ARG;
     const WsLayout L = ws_layout(*desc);
-    if (!workspace || ws_bytes < L.total) return DSMOE_ERR_WORKSPACE;
+    const bool fast = packed && umma_supported(*desc);
+    if (!fast && (!W1 || !W2)) return DSMOE_ERR_UNSUPPORTED;   // packed weights given, but this shape needs the plain path
+    if (!workspace || ws_bytes < (fast ? L.total_packed : L.total_plain)) return DSMOE_ERR_WORKSPACE;
     char* ws = static_cast<char*>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
-    timing_reset();
-    if (packed && umma_supported(*desc)) return launch_mlp_umma(*desc, xp, packed, offsets, ws + L.h, yp, dev_status, s);
-    if (!W1 || !W2) return DSMOE_ERR_UNSUPPORTED;   // packed weights given, but this shape needs the plain path
-    return launch_mlp_generic(*desc, xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h), yp, s);
+    if (fast) return launch_mlp_umma(*desc, xp, packed, offsets, ws + L.h, yp, dev_status, s);
+    return launch_mlp_generic(*desc, xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h_plain), yp, s);
 }
 
 dsmoe_status dsmoe_combine(const dsmoe_layer_desc* desc, const void* yp, const float* row_gate,
@@ -173,7 +220,9 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     if (packed && p.dtype != DSMOE_BF16) return DSMOE_ERR_INVALID_ARG;
     if (!packed && (!W1 || !W2 || !aligned16(W1) || !aligned16(W2))) return DSMOE_ERR_INVALID_ARG;
     const WsLayout L = ws_layout(p);
-    if (!workspace || ws_bytes < L.total || !aligned16(workspace)) return DSMOE_ERR_WORKSPACE;
+    const bool fast = packed && umma_supported(p);
+    if (!fast && (!W1 || !W2)) return DSMOE_ERR_UNSUPPORTED;   // this shape needs the unpacked weights
+    if (!workspace || ws_bytes < (fast ? L.total_packed : L.total_plain) || !aligned16(workspace)) return DSMOE_ERR_WORKSPACE;
     char* ws = static_cast<char*>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
 
@@ -186,10 +235,6 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     int32_t* row_token = reinterpret_cast<int32_t*>(ws + L.row_token);
     float* row_gate = reinterpret_cast<float*>(ws + L.row_gate);
     int32_t* token_rows = reinterpret_cast<int32_t*>(ws + L.token_rows);
-
-    const bool fast = packed && umma_supported(p);
-    if (!fast && (!W1 || !W2)) return DSMOE_ERR_UNSUPPORTED;   // this shape needs the unpacked weights
-    timing_reset();
 
     if (fast && small_supported(p))
         return launch_layer_small(p, x, Wr, br, packed, scores, mask, k_t, counts_out, out, ws, L, dev_status, s);
@@ -212,13 +257,17 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
 
     // grouped path: duplicate tokens per selected expert, run the experts, aggregate
     DSMOE_TRY(launch_finalize(p, mask, counts, offsets, chunk_prefix, counts_out, s));
-    // the tensor-core path needs no grouped copy of the tokens: its up-projection gathers rows of x by row_token
-    DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows,
-                             fast ? nullptr : ws + L.xp, s));
-    if (fast)
-        DSMOE_TRY(launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, ws + L.yp, dev_status, s, x, row_token));
-    else
-        DSMOE_TRY(launch_mlp_generic(p, ws + L.xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h), ws + L.yp, s));
+    if (fast) {
+        // Tensor-core path: no grouped copy of the tokens (the up-projection gathers rows of x by row_token), no
+        // buffer of expert outputs and no aggregation pass (the down-projection's epilogue adds each expert's
+        // gate-weighted output to the token's fp32 sum, in ascending expert order, and writes the final rounding).
+        DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, nullptr, s, out));
+        const CombineArgs cmb{row_token, row_gate, mask, reinterpret_cast<float*>(ws + L.acc),
+                              reinterpret_cast<int*>(ws + L.tile_done), out};
+        return launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, nullptr, dev_status, s, x, row_token, &cmb);
+    }
+    DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, ws + L.xp, s));
+    DSMOE_TRY(launch_mlp_generic(p, ws + L.xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h_plain), ws + L.yp, s));
     return launch_combine(p, ws + L.yp, row_gate, token_rows, k_t, out, s);
 }
 
@@ -240,11 +289,21 @@ dsmoe_status dsmoe_layer_forward_host(const dsmoe_layer_desc* desc, const void* 
     return DSMOE_OK;
 }
 
-dsmoe_status dsmoe_timing_enable(int on) { return timing_enable(on); }
+dsmoe_status dsmoe_stats(const dsmoe_layer_desc* desc, const float* scores, const uint64_t* mask,
+                         dsmoe_selection_stats* stats, dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    if (!stats || (desc->T > 0 && (!scores || !mask))) return DSMOE_ERR_INVALID_ARG;
+    return launch_stats(*desc, scores, mask, stats, (cudaStream_t)stream);
+}
 
-dsmoe_status dsmoe_timing_last(float* ms, int n_max, int* n) {
+dsmoe_status dsmoe_timing_enable(int n_pairs) {
+    if (n_pairs < 0 || n_pairs > (1 << 20)) return DSMOE_ERR_INVALID_ARG;
+    return timing_enable(n_pairs);
+}
+
+dsmoe_status dsmoe_timing_read(float* ms, int n_max, int* n) {
     if (!ms || !n || n_max < 0) return DSMOE_ERR_INVALID_ARG;
-    return timing_last(ms, n_max, n);
+    return timing_read(ms, n_max, n);
 }
 
 }  // extern "C"

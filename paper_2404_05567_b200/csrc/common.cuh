@@ -40,12 +40,30 @@ static inline size_t amax_of(const dsmoe_layer_desc& p) { return (size_t)p.T * (
 dsmoe_status check_desc(const dsmoe_layer_desc* desc);
 static inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
-// Byte offsets of every internal buffer inside the caller's workspace.
+// Byte offsets of every internal buffer inside the caller's workspace.  The small per-token and per-assignment
+// index buffers come first (`stage_total` bytes: all that dsmoe_select and dsmoe_permute touch); the large
+// activation buffers follow and overlap between the execution paths, of which a call takes exactly one:
+//   plain (fp32-FMA GEMMs)     xp, h (fp32), yp
+//   tensor-core paths          h (bf16: grouped [Amax,H]; dense and small-T [T,E*H]), acc (grouped: fp32 [T,d] running
+//                              sum of the expert outputs), partial (small-T), router (split Wr, partial logits)
+// total_packed = bytes a call with packed weights needs; total = the maximum over both kinds of call.
 struct WsLayout {
-    size_t scores, mask, k_t, counts, offsets, chunk_prefix, row_token, row_gate, token_rows;
-    size_t xp, h, yp, partial, sync, router, batch_k, total;
+    size_t scores, mask, k_t, counts, offsets, chunk_prefix, batch_k, sync, tile_done, row_token, row_gate, token_rows;
+    size_t stage_total;
+    size_t xp, h_plain, yp;                 // plain path
+    size_t h, acc, partial, router;         // tensor-core paths
+    size_t total_plain, total_packed, total;
 };
 WsLayout ws_layout(const dsmoe_layer_desc& p);
+
+// What the library keeps per device (attributes that must be set once per device, the SM count).  Entry points
+// are not thread-safe: one host thread at a time may call into the library.
+constexpr int kMaxDeviceSlots = 64;
+struct DeviceState {
+    int sm_count = 0;
+    bool attr_gemm = false, attr_small = false, attr_router_f32 = false, attr_router_bf16 = false;
+};
+dsmoe_status device_state(DeviceState** out, int* device = nullptr);   // of the current device
 
 // ---- router.cu
 dsmoe_status launch_router(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
@@ -57,10 +75,14 @@ dsmoe_status launch_finalize(const dsmoe_layer_desc& p, const uint64_t* mask, in
                              int32_t* offsets, int32_t* chunk_prefix, int32_t* counts_out, cudaStream_t s);
 
 // ---- permute.cu
+// zero_out (optional): the layer output [T,d]; rows of tokens that selected no expert are set to zero
 dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const float* scores,
                             const uint64_t* mask, const int32_t* offsets, const int32_t* chunk_prefix,
                             int32_t* row_token, float* row_gate, int32_t* token_rows, void* xp,
-                            cudaStream_t s);
+                            cudaStream_t s, void* zero_out = nullptr);
+// Selection statistics (see dsmoe_stats)
+dsmoe_status launch_stats(const dsmoe_layer_desc& p, const float* scores, const uint64_t* mask,
+                          dsmoe_selection_stats* stats, cudaStream_t s);
 dsmoe_status launch_combine(const dsmoe_layer_desc& p, const void* yp, const float* row_gate,
                             const int32_t* token_rows, const int32_t* k_t, void* out, cudaStream_t s);
 dsmoe_status launch_pack(const dsmoe_layer_desc& p, const void* W1, const void* W2, void* packed,
@@ -72,9 +94,8 @@ dsmoe_status launch_mlp_generic(const dsmoe_layer_desc& p, const void* xp, const
 
 
 // ---- mlp_umma.cu : tcgen05 / TMEM / TMA kernels on packed bf16 weights
-void timing_reset();
-dsmoe_status timing_enable(int on);
-dsmoe_status timing_last(float* ms, int n_max, int* n);
+dsmoe_status timing_enable(int n_pairs);
+dsmoe_status timing_read(float* ms, int n_max, int* n);
 bool umma_supported(const dsmoe_layer_desc& p);   // bf16, d and H multiples of 64
 // Router for many tokens with the logits on the tensor cores (bf16 x; Wr split exactly into three bf16 terms, fp32
 // accumulation), then softmax and selection.  `scratch` holds router_umma_scratch(p) bytes.
@@ -85,9 +106,19 @@ dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const 
                                 cudaStream_t s);
 // Grouped expert MLPs on expert-sorted rows: h = GeLU(xp.W1[e]) (bf16, in `hbuf`), yp = h.W2[e].
 // With row_token (and x), the up-projection gathers its rows from x by index and xp is not read.
+// With cmb, the down-projection's epilogue also aggregates (Eq. 1's weighted sum, ascending expert order per token):
+// it writes the layer output cmb->out [T,d] and yp is not touched.
+struct CombineArgs {
+    const int32_t* row_token;
+    const float* row_gate;
+    const uint64_t* mask;
+    float* acc;          // fp32 [T,d] running sums (unused when the output itself is fp32)
+    int* tile_done;      // E * ceil(d / 256) ints
+    void* out;
+};
 dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,
                              void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s, const void* x = nullptr,
-                             const int32_t* row_token = nullptr);
+                             const int32_t* row_token = nullptr, const CombineArgs* cmb = nullptr);
 // Whole-layer paths that need no grouping (all experts selected, or few tokens).  *done = false
 // means "not taken": the caller continues with the grouped path.
 // Whole layer for few tokens (T <= 128) in one cooperative launch, router included.

@@ -18,6 +18,8 @@
 #include "router_device.cuh"
 #include "umma.cuh"
 
+#include <stdlib.h>
+
 namespace dsmoe {
 
 namespace {
@@ -44,7 +46,7 @@ constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)SMALL_RING_BYTE
 constexpr size_t SMEM_GEMM_BYTES = 1024 + (size_t)RING_BYTES + SHARED_BYTES;   // umma_gemm_kernel needs no staging tile
 
 enum { GEMM_GROUPED = 0, GEMM_DENSE_UP = 1, GEMM_DENSE_DOWN = 2 };
-enum { EPI_GELU = 0, EPI_STORE = 1 };
+enum { EPI_GELU = 0, EPI_STORE = 1, EPI_COMBINE = 2 };
 constexpr int kUpUnit = 16;          // small-T up-projection: weight rows per work unit
 constexpr int kUpTileUnits = 16;     // ... and units per tile (256 rows)
 constexpr int kRouterBatch = 12;     // rows of Wr a router thread loads at once
@@ -77,6 +79,16 @@ struct GemmParams {
     const int32_t* gather;
     const void* gather_src;
     int gather_rows;
+    // grouped down-projection with the aggregation of Eq. 1 in its epilogue (epi == EPI_COMBINE): row r belongs to
+    // token row_token[r] and carries the router gate row_gate[r]; the epilogue adds gate * (h.W2[e]) to the token's
+    // fp32 running sum `acc` [tokens, n_per_expert] in ascending expert order (tile_done orders the experts), and the
+    // token's last expert writes the rounded result to `out`.  With out_f32 the sum runs in `out` itself.
+    const int32_t* row_token;
+    const float* row_gate;
+    const uint64_t* sel_mask;
+    float* acc;
+    int* tile_done;          // [E][column ranges], zero at launch: epilogue warps that have finished a tile
+    int tokens;
 };
 
 // Tensor maps of one packed weight tensor [E, n, k] with boxes of 16, 32, 64, 128 and 256 rows: a tile of
@@ -202,6 +214,26 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& P, const Shared& s
     }
     t.bn = min(BN, P.n_per_expert - t.n0);
     return t;
+}
+
+// Bounded wait until the int at `flag` (written by other CTAs with a release fence before it) is at least
+// `target`.  false = gave up (limit reached, or another thread of the CTA already had).
+__device__ __forceinline__ bool flag_wait_ge(const int* flag, int target, volatile int* abort_flag) {
+    uint64_t t0 = 0;
+    for (uint32_t spin = 1;; ++spin) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v >= target) return true;
+        if ((spin & 0x3f) == 0) {
+            if (*abort_flag) return false;
+            const uint64_t now = ptx::globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > ptx::kWaitLimitNs) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
 }
 
 __global__ void __launch_bounds__(GATHER_THREADS, 1)
@@ -404,6 +436,86 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (P.gate && valid) g = P.gate[grow * P.E + t.e];
             const uint32_t taddr = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
             const bool warp_has_rows = q * 32 < t.rows_valid;   // warps without a valid row skip the read-back
+            if (P.epi == EPI_COMBINE) {
+                // Aggregation fused into the down-projection.  A token's experts add their outputs to its running
+                // sum one after the other, lowest expert first -- the order of the separate aggregation kernel, so
+                // the result is the same bit for bit and run to run.  That order holds because this tile only
+                // touches the sums once every tile of the previous non-empty expert that covers the same columns has
+                // finished (tiles are handed out in ascending expert order to CTAs that are all resident: the
+                // wait is for work that is already running or done).
+                const int ntn = (P.n_per_expert + BN - 1) / BN, nt = t.n0 / BN;
+                int prev = t.e - 1;
+                while (prev >= 0 && sh.seg1[prev] <= sh.seg0[prev]) --prev;
+                bool ok = true;
+                if (prev >= 0 && warp_has_rows) {
+                    if (lane == 0) {
+                        const int target = 4 * ((sh.seg1[prev] - sh.seg0[prev] + BM - 1) / BM);
+                        ok = flag_wait_ge(P.tile_done + prev * ntn + nt, target, &sh.abort_flag);
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                }
+                if (!ok) break;
+                int tok = 0;
+                float g = 0.f;
+                bool first = true, last = true;
+                if (valid) {
+                    tok = min(max(P.row_token[grow], 0), P.tokens - 1);
+                    g = P.row_gate[grow];
+                    const uint64_t m = P.sel_mask[tok];
+                    first = (m & ((1ull << t.e) - 1ull)) == 0ull;
+                    last = ((m >> t.e) >> 1) == 0ull;
+                }
+                float* arow = P.acc + (long long)tok * P.n_per_expert + t.out_col0;
+                for (int c = 0; warp_has_rows && c < t.bn; c += 32) {
+                    float4 old[8];
+                    if (valid && !first) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) old[j] = __ldcg(reinterpret_cast<const float4*>(arow + c) + j);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) old[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    uint32_t r[32];
+                    ptx::tmem_ld32(taddr + (uint32_t)c, r);
+                    ptx::tmem_ld_wait();
+                    if (!valid) continue;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        old[j].x = fmaf(g, __uint_as_float(r[4 * j]), old[j].x);
+                        old[j].y = fmaf(g, __uint_as_float(r[4 * j + 1]), old[j].y);
+                        old[j].z = fmaf(g, __uint_as_float(r[4 * j + 2]), old[j].z);
+                        old[j].w = fmaf(g, __uint_as_float(r[4 * j + 3]), old[j].w);
+                    }
+                    if (last && !P.out_f32) {
+                        uint4 pk[4];
+                        __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            hv[2 * j] = __floats2bfloat162_rn(old[j].x, old[j].y);
+                            hv[2 * j + 1] = __floats2bfloat162_rn(old[j].z, old[j].w);
+                        }
+                        uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) +
+                                                              (long long)tok * P.ld_out + t.out_col0 + c);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) dst[j] = pk[j];
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) __stcg(reinterpret_cast<float4*>(arow + c) + j, old[j]);
+                    }
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    ptx::mbar_arrive(ptx::smem_u32(&sh.tempty[acc]));
+                    __threadfence();                       // the warp's sums are visible before its arrival is
+                    atomicAdd(P.tile_done + t.e * ntn + nt, 1);
+                }
+                if (++acc == 2) {
+                    acc = 0;
+                    aph ^= 1u;
+                }
+                continue;
+            }
             for (int c = 0; warp_has_rows && c < t.bn; c += 32) {
                 uint32_t r[32];
                 ptx::tmem_ld32(taddr + (uint32_t)c, r);
@@ -1474,35 +1586,105 @@ dsmoe_status make_bmaps(BMaps* b, const void* ptr, uint64_t E, uint64_t n, uint6
 }
 
 int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    }
-    return n;
+    DeviceState* st = nullptr;
+    return device_state(&st) == DSMOE_OK ? st->sm_count : 148;   // no device (host-only sizing): the B200's count
 }
 
-// Optional per-launch timing of the tensor-core kernels (a measurement aid for benchmarks): event pairs
-// around each launch of the most recent call.
-constexpr int kMaxTimed = 8;
+// Tensor maps depend only on the buffer and the shape, and encoding one is a driver call of a few microseconds
+// (a layer call needs up to 23): they are encoded once and found again by (address, shape).  A decode loop or a
+// serving loop calls with the same buffers every step.  Not thread-safe, like the rest of the host side.
+struct MapKey {
+    const void* ptr;
+    uint64_t a, b, c;
+    int kind;
+    bool operator==(const MapKey& o) const { return ptr == o.ptr && a == o.a && b == o.b && c == o.c && kind == o.kind; }
+};
+template <typename M, int N>
+struct MapCache {
+    MapKey key[N];
+    M map[N];
+    int n = 0, next = 0;
+    M* find(const MapKey& k) {
+        for (int i = 0; i < n; ++i)
+            if (key[i] == k) return &map[i];
+        return nullptr;
+    }
+    M* slot(const MapKey& k) {
+        const int i = n < N ? n++ : (next++ % N);
+        key[i] = k;
+        return &map[i];
+    }
+};
+MapCache<CUtensorMap, 256> g_maps2d;
+MapCache<BMaps, 128> g_bmaps;
+MapCache<BMaps16, 64> g_bmaps16;
+
+dsmoe_status cached_map_2d(const CUtensorMap** out, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    const MapKey k{ptr, rows, cols, box_rows, 0};
+    CUtensorMap* m = g_maps2d.find(k);
+    if (!m) {
+        CUtensorMap tmp;
+        DSMOE_TRY(make_map_2d(&tmp, ptr, rows, cols, box_rows));
+        m = g_maps2d.slot(k);
+        *m = tmp;
+    }
+    *out = m;
+    return DSMOE_OK;
+}
+dsmoe_status cached_bmaps(const BMaps** out, const void* ptr, uint64_t E, uint64_t n, uint64_t kk) {
+    const MapKey k{ptr, E, n, kk, 1};
+    BMaps* m = g_bmaps.find(k);
+    if (!m) {
+        BMaps tmp;
+        DSMOE_TRY(make_bmaps(&tmp, ptr, E, n, kk));
+        m = g_bmaps.slot(k);
+        *m = tmp;
+    }
+    *out = m;
+    return DSMOE_OK;
+}
+dsmoe_status cached_bmaps16(const BMaps16** out, const void* ptr, uint64_t E, uint64_t n, uint64_t kk) {
+    const MapKey k{ptr, E, n, kk, 2};
+    BMaps16* m = g_bmaps16.find(k);
+    if (!m) {
+        BMaps16 tmp;
+        DSMOE_TRY(make_bmaps16(&tmp, ptr, E, n, kk));
+        m = g_bmaps16.slot(k);
+        *m = tmp;
+    }
+    *out = m;
+    return DSMOE_OK;
+}
+
+// Optional per-launch timing of the tensor-core kernels (a measurement aid for benchmarks): a ring of CUDA event
+// pairs; every timed launch takes the next pair until the ring is full.  The events sit on the caller's stream, so a
+// benchmark can leave them inside its un-synchronised step loop and read all durations afterwards.
 struct Timing {
-    bool on = false, made = false;
-    int n = 0;
-    cudaEvent_t start[kMaxTimed], stop[kMaxTimed];
+    bool on = false;
+    int n = 0, cap = 0;
+    cudaEvent_t *start = nullptr, *stop = nullptr;
 } g_timing;
 
 dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams& P, int grid, cudaStream_t s,
                          bool may_time = true) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    DeviceState* st = nullptr;
+    DSMOE_TRY(device_state(&st));
+    if (!st->attr_gemm) {
         DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_BYTES));
-        attr_set = true;
+        st->attr_gemm = true;
     }
-    const bool timed = may_time && g_timing.on && g_timing.n < kMaxTimed;
+    const bool timed = may_time && g_timing.on && g_timing.n < g_timing.cap;
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
-    umma_gemm_kernel<<<grid, P.gather ? GATHER_THREADS : NUM_THREADS, SMEM_GEMM_BYTES, s>>>(a, b, P);
-    DSMOE_CUDA_TRY(cudaGetLastError());
+    const int threads = P.gather ? GATHER_THREADS : NUM_THREADS;
+    if (P.epi == EPI_COMBINE) {
+        // its epilogues wait for one another's tiles: every CTA must be resident
+        void* args[] = {const_cast<CUtensorMap*>(&a), const_cast<BMaps*>(&b), const_cast<GemmParams*>(&P)};
+        DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(umma_gemm_kernel), dim3(grid), dim3(threads),
+                                                   args, SMEM_GEMM_BYTES, s));
+    } else {
+        umma_gemm_kernel<<<grid, threads, SMEM_GEMM_BYTES, s>>>(a, b, P);
+        DSMOE_CUDA_TRY(cudaGetLastError());
+    }
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.stop[g_timing.n++], s));
     return DSMOE_OK;
 }
@@ -1565,13 +1747,15 @@ dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const 
     float* sums = reinterpret_cast<float*>(scratch + split_bytes);
     router_split_kernel<<<ceil_div(EP * p.d, 256), 256, 0, s>>>(Wr, wsplit, p.d, p.E, EP);
     DSMOE_CUDA_TRY(cudaGetLastError());
-    CUtensorMap mA;
-    BMaps mB;
-    DSMOE_TRY(make_map_2d(&mA, x, p.T, p.d, BM));
-    DSMOE_TRY(make_bmaps(&mB, wsplit, 1, 3 * EP, p.d));
-    GemmParams g{GEMM_DENSE_DOWN, EPI_STORE, 1, 3 * EP, p.d, p.T, nullptr, nullptr, sums, 3 * EP, 1, dev_status};
+    const CUtensorMap* mA;
+    const BMaps* mB;
+    DSMOE_TRY(cached_map_2d(&mA, x, p.T, p.d, BM));
+    DSMOE_TRY(cached_bmaps(&mB, wsplit, 1, 3 * EP, p.d));
+    GemmParams g{};
+    g.mode = GEMM_DENSE_DOWN; g.epi = EPI_STORE; g.E = 1; g.n_per_expert = 3 * EP; g.k_per_expert = p.d; g.rows = p.T;
+    g.out = sums; g.ld_out = 3 * EP; g.out_f32 = 1; g.dev_status = dev_status;
     const int tiles = ceil_div(p.T, BM);
-    DSMOE_TRY(launch_gemm(mA, mB, g, tiles < sm_count() ? tiles : sm_count(), s, false));
+    DSMOE_TRY(launch_gemm(*mA, *mB, g, tiles < sm_count() ? tiles : sm_count(), s, false));
     router_finish_kernel<<<ceil_div(p.T, 8), 256, 0, s>>>(sums, br, scores, mask, k_t, p.T, EP,
                                                          SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k, nullptr});
     DSMOE_CUDA_TRY(cudaGetLastError());
@@ -1584,29 +1768,32 @@ extern "C" __attribute__((visibility("default"))) int dsmoe_trace_read(unsigned 
 }
 #endif
 
-void timing_reset() { g_timing.n = 0; }
-
-dsmoe_status timing_enable(int on) {
-    if (on && !g_timing.made) {
-        for (int i = 0; i < kMaxTimed; ++i) {
+dsmoe_status timing_enable(int n_pairs) {
+    if (n_pairs > g_timing.cap) {
+        cudaEvent_t* a = static_cast<cudaEvent_t*>(realloc(g_timing.start, sizeof(cudaEvent_t) * n_pairs));
+        cudaEvent_t* b = static_cast<cudaEvent_t*>(realloc(g_timing.stop, sizeof(cudaEvent_t) * n_pairs));
+        if (a) g_timing.start = a;
+        if (b) g_timing.stop = b;
+        if (!a || !b) return DSMOE_ERR_CUDA;
+        for (int i = g_timing.cap; i < n_pairs; ++i) {
             DSMOE_CUDA_TRY(cudaEventCreate(&g_timing.start[i]));
             DSMOE_CUDA_TRY(cudaEventCreate(&g_timing.stop[i]));
+            g_timing.cap = i + 1;
         }
-        g_timing.made = true;
     }
-    g_timing.on = on != 0;
+    g_timing.on = n_pairs > 0;
     g_timing.n = 0;
     return DSMOE_OK;
 }
 
-dsmoe_status timing_last(float* ms, int n_max, int* n) {
+dsmoe_status timing_read(float* ms, int n_max, int* n) {
     *n = 0;
-    if (!g_timing.on) return DSMOE_OK;
     for (int i = 0; i < g_timing.n && i < n_max; ++i) {
         DSMOE_CUDA_TRY(cudaEventSynchronize(g_timing.stop[i]));
         DSMOE_CUDA_TRY(cudaEventElapsedTime(&ms[i], g_timing.start[i], g_timing.stop[i]));
         *n = i + 1;
     }
+    g_timing.n = 0;
     return DSMOE_OK;
 }
 
@@ -1616,27 +1803,44 @@ bool umma_supported(const dsmoe_layer_desc& p) {
 
 dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,
                              void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s, const void* x,
-                             const int32_t* row_token) {
+                             const int32_t* row_token, const CombineArgs* cmb) {
     if (p.T == 0) return DSMOE_OK;
     if (!umma_supported(p)) return DSMOE_ERR_UNSUPPORTED;
     const size_t amax = amax_of(p);
     const __nv_bfloat16* w1t = static_cast<const __nv_bfloat16*>(packed);
     const __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
-    CUtensorMap mA1, mA2;
-    BMaps mB1, mB2;
+    const CUtensorMap *mA1, *mA2;
+    const BMaps *mB1, *mB2;
     // with row_token, the up-projection fetches its rows straight from x (no grouped copy of the tokens); its A
     // tensor map is then unused, any valid one will do
-    DSMOE_TRY(make_map_2d(&mA1, row_token ? hbuf : xp, amax, row_token ? p.H : p.d, BM));
-    DSMOE_TRY(make_bmaps(&mB1, w1t, p.E, p.H, p.d));
-    DSMOE_TRY(make_map_2d(&mA2, hbuf, amax, p.H, BM));
-    DSMOE_TRY(make_bmaps(&mB2, w2t, p.E, p.d, p.H));
-    GemmParams up{GEMM_GROUPED, EPI_GELU, p.E, p.H, p.d, (int)amax, offsets, nullptr, hbuf, p.H, 0, dev_status};
+    DSMOE_TRY(cached_map_2d(&mA1, row_token ? hbuf : xp, amax, row_token ? p.H : p.d, BM));
+    DSMOE_TRY(cached_bmaps(&mB1, w1t, p.E, p.H, p.d));
+    DSMOE_TRY(cached_map_2d(&mA2, hbuf, amax, p.H, BM));
+    DSMOE_TRY(cached_bmaps(&mB2, w2t, p.E, p.d, p.H));
+    GemmParams up{};
+    up.mode = GEMM_GROUPED; up.epi = EPI_GELU; up.E = p.E; up.n_per_expert = p.H; up.k_per_expert = p.d;
+    up.rows = (int)amax; up.offsets = offsets; up.out = hbuf; up.ld_out = p.H; up.dev_status = dev_status;
     up.gather = row_token;
     up.gather_src = x;
     up.gather_rows = p.T;
-    GemmParams down{GEMM_GROUPED, EPI_STORE, p.E, p.d, p.H, (int)amax, offsets, nullptr, yp, p.d, 0, dev_status};
-    DSMOE_TRY(launch_gemm(mA1, mB1, up, sm_count(), s));
-    DSMOE_TRY(launch_gemm(mA2, mB2, down, sm_count(), s));
+    GemmParams down{};
+    down.mode = GEMM_GROUPED; down.epi = EPI_STORE; down.E = p.E; down.n_per_expert = p.d; down.k_per_expert = p.H;
+    down.rows = (int)amax; down.offsets = offsets; down.out = yp; down.ld_out = p.d; down.dev_status = dev_status;
+    if (cmb) {
+        // Eq. 1's weighted sum inside the down-projection's epilogue: no expert-output buffer, no aggregation pass
+        down.epi = EPI_COMBINE;
+        down.out = cmb->out;
+        down.out_f32 = p.out_fp32 ? 1 : 0;
+        down.row_token = cmb->row_token;
+        down.row_gate = cmb->row_gate;
+        down.sel_mask = cmb->mask;
+        down.acc = p.out_fp32 ? static_cast<float*>(cmb->out) : cmb->acc;
+        down.tile_done = cmb->tile_done;
+        down.tokens = p.T;
+        DSMOE_CUDA_TRY(cudaMemsetAsync(cmb->tile_done, 0, (size_t)p.E * ceil_div(p.d, BN) * sizeof(int), s));
+    }
+    DSMOE_TRY(launch_gemm(*mA1, *mB1, up, sm_count(), s));
+    DSMOE_TRY(launch_gemm(*mA2, *mB2, down, sm_count(), s));
     return DSMOE_OK;
 }
 
@@ -1655,47 +1859,24 @@ bool small_supported(const dsmoe_layer_desc& p) {
 dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
                                 const void* packed, float* scores, uint64_t* mask, int32_t* k_t, int32_t* counts_out,
                                 void* out, char* ws, const WsLayout& L, int32_t* dev_status, cudaStream_t s) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    DeviceState* st = nullptr;
+    DSMOE_TRY(device_state(&st));
+    if (!st->attr_small) {
         DSMOE_CUDA_TRY(cudaFuncSetAttribute(small_layer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-        attr_set = true;
+        st->attr_small = true;
     }
     const __nv_bfloat16* w1t = static_cast<const __nv_bfloat16*>(packed);
     const __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
     const int t_pad = (p.T + 7) / 8 * 8;
     int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
     void* hg = ws + L.h;
-    // The 23 tensor maps of a call depend only on the buffers and the shape: encoded once, then reused
-    // (decode loops call with the same buffers every step).  Not thread-safe, like the timing aid.
-    struct MapSet {
-        const void *x, *hg, *packed;
-        int T, d, H, E;
-        CUtensorMap mX, mHg;
-        BMaps16 mW1;
-        BMaps mW2;
-    };
-    constexpr int kCache = 64;
-    static MapSet cache[kCache];
-    static int n_cached = 0, next_slot = 0;
-    MapSet* ms = nullptr;
-    for (int i = 0; i < n_cached; ++i) {
-        MapSet& c = cache[i];
-        if (c.x == x && c.hg == hg && c.packed == packed && c.T == p.T && c.d == p.d && c.H == p.H && c.E == p.E) {
-            ms = &c;
-            break;
-        }
-    }
-    if (!ms) {
-        MapSet c;
-        c.x = x; c.hg = hg; c.packed = packed; c.T = p.T; c.d = p.d; c.H = p.H; c.E = p.E;
-        DSMOE_TRY(make_map_2d(&c.mX, x, p.T, p.d, t_pad));
-        DSMOE_TRY(make_bmaps16(&c.mW1, w1t, p.E, p.H, p.d));
-        DSMOE_TRY(make_map_2d(&c.mHg, hg, p.T, (uint64_t)p.E * p.H, t_pad));
-        DSMOE_TRY(make_bmaps(&c.mW2, w2t, p.E, p.d, p.H));
-        const int slot = n_cached < kCache ? n_cached++ : (next_slot++ % kCache);
-        cache[slot] = c;
-        ms = &cache[slot];
-    }
+    const CUtensorMap *mX, *mHg;
+    const BMaps16* mW1;
+    const BMaps* mW2;
+    DSMOE_TRY(cached_map_2d(&mX, x, p.T, p.d, t_pad));
+    DSMOE_TRY(cached_bmaps16(&mW1, w1t, p.E, p.H, p.d));
+    DSMOE_TRY(cached_map_2d(&mHg, hg, p.T, (uint64_t)p.E * p.H, t_pad));
+    DSMOE_TRY(cached_bmaps(&mW2, w2t, p.E, p.d, p.H));
     SmallParams P;
     P.T = p.T; P.d = p.d; P.H = p.H; P.E = p.E; P.t_pad = t_pad;
     P.x = static_cast<const __nv_bfloat16*>(x);
@@ -1712,12 +1893,13 @@ dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const 
     P.out_f32 = p.out_fp32 ? 1 : 0;
     P.sync = reinterpret_cast<int*>(ws + L.sync);
     P.dev_status = dev_status;
-    // With 16 tokens or more it is rare that an expert is selected by none of them, so the kernel starts the
+    // From kSpecMinT tokens on it is rare that an expert is selected by none of them, so the kernel starts the
     // up-projection under that assumption while its router is still running; it starts over if the router disagrees.
     P.spec = p.T >= kSpecMinT ? 1 : 0;
     DSMOE_CUDA_TRY(cudaMemsetAsync(P.sync, 0, 32, s));
-    void* args[] = {&ms->mX, &ms->mW1, &ms->mHg, &ms->mW2, &P};
-    const bool timed = g_timing.on && g_timing.n < kMaxTimed;
+    void* args[] = {const_cast<CUtensorMap*>(mX), const_cast<BMaps16*>(mW1), const_cast<CUtensorMap*>(mHg),
+                    const_cast<BMaps*>(mW2), &P};
+    const bool timed = g_timing.on && g_timing.n < g_timing.cap;
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
     DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(small_layer_kernel), dim3(G), dim3(SMALL_THREADS),
                                                args, SMEM_BYTES, s));
@@ -1735,19 +1917,22 @@ dsmoe_status launch_layer_umma(const dsmoe_layer_desc& p, const void* x, const v
     const __nv_bfloat16* w1t = static_cast<const __nv_bfloat16*>(packed);
     const __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
     void* hg = ws + L.h;                                        // [T, E*H] bf16
-    CUtensorMap mA1, mA2;
-    BMaps mB1, mB2;
-    DSMOE_TRY(make_map_2d(&mA1, x, p.T, p.d, BM));
-    DSMOE_TRY(make_bmaps(&mB1, w1t, p.E, p.H, p.d));
-    DSMOE_TRY(make_map_2d(&mA2, hg, p.T, (uint64_t)p.E * p.H, BM));
-    DSMOE_TRY(make_bmaps(&mB2, w2t, p.E, p.d, p.H));
-    const int out_f32 = p.out_fp32 ? 1 : 0;
-    GemmParams up{GEMM_DENSE_UP, EPI_GELU, p.E, p.H, p.d, p.T, nullptr, scores, hg, (long long)p.E * p.H, 0, dev_status};
-    GemmParams down{GEMM_DENSE_DOWN, EPI_STORE, p.E, p.d, p.H, p.T, nullptr, nullptr, out, p.d, out_f32, dev_status};
+    const CUtensorMap *mA1, *mA2;
+    const BMaps *mB1, *mB2;
+    DSMOE_TRY(cached_map_2d(&mA1, x, p.T, p.d, BM));
+    DSMOE_TRY(cached_bmaps(&mB1, w1t, p.E, p.H, p.d));
+    DSMOE_TRY(cached_map_2d(&mA2, hg, p.T, (uint64_t)p.E * p.H, BM));
+    DSMOE_TRY(cached_bmaps(&mB2, w2t, p.E, p.d, p.H));
+    GemmParams up{};
+    up.mode = GEMM_DENSE_UP; up.epi = EPI_GELU; up.E = p.E; up.n_per_expert = p.H; up.k_per_expert = p.d; up.rows = p.T;
+    up.gate = scores; up.out = hg; up.ld_out = (long long)p.E * p.H; up.dev_status = dev_status;
+    GemmParams down{};
+    down.mode = GEMM_DENSE_DOWN; down.epi = EPI_STORE; down.E = p.E; down.n_per_expert = p.d; down.k_per_expert = p.H;
+    down.rows = p.T; down.out = out; down.ld_out = p.d; down.out_f32 = p.out_fp32 ? 1 : 0; down.dev_status = dev_status;
     const int mt = ceil_div(p.T, BM);
     const int tiles_up = mt * ceil_div(p.H, BN) * p.E, tiles_down = mt * ceil_div(p.d, BN);
-    DSMOE_TRY(launch_gemm(mA1, mB1, up, tiles_up < sm_count() ? tiles_up : sm_count(), s));
-    DSMOE_TRY(launch_gemm(mA2, mB2, down, tiles_down < sm_count() ? tiles_down : sm_count(), s));
+    DSMOE_TRY(launch_gemm(*mA1, *mB1, up, tiles_up < sm_count() ? tiles_up : sm_count(), s));
+    DSMOE_TRY(launch_gemm(*mA2, *mB2, down, tiles_down < sm_count() ? tiles_down : sm_count(), s));
     if (counts_out) {
         int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
         int32_t* offsets = reinterpret_cast<int32_t*>(ws + L.offsets);

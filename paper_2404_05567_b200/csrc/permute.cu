@@ -14,7 +14,7 @@ __global__ void __launch_bounds__(256) permute_index_kernel(const uint64_t* __re
                                                             const int32_t* __restrict__ chunk_prefix,
                                                             int32_t* __restrict__ row_token, float* __restrict__ row_gate,
                                                             int32_t* __restrict__ token_rows, int T, int E, int W,
-                                                            int64_t amax) {
+                                                            int64_t amax, uint4* __restrict__ zero_out, int row_vecs) {
     const int lane = threadIdx.x & 31;
     const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (c * kChunk >= T) return;
@@ -36,6 +36,16 @@ __global__ void __launch_bounds__(256) permute_index_kernel(const uint64_t* __re
     }
     if (t < T)
         for (; slot < W; ++slot) token_rows[(size_t)t * W + slot] = -1;
+    if (zero_out) {
+        // Eq. 1 with an empty selection is the zero vector: no expert tile will ever write this token's row
+        unsigned none = __ballot_sync(0xffffffffu, t < T && m == 0);
+        while (none) {
+            const int l = __ffs(none) - 1;
+            none &= none - 1;
+            uint4* row = zero_out + (size_t)(c * kChunk + l) * row_vecs;
+            for (int v = lane; v < row_vecs; v += 32) row[v] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
 }
 
 // xp[r,:] = x[row_token[r],:] for r < A, 16 bytes per lane per step, one warp per row.
@@ -160,12 +170,14 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
 
 dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const float* scores, const uint64_t* mask,
                             const int32_t* offsets, const int32_t* chunk_prefix, int32_t* row_token, float* row_gate,
-                            int32_t* token_rows, void* xp, cudaStream_t s) {
+                            int32_t* token_rows, void* xp, cudaStream_t s, void* zero_out) {
     if (p.T == 0) return DSMOE_OK;
     const int nchunks = ceil_div(p.T, kChunk);
     const int64_t amax = (int64_t)amax_of(p);
+    const int row_vecs = (int)((size_t)p.d * (p.out_fp32 ? 4 : elem_size(p.dtype)) / 16);
     permute_index_kernel<<<ceil_div(nchunks, 8), 256, 0, s>>>(mask, scores, offsets, chunk_prefix, row_token, row_gate,
-                                                             token_rows, p.T, p.E, width_of(p), amax);
+                                                             token_rows, p.T, p.E, width_of(p), amax,
+                                                             static_cast<uint4*>(zero_out), row_vecs);
     DSMOE_CUDA_TRY(cudaGetLastError());
     if (xp) {
         const int vec_per_row = (int)((size_t)p.d * elem_size(p.dtype) / 16);
@@ -193,6 +205,65 @@ dsmoe_status launch_combine(const dsmoe_layer_desc& p, const void* yp, const flo
         combine_f32_kernel<<<p.T, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t,
                                                static_cast<float4*>(out), p.d, W, amax);
     }
+    DSMOE_CUDA_TRY(cudaGetLastError());
+    return DSMOE_OK;
+}
+
+// Selection statistics.  One warp per token; integer atomics only, so the counts do not depend on the order.
+__global__ void __launch_bounds__(256) stats_kernel(const float* __restrict__ scores, const uint64_t* __restrict__ mask,
+                                                    dsmoe_selection_stats* __restrict__ st, int T, int E, int mode, float eps,
+                                                    int eps_normalized) {
+    __shared__ int cnt_s[kMaxExperts];
+    __shared__ unsigned long long near_s, a_s;
+    __shared__ int zero_s;
+    if (threadIdx.x < kMaxExperts) cnt_s[threadIdx.x] = 0;
+    if (threadIdx.x == 0) {
+        near_s = 0ull;
+        a_s = 0ull;
+        zero_s = 0;
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const bool thr = mode == DSMOE_SELECT_THRESHOLD || mode == DSMOE_SELECT_THRESHOLD_TOPK;
+    for (int t = blockIdx.x * 8 + (threadIdx.x >> 5); t < T; t += gridDim.x * 8) {
+        const uint64_t m = mask[t];
+        if (lane == 0) {
+            atomicAdd(&a_s, (unsigned long long)__popcll(m));
+            if (m == 0) atomicAdd(&zero_s, 1);
+        }
+        for (int e = lane; e < E; e += 32) {
+            if ((m >> e) & 1ull) atomicAdd(&cnt_s[e], 1);
+            if (thr) {
+                const float sc = scores[(size_t)t * E + e];
+                const float v = eps_normalized ? __fmul_rn(sc, (float)E) : sc;   // the value the rule compares
+                if (fabs((double)v - (double)eps) <= 1e-6) atomicAdd(&near_s, 1ull);
+            }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < E && cnt_s[threadIdx.x]) atomicAdd(&st->counts[threadIdx.x], cnt_s[threadIdx.x]);
+    if (threadIdx.x == 0) {
+        atomicAdd(reinterpret_cast<unsigned long long*>(&st->assignments), a_s);
+        atomicAdd(reinterpret_cast<unsigned long long*>(&st->near_threshold), near_s);
+        atomicAdd(&st->zero_tokens, zero_s);
+    }
+}
+
+__global__ void stats_finish_kernel(dsmoe_selection_stats* st, int E) {
+    int n = 0;
+    for (int e = 0; e < E; ++e) n += st->counts[e] == 0;
+    st->empty_experts = n;
+}
+
+dsmoe_status launch_stats(const dsmoe_layer_desc& p, const float* scores, const uint64_t* mask,
+                          dsmoe_selection_stats* stats, cudaStream_t s) {
+    DSMOE_CUDA_TRY(cudaMemsetAsync(stats, 0, sizeof(dsmoe_selection_stats), s));
+    if (p.T > 0) {
+        const int grid = ceil_div(p.T, 8) < 1184 ? ceil_div(p.T, 8) : 1184;
+        stats_kernel<<<grid, 256, 0, s>>>(scores, mask, stats, p.T, p.E, p.mode, p.eps, p.eps_normalized);
+        DSMOE_CUDA_TRY(cudaGetLastError());
+    }
+    stats_finish_kernel<<<1, 1, 0, s>>>(stats, p.E);
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
 }

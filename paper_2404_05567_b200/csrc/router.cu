@@ -338,7 +338,9 @@ static dsmoe_status launch_router_t(const dsmoe_layer_desc& p, const XT* x, cons
         else router_small_kernel<XT, 64><<<p.T, 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.d, q);
     } else {
         const int grid = ceil_div(p.T, kRtTB);
-        static bool attr_set = false;     // per instantiation (XT)
+        DeviceState* st = nullptr;
+        DSMOE_TRY(device_state(&st));
+        bool& attr_set = sizeof(XT) == 4 ? st->attr_router_f32 : st->attr_router_bf16;
         if (!attr_set) {
             DSMOE_CUDA_TRY(cudaFuncSetAttribute(router_tile_kernel<XT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 (int)router_tile_smem<4>()));

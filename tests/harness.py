@@ -2,6 +2,9 @@
 through the binding, fetch results as numpy, and compare with the CPU oracle."""
 from __future__ import annotations
 
+import json
+import os
+
 import numpy as np
 import torch
 
@@ -12,6 +15,17 @@ import paper_2404_05567_b200 as dm
 TOL_BF16 = 2e-2      # max|gpu - oracle| <= 2e-2 * RMS(oracle)   (bf16 storage, fp32 accumulate)
 TOL_F32 = 1e-4       # max|gpu - oracle| <= 1e-4 * RMS(oracle)   (fp32)
 NEAR = 1e-6          # scores this close to a decision boundary may legitimately flip
+
+
+def record(kind: str, **fields):
+    """Puts a measured figure on record: printed (pytest shows it with -s or on failure) and, when the
+    environment variable DSMOE_PARITY_LOG names a file, appended there as one JSON line."""
+    line = dict(kind=kind, **fields)
+    print("[dsmoe]", json.dumps(line))
+    path = os.environ.get("DSMOE_PARITY_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps(line) + "\n")
 
 
 def to_dev(a: np.ndarray) -> torch.Tensor:
@@ -55,11 +69,13 @@ class Layer:
         self.W1, self.W2 = gi.experts(s, layer)
         self.x_d, self.Wr_d, self.br_d = to_dev(self.x), to_dev(self.Wr), to_dev(self.br)
         self.W1_d, self.W2_d = to_dev(self.W1), to_dev(self.W2)
-        self.ws = torch.empty(dm.dsmoe_workspace_size(self.desc), dtype=torch.uint8, device="cuda")
         self.packed = None
         if pack and s.dtype == "bf16" and s.d % 64 == 0 and s.H % 64 == 0:      # the packed layout is in blocks of 64
             self.packed = torch.empty(dm.dsmoe_packed_size(self.desc), dtype=torch.uint8, device="cuda")
             dm.dsmoe_pack_weights(self.desc, self.W1_d, self.W2_d, self.packed)
+        # a call with packed weights needs only the tensor-core paths' (smaller) workspace
+        nbytes = dm.dsmoe_workspace_size_packed(self.desc) if self.packed is not None else dm.dsmoe_workspace_size(self.desc)
+        self.ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         self.dev_status = torch.zeros(1, dtype=torch.int32, device="cuda")
         self.native = torch.float32 if s.dtype == "f32" else torch.bfloat16
         self.out = torch.empty((s.T, s.d), dtype=torch.float32 if s.out_fp32 else self.native, device="cuda")
@@ -163,10 +179,22 @@ def layer_parity(s: gi.LayerSpec, pack: bool = True, sample: int | None = None):
     counts_from_mask = np.array([int(((mask_gpu >> np.uint64(e)) & np.uint64(1)).sum()) for e in range(s.E)])
     assert np.array_equal(counts_gpu, counts_from_mask)
     ids = None if sample is None or sample >= s.T else gi.sample_tokens(s, sample)
+    if ids is not None:
+        # the compared tokens must reach every expert that any token selected: where the seeded sample misses
+        # one, the first token that selected it joins the sample
+        seen = np.bitwise_or.reduce(mask_gpu[ids]) if len(ids) else np.uint64(0)
+        missing = int(np.bitwise_or.reduce(mask_gpu)) & ~int(seen)
+        extra = [int(np.nonzero((mask_gpu >> np.uint64(e)) & np.uint64(1))[0][0]) for e in range(s.E) if (missing >> e) & 1]
+        if extra:
+            ids = np.unique(np.concatenate([ids, np.array(extra, dtype=ids.dtype)]))
     ref = oracle.layer(L.x, L.W1, L.W2, S, mask_gpu, token_ids=ids)
     got = out if ids is None else out[ids]
     # the tolerance is relative to the RMS of the oracle's output over the compared tokens
     err = rel_err(got, ref) if ref.size else 0.0
-    return dict(err=err, err_rows=rel_err_rows(got, ref) if ref.size else 0.0, flips=flips, near=near, A=int(counts_gpu.sum()), layer=L, ref=ref, got=got,
+    err_rows = rel_err_rows(got, ref) if ref.size else 0.0
+    record("layer_parity", name=s.name, T=s.T, d=s.d, H=s.H, E=s.E, dtype=s.dtype, mode=s.mode, eps=s.eps, K=s.K,
+           packed=bool(L.packed is not None), tokens_compared=int(ref.shape[0]), err_global=err, err_per_token=err_rows,
+           flips=flips, near_threshold=near, A=int(counts_gpu.sum()))
+    return dict(err=err, err_rows=err_rows, flips=flips, near=near, A=int(counts_gpu.sum()), layer=L, ref=ref, got=got,
                 empty_experts=int((counts_gpu == 0).sum()),
                 zero_tokens=int((mask_gpu == 0).sum()))

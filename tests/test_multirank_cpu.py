@@ -60,3 +60,18 @@ def test_two_gloo_ranks_shard_by_token_and_reduce_the_timing():
         assert n == 2 and ms == 20.0                       # max over ranks
         assert value == pytest.approx(2000 / 20e-3)        # all tokens over the slowest rank's time
         assert np.array_equal(joined, full)                # sharding by token changes nothing
+
+
+def test_bench_gpus_2_starts_two_ranks_itself():
+    """`bench.py --gpus 2` outside torchrun starts its own ranks; --rendezvous-only runs that launch path, the
+    process group (gloo here, NCCL on GPUs) and the timing reduction without any GPU work."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["CUDA_VISIBLE_DEVICES"] = ""                        # the CPU path, also on a box with GPUs
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rendezvous-only"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["n_gpus"] == 2 and line["backend"] == "gloo"
+    assert line["ms_per_step"] == 20.0 and line["value"] == pytest.approx(2000 / 20e-3)

@@ -11,6 +11,7 @@ import pytest
 import torch
 
 import dsmoe_inputs as gi
+import oracle
 import paper_2404_05567_b200 as dm
 
 pytestmark = pytest.mark.gpu
@@ -37,6 +38,14 @@ def _both(desc, S):
     torch.cuda.synchronize()
     for a, b in zip(got, ref):
         assert torch.equal(a, b)
+    # ... and both against the CPU oracle's selection and grouping of the same scores
+    S_np = S.cpu().numpy()
+    mask_ref, k_ref = oracle.select(S_np, desc.mode, desc.eps, desc.eps_normalized, desc.K, desc.min_k)
+    g = oracle.group(mask_ref, S_np, width=dm.width(desc))
+    assert np.array_equal(got[0].cpu().numpy().view(np.uint64), mask_ref)
+    assert np.array_equal(got[1].cpu().numpy(), k_ref)
+    assert np.array_equal(got[2].cpu().numpy(), g["counts"])
+    assert np.array_equal(got[3].cpu().numpy(), g["offsets"])
     return got
 
 
