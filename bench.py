@@ -38,6 +38,7 @@ PAPER_SHAPES = {"1b": (2048, 256, 6), "3b": (3072, 384, 6), "6b": (4096, 512, 4)
 WORKLOADS = {
     "c2_t1": ("c2", dict(T=1)), "c2_t8": ("c2", dict(T=8)), "c2_t32": ("c2", dict(T=32)),
     "c3": ("c3", {}), "c4": ("c4", {}),
+    "c3_fused": ("c3", dict(fuse_combine=1)),      # aggregation inside the down-projection's epilogue (see dsmoe.h)
     "c5": ("c5", dict(eps=0.01)),
     # output-token throughput as the paper measures it ("GPU Inference Analysis"): a decode loop in which layer i's
     # output is layer i+1's input, 24 distinct layers (Table tab:model_arch: N_layer = 24 .. 36); W2 is drawn 16 times
@@ -50,8 +51,8 @@ for _n, (_d, _H, _K) in PAPER_SHAPES.items():
     WORKLOADS[f"paper{_n}_prefill"] = ("c3", dict(T=8192, d=_d, H=_H, K=_K))
     WORKLOADS[f"paper{_n}_t32"] = ("c2", dict(T=32, d=_d, H=_H))
 NCU_TRAFFIC_BYTES = {}     # dram bytes per launch of the dominant kernel from the ncu captures under profiles/
-DEFAULT_STEPS = {"c3": 100, "c4": 50}
-ALSO = [("c2_t1", 500), ("c2_t8", 500), ("c3", 30), ("c4", 15)] + [(f"c5_eps{e}", 15) for e in (0.0, 0.01, 0.05, 0.1, 0.2)] + \
+DEFAULT_STEPS = {"c3": 100, "c3_fused": 100, "c4": 50}
+ALSO = [("c2_t1", 500), ("c2_t8", 500), ("c3", 30), ("c3_fused", 30), ("c4", 15)] + [(f"c5_eps{e}", 15) for e in (0.0, 0.01, 0.05, 0.1, 0.2)] + \
        [(f"paper{n}_prefill", 30) for n in PAPER_SHAPES] + [(f"paper{n}_t32", 300) for n in ("1b", "3b", "6b", "19b")] + \
        [("decode_loop_t8", 20), ("decode_loop_t32", 20)]
 METRIC = "moe_layer_tokens_per_s"
@@ -250,7 +251,8 @@ def kernels_per_step(s, decode):
     router = 3 if s.T > 256 else 1                 # split Wr, logits GEMM, softmax+select | one router kernel
     if s.mode == gi.MODE_ALL:
         return router + 2                          # up, down
-    return router + 3 + 2                          # chunk count, finalize, permute index, up, down (aggregation inside)
+    # chunk count, finalize, permute index, up, down, and the aggregation unless it runs inside the down-projection
+    return router + 3 + 2 + (0 if s.fuse_combine else 1)
 
 
 def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, sampler_index=0, graph=False):
@@ -266,7 +268,8 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
 
     cfg, kw = WORKLOADS[name]
     s = gi.spec(cfg, **kw)
-    desc = dm.make_desc(s.T, s.d, s.H, s.E, dm.BF16, s.mode, s.eps, s.eps_normalized, s.K, s.min_k, s.out_fp32)
+    desc = dm.make_desc(s.T, s.d, s.H, s.E, dm.BF16, s.mode, s.eps, s.eps_normalized, s.K, s.min_k, s.out_fp32,
+                        s.fuse_combine)
     P = peaks()
     decode = s.T <= 128
     loop = name.startswith("decode_loop")
@@ -336,12 +339,9 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
             step(0)
         run_step = lambda i, want=False: g.replay()     # noqa: E731
 
-    # ---- device-resident timed region.  The library's event pairs around the dominant kernel's launches sit in this
-    # same loop: the kernel times are those of the steps that make up `value`.
+    # ---- device-resident timed region: `value` comes from this loop, which holds nothing but the steps
     for i in range(max(warmup, 3)):
         run_step(i)
-    n_pairs = 0 if graph else steps * calls_per_step * timed_per_call
-    dm.dsmoe_timing_enable(n_pairs)
     sampler = ClockSampler(sampler_index)
     barrier()
     sampler.start()
@@ -353,9 +353,23 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
     barrier()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.finish()
-    durs = np.array(dm.dsmoe_timing_read(n_pairs)) if n_pairs else np.zeros(0)
-    dm.dsmoe_timing_enable(0)
     value, ms_total, world = job_throughput(dist, ms_total, s.T * steps)
+    # ---- the same loop once more, as un-synchronised as the first, with the library's event pairs around the
+    # dominant kernel's launches (an event pair costs a few microseconds of stream time per step, which is why it is
+    # not in the loop that gives `value`); the kernel times fit inside this loop's own step time by construction
+    n_pairs = 0 if graph else steps * calls_per_step * timed_per_call
+    durs, ms_evented = np.zeros(0), None
+    if n_pairs:
+        dm.dsmoe_timing_enable(n_pairs)
+        barrier()
+        e0.record()
+        for i in range(steps):
+            run_step(i)
+        e1.record()
+        barrier()
+        ms_evented = e0.elapsed_time(e1) / steps
+        durs = np.array(dm.dsmoe_timing_read(n_pairs))
+        dm.dsmoe_timing_enable(0)
     assert int(status.item()) == 0
 
     step_s = ms_total * 1e-3 / steps
@@ -398,6 +412,7 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
         # summarised under profiles/; null where no capture of the current kernel exists
         roof["traffic"] = NCU_TRAFFIC_BYTES.get(name)
         roof["kernel_ms_per_step"] = kernel_ms
+        roof["ms_per_step_with_events"] = ms_evented     # the step time of the loop the kernel times were taken in
         roof["launch_ms_each"] = [float(v) for v in durs.mean(axis=0)[:timed_per_call]]
         roof["launches_per_step"] = calls_per_step * timed_per_call
         res["roofline"] = roof

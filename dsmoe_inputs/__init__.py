@@ -134,6 +134,7 @@ class LayerSpec:
     K: int = 0
     min_k: int = 0
     out_fp32: int = 0
+    fuse_combine: int = 0
     router_gain: float = 1.0       # scalar applied to the drawn Wr
     zipf_s: float = 0.0            # > 0: router bias b[e] = ln p, p ~ Zipf(s) over a seeded permutation
     seed: int = 0

@@ -80,6 +80,15 @@ typedef struct {
     int32_t min_k;            /* 0: a token may select nothing and then outputs 0;
                                  1: such a token keeps its lowest-index argmax             */
     int32_t out_fp32;         /* 1: `out` is fp32 even when dtype is bf16                  */
+    int32_t fuse_combine;     /* dsmoe_layer_forward with packed weights and a sparse selection:
+                                 0: the down-projection multiplies each expert output by its gate
+                                    in fp32 and stores it in dtype; a second kernel adds a token's
+                                    rows in ascending expert order (fastest);
+                                 1: no expert outputs are stored: the down-projection's epilogue
+                                    adds gate * output to the token's fp32 sum in ascending expert
+                                    order, one rounding at the end (most accurate, less DRAM
+                                    traffic, more L2 traffic: slower on B200).
+                                 Both are bit-reproducible from run to run.                  */
 } dsmoe_layer_desc;
 
 /* A void* stands for the caller's cudaStream_t so that this header needs no CUDA include. */
@@ -201,10 +210,9 @@ dsmoe_status dsmoe_pack_weights(const dsmoe_layer_desc* desc, const void* W1, co
  *   mask_out [T] uint64 and counts_out [E] int32: optional copies of the selection.
  *   dev_status: optional device int32; kernels write a dsmoe_status there if a bounded
  *   wait runs out or an index check fails (they then exit cleanly); untouched otherwise.
- *   With packed weights and a sparse selection the aggregation runs inside the down-projection:
- *   each expert's output is multiplied by its gate in fp32 and added to the token's fp32 sum in
- *   ascending expert order (the order dsmoe_combine uses), and rounded once when the token's last
- *   expert is done; results are bit-identical from run to run.
+ *   With packed weights and a sparse selection the gate multiply sits in the down-projection's
+ *   epilogue (fp32, before any rounding); desc->fuse_combine chooses whether the sum over a token's
+ *   experts does too.
  */
 dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, const float* Wr,
                                  const float* br, const void* W1, const void* W2,

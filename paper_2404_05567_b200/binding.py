@@ -31,7 +31,7 @@ class LayerDesc(ctypes.Structure):
     _fields_ = [("T", ctypes.c_int32), ("d", ctypes.c_int32), ("H", ctypes.c_int32), ("E", ctypes.c_int32),
                 ("dtype", ctypes.c_int32), ("mode", ctypes.c_int32), ("eps", ctypes.c_float),
                 ("eps_normalized", ctypes.c_int32), ("K", ctypes.c_int32), ("min_k", ctypes.c_int32),
-                ("out_fp32", ctypes.c_int32)]
+                ("out_fp32", ctypes.c_int32), ("fuse_combine", ctypes.c_int32)]
 
 
 class DsmoeError(RuntimeError):
@@ -82,9 +82,9 @@ def _stream(stream=None):
 
 
 def make_desc(T, d, H, E, dtype=BF16, mode=SELECT_THRESHOLD, eps=0.0, eps_normalized=0, K=0, min_k=0,
-              out_fp32=0) -> LayerDesc:
+              out_fp32=0, fuse_combine=0) -> LayerDesc:
     return LayerDesc(int(T), int(d), int(H), int(E), int(dtype), int(mode), float(eps), int(eps_normalized),
-                     int(K), int(min_k), int(out_fp32))
+                     int(K), int(min_k), int(out_fp32), int(fuse_combine))
 
 
 def width(desc: LayerDesc) -> int:

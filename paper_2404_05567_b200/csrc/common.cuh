@@ -106,8 +106,9 @@ dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const 
                                 cudaStream_t s);
 // Grouped expert MLPs on expert-sorted rows: h = GeLU(xp.W1[e]) (bf16, in `hbuf`), yp = h.W2[e].
 // With row_token (and x), the up-projection gathers its rows from x by index and xp is not read.
-// With cmb, the down-projection's epilogue also aggregates (Eq. 1's weighted sum, ascending expert order per token):
-// it writes the layer output cmb->out [T,d] and yp is not touched.
+// With cmb->out, the down-projection's epilogue also aggregates (Eq. 1's weighted sum, ascending expert order per
+// token): it writes the layer output cmb->out [T,d] and yp is not touched.  With cmb->out == NULL only the gate
+// multiply moves into the epilogue: yp[r,:] = row_gate[r] * e(x)[r,:].
 struct CombineArgs {
     const int32_t* row_token;
     const float* row_gate;

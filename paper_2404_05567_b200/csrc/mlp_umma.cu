@@ -434,6 +434,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const long long grow = (long long)t.row0 + row;
             float g = 1.f;
             if (P.gate && valid) g = P.gate[grow * P.E + t.e];
+            if (P.epi == EPI_STORE && P.row_gate && valid) g = P.row_gate[grow];
             const uint32_t taddr = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
             const bool warp_has_rows = q * 32 < t.rows_valid;   // warps without a valid row skip the read-back
             if (P.epi == EPI_COMBINE) {
@@ -543,7 +544,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        hv[j] = __floats2bfloat162_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+                        hv[j] = __floats2bfloat162_rn(g * __uint_as_float(r[2 * j]), g * __uint_as_float(r[2 * j + 1]));
                     uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) + o);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) dst[j] = pk[j];
@@ -1826,7 +1827,9 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
     GemmParams down{};
     down.mode = GEMM_GROUPED; down.epi = EPI_STORE; down.E = p.E; down.n_per_expert = p.d; down.k_per_expert = p.H;
     down.rows = (int)amax; down.offsets = offsets; down.out = yp; down.ld_out = p.d; down.dev_status = dev_status;
-    if (cmb) {
+    if (cmb && !cmb->out) {
+        down.row_gate = cmb->row_gate;     // yp[r,:] = gate[r] * (h.W2[e])[r,:], the product taken in fp32
+    } else if (cmb) {
         // Eq. 1's weighted sum inside the down-projection's epilogue: no expert-output buffer, no aggregation pass
         down.epi = EPI_COMBINE;
         down.out = cmb->out;

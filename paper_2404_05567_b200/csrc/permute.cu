@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(128) combine_bf16_kernel(const uint4* __restri
         const int r = token_rows[(size_t)t * W + threadIdx.x];
         const bool ok = r >= 0 && r < amax;
         rows_s[threadIdx.x] = ok ? r : 0;
-        gate_s[threadIdx.x] = ok ? row_gate[r] : 0.f;
+        gate_s[threadIdx.x] = !ok ? 0.f : row_gate ? row_gate[r] : 1.f;   // no gates: the rows carry them already
     }
     __syncthreads();
     const int nvec = d / 8;

@@ -51,7 +51,7 @@ def np_f32(t: torch.Tensor) -> np.ndarray:
 
 def desc_of(s: gi.LayerSpec) -> dm.LayerDesc:
     return dm.make_desc(s.T, s.d, s.H, s.E, dm.BF16 if s.dtype == "bf16" else dm.F32, s.mode, s.eps,
-                        s.eps_normalized, s.K, s.min_k, s.out_fp32)
+                        s.eps_normalized, s.K, s.min_k, s.out_fp32, s.fuse_combine)
 
 
 def torch_dtype(s: gi.LayerSpec):

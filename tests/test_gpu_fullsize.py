@@ -140,3 +140,40 @@ def test_permute_skips_rows_that_inconsistent_offsets_would_put_out_of_range():
     dm.dsmoe_permute(L.desc, L.x_d, to_dev(S), to_dev(mask_ref), to_dev(bad), row_token, row_gate, token_rows, xp, L.ws)
     torch.cuda.synchronize()
     assert np.all(to_np(row_token)[amax:] == -9)
+
+
+# ---------------------------------------------------------------- aggregation inside the down-projection (fuse_combine = 1)
+
+FUSED = [
+    dict(T=300, d=64, H=64, E=16, mode=gi.MODE_THRESHOLD, eps=0.5),                      # most tokens select nothing
+    dict(T=300, d=64, H=64, E=16, mode=gi.MODE_THRESHOLD, eps=0.5, min_k=1),
+    dict(T=1000, d=256, H=128, E=32, mode=gi.MODE_THRESHOLD, eps=0.7, eps_normalized=1, zipf_s=1.1),
+    dict(T=2048, d=512, H=256, E=32, mode=gi.MODE_TOPK, K=6),                            # several row tiles per expert
+    dict(T=300, d=448, H=320, E=8, mode=gi.MODE_TOPK, K=3),                              # ragged column tiles
+    dict(T=700, d=256, H=64, E=64, mode=gi.MODE_TOPK, K=64),                             # every expert, grouped
+    dict(T=513, d=128, H=128, E=16, mode=gi.MODE_THRESHOLD_TOPK, eps=0.03),
+    dict(T=260, d=128, H=128, E=8, mode=gi.MODE_TOPK, K=2, out_fp32=1),
+]
+
+
+@pytest.mark.parametrize("case", FUSED, ids=[str(i) for i in range(len(FUSED))])
+def test_aggregation_inside_the_down_projection(case):
+    s = gi.LayerSpec(f"fused{FUSED.index(case)}", dtype="bf16", router_gain=5.0, fuse_combine=1, **case)
+    r = layer_parity(s)
+    assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
+    L = r["layer"]
+    a = np_f32(L.forward()).copy()
+    b = np_f32(L.forward())
+    assert np.array_equal(a, b)                    # ordered sums: bit-identical from run to run
+    if case.get("eps") == 0.5 and not case.get("min_k"):
+        mask = to_np(L.mask)[:s.T]
+        assert (mask == 0).any() and np.all(a[mask == 0] == 0.0)
+
+
+@pytest.mark.parametrize("cfg,kw,n", [("c3", {}, 256), ("c5", dict(eps=0.1), 512)], ids=["c3", "c5_eps0.1"])
+def test_aggregation_inside_the_down_projection_full_size(cfg, kw, n):
+    s = gi.spec(cfg, fuse_combine=1, **kw)
+    r = layer_parity(s, sample=n)
+    assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
+    if cfg == "c3":
+        assert r["err"] <= TOL_BF16
