@@ -40,8 +40,12 @@ def test_small_layers(case, pack, dtype):
     s = gi.LayerSpec(f"small{SMALL.index(case)}", dtype=dtype, router_gain=6.0, **case)
     r = layer_parity(s, pack=pack)
     tol = TOL_F32 if dtype == "f32" else TOL_BF16
-    # adversarial shapes mix tokens with very different numbers of experts: the bar is applied per token
+    # adversarial shapes mix tokens with very different numbers of experts: the bar is applied per token ...
     assert r["err_rows"] <= tol, (r["err_rows"], r["err"])
+    # ... and over the whole output as well, except where most tokens select nothing: their rows of exact zeros
+    # pull the whole-output RMS far below that of the rows that carry values (measured there: up to 8e-2)
+    if case.get("eps") != 0.5:
+        assert r["err"] <= tol, r["err"]
     if case.get("eps") == 0.5 and not case.get("min_k"):
         assert r["zero_tokens"] > 0
         out = np_f32(r["layer"].out)
@@ -113,8 +117,11 @@ def test_c5_skewed_router_threshold_sweep(eps):
         assert r["A"] == s.T * s.E                       # no score underflows to 0 in this recipe
     if eps >= 0.1:
         assert r["empty_experts"] > 0 or r["zero_tokens"] > 0
-    # rows differ wildly in scale here (1 to 64 experts per token): the bar is applied per token
+    # rows differ wildly in scale here (1 to 64 experts per token): the bar is applied per token; the bar over the
+    # whole output holds too while few tokens select nothing (eps = 0.2: 28 % of the rows are exact zeros)
     assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
+    if eps < 0.1:
+        assert r["err"] <= TOL_BF16, r["err"]
 
 
 # ---------------------------------------------------------------- decode path corner cases
@@ -147,6 +154,7 @@ def test_decode_path_when_some_experts_are_unselected(case):
     s = gi.LayerSpec("dec_" + str(case["T"]), dtype="bf16", router_gain=8.0, **kw)
     r = layer_parity(s)
     assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
+    assert r["err"] <= TOL_BF16, r["err"]
     if case.get("eps") == 0.999:
         assert r["A"] == 0 and np.all(np_f32(r["layer"].out) == 0.0)
     if case["mode"] == gi.MODE_TOPK and case["K"] == 1:
@@ -168,7 +176,8 @@ def test_threshold_topk_layer(case, dtype):
     k = np_popcounts(r["layer"].mask, s.T)
     assert len(set(k.tolist())) == 1 and 1 <= int(k[0]) <= s.E        # every token got the same K
     assert r["A"] == s.T * int(k[0])
-    assert r["err_rows"] <= (TOL_BF16 if dtype == "bf16" else TOL_F32), (r["err_rows"], r["err"])
+    tol = TOL_BF16 if dtype == "bf16" else TOL_F32
+    assert r["err_rows"] <= tol and r["err"] <= tol, (r["err_rows"], r["err"])
 
 
 def np_popcounts(mask_t, T):
@@ -189,13 +198,13 @@ def test_paper_shaped_decode(name, d, H, T):
     s = gi.LayerSpec(f"paper_{name}_t{T}", T=T, d=d, H=H, E=32, dtype="bf16", mode=gi.MODE_THRESHOLD, eps=0.03,
                      router_gain=2.0)
     r = layer_parity(s)
-    assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
+    assert r["err_rows"] <= TOL_BF16 and r["err"] <= TOL_BF16, (r["err_rows"], r["err"])
 
 
 @pytest.mark.parametrize("name,d,H", PAPER_SHAPES, ids=[p[0] for p in PAPER_SHAPES])
 @pytest.mark.parametrize("K", [4, 6])
 def test_paper_shaped_prefill_topk(name, d, H, K):
     s = gi.LayerSpec(f"paper_{name}_k{K}", T=2048, d=d, H=H, E=32, dtype="bf16", mode=gi.MODE_TOPK, K=K)
-    r = layer_parity(s, sample=24)
+    r = layer_parity(s, sample=256)
     assert r["A"] == 2048 * K
-    assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
+    assert r["err_rows"] <= TOL_BF16 and r["err"] <= TOL_BF16, (r["err_rows"], r["err"])
