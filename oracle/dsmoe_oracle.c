@@ -15,6 +15,8 @@
  *              e(X) an MLP with GeLU       ("Model Hyperparameters" paragraph)
  *   dense      every expert evaluated and weighted by its score: the forward
  *              whose gradients are Eq. 3   ("Dense Training" paragraph)
+ *   training   the gradients of Eq. 2 and Eq. 3 for a given output gradient, and
+ *              the mutual-information loss of the router (Eq. 4-6)
  *
  * Readings where the paper is silent (each also listed in the design notes):
  * router h is linear (x.Wr + b); GeLU is the exact erf form; expert MLPs carry
@@ -248,6 +250,91 @@ void oracle_combine(const float *yp, const float *row_gate, const int32_t *token
             double g = (double)row_gate[r];
             for (int64_t c = 0; c < d; ++c) o[c] += g * (double)yp[(size_t)r * d + c];
         }
+    }
+}
+
+/*
+ * Mutual-information loss of the router ("Mutual Information Loss" paragraph, Eq. 4-6) over the T tokens
+ * of a minibatch, natural logarithms, 0 log 0 = 0:
+ *     p(e_i)   = (1/T) sum_X S_i(X)                  the experts' marginal distribution (Eq. 4's p(e); the
+ *                                                    paper's formula drops the index i)
+ *     H(e)     = - sum_i p(e_i) log p(e_i)           (Eq. 4)
+ *     H(e|X)   = - sum_i S_i(X) log S_i(X)
+ *     L_MI     = - H(e) + (1/T) sum_X H(e|X)         (Eq. 5)
+ * out3 = {L_MI, H(e), (1/T) sum_X H(e|X)}.  grad (optional, [T,E]) = dL_MI/dS, differentiating the three lines
+ * above term by term: (log p(e_i) - log S_i(X)) / T  (0 where S_i(X) = 0).
+ */
+void oracle_mi_loss(const float *scores, int64_t T, int64_t E, double *out3, double *grad) {
+    double p[64];
+    for (int64_t e = 0; e < E; ++e) p[e] = 0.0;
+    double hcond = 0.0;
+    for (int64_t t = 0; t < T; ++t)
+        for (int64_t e = 0; e < E; ++e) {
+            double s = (double)scores[t * E + e];
+            p[e] += s;
+            if (s > 0.0) hcond -= s * log(s);
+        }
+    double he = 0.0;
+    for (int64_t e = 0; e < E; ++e) {
+        p[e] /= (double)T;
+        if (p[e] > 0.0) he -= p[e] * log(p[e]);
+    }
+    hcond /= (double)T;
+    out3[0] = -he + hcond;
+    out3[1] = he;
+    out3[2] = hcond;
+    if (grad)
+        for (int64_t t = 0; t < T; ++t)
+            for (int64_t e = 0; e < E; ++e) {
+                double s = (double)scores[t * E + e];
+                grad[t * E + e] = s > 0.0 ? (log(p[e]) - log(s)) / (double)T : 0.0;
+            }
+}
+
+/*
+ * Gradients of dense training ("Dense Training" paragraph).  Given the gradient dO of the layer output,
+ *     grad S_j     = < e_j(X), dO >     for every expert j                       (Eq. 3, first half)
+ *     grad e_j(X)  = S_j dO                                                      (Eq. 3, second half)
+ * and, with a mask M (Eq. 2: sparse training), both only for the experts that M marks active.  The second
+ * gradient is returned one linear step further down, at the expert's hidden activation
+ * a_j = GeLU(X.W1[j]) (e_j(X) = a_j.W2[j]):  dA[t,j,:] = (S_j dO).W2[j]^T, which is what the backward pass of the
+ * expert consumes next.  dO has the storage type of x.  Outputs in double: dS [n,E], dA [n,E,H] (optional);
+ * row i is token token_ids[i] (or i).
+ */
+void oracle_dense_backward(const void *x, const void *W1, const void *W2, int dtype, const float *scores,
+                           const uint64_t *mask, const void *dO, const int64_t *token_ids, int64_t n_tokens,
+                           int64_t d, int64_t H, int64_t E, double *dS, double *dA) {
+#pragma omp parallel
+    {
+        double *hbuf = (double *)malloc(sizeof(double) * (size_t)H);
+        double *y = (double *)malloc(sizeof(double) * (size_t)d);
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t i = 0; i < n_tokens; ++i) {
+            int64_t t = token_ids ? token_ids[i] : i;
+            for (int64_t e = 0; e < E; ++e) {
+                int active = mask ? (int)((mask[t] >> e) & 1) : 1;
+                double acc = 0.0;
+                if (active) {
+                    expert_apply(x, dtype, (size_t)(t * d), W1, W2, e, d, H, hbuf, y);
+                    for (int64_t c = 0; c < d; ++c) acc += y[c] * load_val(dO, dtype, (size_t)(t * d + c));
+                }
+                dS[i * E + e] = acc;
+                if (dA) {
+                    double s = (double)scores[t * E + e];
+                    for (int64_t k = 0; k < H; ++k) {
+                        double g = 0.0;
+                        if (active) {
+                            size_t base = (size_t)((e * H + k) * d);
+                            for (int64_t c = 0; c < d; ++c)
+                                g += load_val(dO, dtype, (size_t)(t * d + c)) * load_val(W2, dtype, base + (size_t)c);
+                        }
+                        dA[(i * E + e) * H + k] = s * g;
+                    }
+                }
+            }
+        }
+        free(hbuf);
+        free(y);
     }
 }
 

@@ -21,7 +21,7 @@ _lib = None
 MODE_THRESHOLD, MODE_TOPK, MODE_ALL, MODE_THRESHOLD_TOPK = 0, 1, 2, 3
 
 __all__ = [
-    "build", "router_scores", "select", "group", "layer", "expert_rows", "combine",
+    "build", "router_scores", "select", "group", "layer", "expert_rows", "combine", "mi_loss", "dense_backward",
     "num_threads", "MODE_THRESHOLD", "MODE_TOPK", "MODE_ALL", "MODE_THRESHOLD_TOPK",
 ]
 
@@ -146,6 +146,38 @@ def expert_rows(xp, W1, W2, row_expert, rows=None) -> np.ndarray:
     _load().oracle_expert_rows(_p(xp), _p(W1), _p(W2), dt, _p(row_expert), _p(ids),
                                ctypes.c_int64(n), ctypes.c_int64(d), ctypes.c_int64(H), _p(yp))
     return yp
+
+
+def mi_loss(scores, want_grad: bool = False):
+    """Mutual-information loss of the router (Eq. 4-6): returns (L_MI, H(e), mean H(e|X)) and, with
+    ``want_grad``, also dL_MI/dS as float64 [T,E]."""
+    S = _c(scores, np.float32)
+    T, E = S.shape
+    out3 = np.zeros(3, dtype=np.float64)
+    grad = np.empty((T, E), dtype=np.float64) if want_grad else None
+    _load().oracle_mi_loss(_p(S), ctypes.c_int64(T), ctypes.c_int64(E), _p(out3), _p(grad))
+    res = (float(out3[0]), float(out3[1]), float(out3[2]))
+    return res + (grad,) if want_grad else res
+
+
+def dense_backward(x, W1, W2, scores, dO, mask=None, token_ids=None, want_dA: bool = True):
+    """Gradients of dense training (Eq. 3; Eq. 2 with ``mask``): dS[n,E] = <e_j(x), dO> and dA[n,E,H] =
+    (S_j dO).W2[j]^T, the gradient at the experts' hidden activations.  float64."""
+    x, W1, W2, dO = _c(x), _c(W1), _c(W2), _c(dO)
+    S = _c(scores, np.float32)
+    T, d = x.shape
+    E, d1, H = W1.shape
+    assert d1 == d and W2.shape == (E, H, d) and S.shape == (T, E) and dO.shape == (T, d)
+    dt = _dtype_code(x)
+    assert _dtype_code(W1) == dt and _dtype_code(W2) == dt and _dtype_code(dO) == dt
+    mask = None if mask is None else _c(mask, np.uint64)
+    ids = None if token_ids is None else _c(token_ids, np.int64)
+    n = T if ids is None else ids.shape[0]
+    dS = np.empty((n, E), dtype=np.float64)
+    dA = np.empty((n, E, H), dtype=np.float64) if want_dA else None
+    _load().oracle_dense_backward(_p(x), _p(W1), _p(W2), dt, _p(S), _p(mask), _p(dO), _p(ids), ctypes.c_int64(n),
+                                  ctypes.c_int64(d), ctypes.c_int64(H), ctypes.c_int64(E), _p(dS), _p(dA))
+    return dS, dA
 
 
 def combine(yp, row_gate, token_rows) -> np.ndarray:
