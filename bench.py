@@ -38,7 +38,7 @@ PAPER_SHAPES = {"1b": (2048, 256, 6), "3b": (3072, 384, 6), "6b": (4096, 512, 4)
 WORKLOADS = {
     "c2_t1": ("c2", dict(T=1)), "c2_t8": ("c2", dict(T=8)), "c2_t32": ("c2", dict(T=32)),
     "c3": ("c3", {}), "c4": ("c4", {}),
-    "c3_fused": ("c3", dict(fuse_combine=1)),      # aggregation inside the down-projection's epilogue (see dsmoe.h)
+    "c3_separate": ("c3", dict(fuse_combine=2)),   # aggregation as a second kernel instead of inside the down-projection (see dsmoe.h)
     "c5": ("c5", dict(eps=0.01)),
     # output-token throughput as the paper measures it ("GPU Inference Analysis"): a decode loop in which layer i's
     # output is layer i+1's input, 24 distinct layers (Table tab:model_arch: N_layer = 24 .. 36); W2 is drawn 16 times
@@ -51,8 +51,8 @@ for _n, (_d, _H, _K) in PAPER_SHAPES.items():
     WORKLOADS[f"paper{_n}_prefill"] = ("c3", dict(T=8192, d=_d, H=_H, K=_K))
     WORKLOADS[f"paper{_n}_t32"] = ("c2", dict(T=32, d=_d, H=_H))
 NCU_TRAFFIC_BYTES = {}     # dram bytes per launch of the dominant kernel from the ncu captures under profiles/
-DEFAULT_STEPS = {"c3": 100, "c3_fused": 100, "c4": 50}
-ALSO = [("c2_t1", 500), ("c2_t8", 500), ("c3", 30), ("c3_fused", 30), ("c4", 15)] + [(f"c5_eps{e}", 15) for e in (0.0, 0.01, 0.05, 0.1, 0.2)] + \
+DEFAULT_STEPS = {"c3": 100, "c3_separate": 100, "c4": 50}
+ALSO = [("c2_t1", 500), ("c2_t8", 500), ("c3", 30), ("c3_separate", 30), ("c4", 15)] + [(f"c5_eps{e}", 15) for e in (0.0, 0.01, 0.05, 0.1, 0.2)] + \
        [(f"paper{n}_prefill", 30) for n in PAPER_SHAPES] + [(f"paper{n}_t32", 300) for n in ("1b", "3b", "6b", "19b")] + \
        [("decode_loop_t8", 20), ("decode_loop_t32", 20)]
 METRIC = "moe_layer_tokens_per_s"
@@ -252,7 +252,8 @@ def kernels_per_step(s, decode):
     if s.mode == gi.MODE_ALL:
         return router + 2                          # up, down
     # chunk count, finalize, permute index, up, down, and the aggregation unless it runs inside the down-projection
-    return router + 3 + 2 + (0 if s.fuse_combine else 1)
+    fused = s.fuse_combine == 1 or (s.fuse_combine == 0 and s.H >= 1024)      # the library's rule (dsmoe.h)
+    return router + 3 + 2 + (0 if fused else 1)
 
 
 def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, sampler_index=0, graph=False):
@@ -501,6 +502,8 @@ def main():
     ap.add_argument("--workload", default="c2_t32", choices=sorted(WORKLOADS))
     ap.add_argument("--no-extra", action="store_true")
     ap.add_argument("--graph", action="store_true", help="replay each step as one CUDA graph")
+    ap.add_argument("--fuse-combine", type=int, default=None, choices=[0, 1, 2],
+                    help="override the workload's fuse_combine (see dsmoe.h)")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--rendezvous-only", action="store_true",
                     help="start the ranks, reduce a stand-in timing and print n_gpus; no GPU work")
@@ -513,6 +516,9 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.fuse_combine is not None:
+        for k in WORKLOADS:
+            WORKLOADS[k] = (WORKLOADS[k][0], dict(WORKLOADS[k][1], fuse_combine=args.fuse_combine))
     cfg, kw = WORKLOADS[name]
     s = gi.spec(cfg, **kw)
 

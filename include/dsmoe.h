@@ -80,15 +80,18 @@ typedef struct {
     int32_t min_k;            /* 0: a token may select nothing and then outputs 0;
                                  1: such a token keeps its lowest-index argmax             */
     int32_t out_fp32;         /* 1: `out` is fp32 even when dtype is bf16                  */
-    int32_t fuse_combine;     /* dsmoe_layer_forward with packed weights and a sparse selection:
-                                 0: the down-projection multiplies each expert output by its gate
-                                    in fp32 and stores it in dtype; a second kernel adds a token's
-                                    rows in ascending expert order (fastest);
-                                 1: no expert outputs are stored: the down-projection's epilogue
-                                    adds gate * output to the token's fp32 sum in ascending expert
-                                    order, one rounding at the end (most accurate, less DRAM
-                                    traffic, more L2 traffic: slower on B200).
-                                 Both are bit-reproducible from run to run.                  */
+    int32_t fuse_combine;     /* dsmoe_layer_forward with packed weights and a sparse selection -- where
+                                 Eq. 1's sum over a token's experts is taken.  Either way each expert
+                                 output is multiplied by its gate in fp32 in the down-projection's
+                                 epilogue and nothing is rounded before the sum; the sum runs in
+                                 ascending expert order and is bit-reproducible from run to run.
+                                 1: inside the down-projection: its epilogue adds gate * output to the
+                                    token's fp32 running sum; no expert outputs are stored, no second
+                                    pass (least DRAM traffic; the read-modify-write of the sums goes
+                                    through L2 and is hidden only when the experts are wide);
+                                 2: the epilogue stores the gate-weighted outputs as fp32 rows and a
+                                    second kernel adds a token's rows;
+                                 0: the library chooses: 1 for H >= 1024, else 2.               */
 } dsmoe_layer_desc;
 
 /* A void* stands for the caller's cudaStream_t so that this header needs no CUDA include. */

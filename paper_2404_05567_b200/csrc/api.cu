@@ -15,7 +15,7 @@ dsmoe_status check_desc(const dsmoe_layer_desc* p) {
     if (p->min_k != 0 && p->min_k != 1) return DSMOE_ERR_INVALID_ARG;
     if (p->eps_normalized != 0 && p->eps_normalized != 1) return DSMOE_ERR_INVALID_ARG;
     if (p->out_fp32 != 0 && p->out_fp32 != 1) return DSMOE_ERR_INVALID_ARG;
-    if (p->fuse_combine != 0 && p->fuse_combine != 1) return DSMOE_ERR_INVALID_ARG;
+    if (p->fuse_combine < 0 || p->fuse_combine > 2) return DSMOE_ERR_INVALID_ARG;
     if ((p->mode == DSMOE_SELECT_THRESHOLD || p->mode == DSMOE_SELECT_THRESHOLD_TOPK) && !(p->eps == p->eps))
         return DSMOE_ERR_INVALID_ARG;   // NaN
     if ((p->d & 7) || (p->H & 7)) return DSMOE_ERR_INVALID_ARG;
@@ -63,8 +63,9 @@ WsLayout ws_layout(const dsmoe_layer_desc& p) {
             h_bytes = T * E * p.H * 2;                              // dense forward, small-T: [T, E*H]
     }
     L.h = take(h_bytes);
-    // grouped: gate-weighted expert outputs [Amax,d] bf16, or (fuse_combine) the tokens' fp32 running sums [T,d]
-    L.acc = take(!umma_supported(p) ? 0 : p.fuse_combine ? T * p.d * 4 : amax * p.d * 2);
+    // grouped: the tokens' fp32 running sums [T,d] (aggregation inside the down-projection), or the gate-weighted
+    // expert outputs [Amax,d] in fp32 (separate aggregation)
+    L.acc = take(!umma_supported(p) ? 0 : fuses_combine(p) ? T * p.d * 4 : amax * p.d * 4);
     // fp32 partial sums of the small-T path: (CTA, 2 column ranges, T, 256)
     L.partial = take(umma_supported(p) && p.T <= kSmallMaxT ? (size_t)kSmallMaxCtas * 2 * T * 256 * 4 : 0);
     L.router = take(router_umma_supported(p) ? router_umma_scratch(p) : 0);   // tensor-core router: split Wr, partial logits
@@ -259,7 +260,7 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
 
     // grouped path: duplicate tokens per selected expert, run the experts, aggregate
     DSMOE_TRY(launch_finalize(p, mask, counts, offsets, chunk_prefix, counts_out, s));
-    if (fast && p.fuse_combine) {
+    if (fast && fuses_combine(p)) {
         // no grouped copy of the tokens (the up-projection gathers rows of x by row_token), no buffer of expert
         // outputs and no aggregation pass: the down-projection's epilogue adds each expert's gate-weighted output
         // to the token's fp32 sum, in ascending expert order, and writes the final rounding
@@ -269,11 +270,11 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
         return launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, nullptr, dev_status, s, x, row_token, &cmb);
     }
     if (fast) {
-        // the down-projection's epilogue multiplies by the gate (fp32) and stores; the aggregation only adds
+        // the down-projection's epilogue multiplies by the gate and stores fp32 rows; the aggregation only adds
         DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, nullptr, s));
         const CombineArgs gated{row_token, row_gate, nullptr, nullptr, nullptr, nullptr};
         DSMOE_TRY(launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, ws + L.acc, dev_status, s, x, row_token, &gated));
-        return launch_combine(p, ws + L.acc, nullptr, token_rows, k_t, out, s);
+        return launch_combine(p, ws + L.acc, nullptr, token_rows, k_t, out, s, true);
     }
     DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, ws + L.xp, s));
     DSMOE_TRY(launch_mlp_generic(p, ws + L.xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h_plain), ws + L.yp, s));

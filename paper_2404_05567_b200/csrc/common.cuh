@@ -83,8 +83,14 @@ dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const floa
 // Selection statistics (see dsmoe_stats)
 dsmoe_status launch_stats(const dsmoe_layer_desc& p, const float* scores, const uint64_t* mask,
                           dsmoe_selection_stats* stats, cudaStream_t s);
+// yp_f32: the rows are fp32 whatever p.dtype says; row_gate == NULL: the rows are gate-weighted already
 dsmoe_status launch_combine(const dsmoe_layer_desc& p, const void* yp, const float* row_gate,
-                            const int32_t* token_rows, const int32_t* k_t, void* out, cudaStream_t s);
+                            const int32_t* token_rows, const int32_t* k_t, void* out, cudaStream_t s,
+                            bool yp_f32 = false);
+// Whether dsmoe_layer_forward's tensor-core grouped path aggregates inside the down-projection (see dsmoe.h)
+static inline bool fuses_combine(const dsmoe_layer_desc& p) {
+    return p.fuse_combine == 1 || (p.fuse_combine == 0 && p.H >= 1024);
+}
 dsmoe_status launch_pack(const dsmoe_layer_desc& p, const void* W1, const void* W2, void* packed,
                          cudaStream_t s);
 
@@ -108,7 +114,7 @@ dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const 
 // With row_token (and x), the up-projection gathers its rows from x by index and xp is not read.
 // With cmb->out, the down-projection's epilogue also aggregates (Eq. 1's weighted sum, ascending expert order per
 // token): it writes the layer output cmb->out [T,d] and yp is not touched.  With cmb->out == NULL only the gate
-// multiply moves into the epilogue: yp[r,:] = row_gate[r] * e(x)[r,:].
+// multiply moves into the epilogue: yp[r,:] = row_gate[r] * e(x)[r,:], stored as fp32.
 struct CombineArgs {
     const int32_t* row_token;
     const float* row_gate;

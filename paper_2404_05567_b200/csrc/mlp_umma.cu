@@ -43,7 +43,11 @@ constexpr int STG_BYTES = BM * 36 * 4;                                 // epilog
 // small_layer_kernel asks only for the ring bytes it keeps in flight: what it leaves stays with the SM's L1, which
 // serves the kernel's many small loads (its parameters' copy, the router's operands)
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)SMALL_RING_BYTES + SHARED_BYTES + STG_BYTES;
-constexpr size_t SMEM_GEMM_BYTES = 1024 + (size_t)RING_BYTES + SHARED_BYTES;   // umma_gemm_kernel needs no staging tile
+constexpr size_t SMEM_GEMM_BYTES = 1024 + (size_t)RING_BYTES + SHARED_BYTES;   // umma_gemm_kernel needs no staging tile ...
+// ... except with the aggregation in its epilogue: 12 epilogue warps, each with a 32 x 16 fp32 transposition tile
+constexpr int CMB_WARPS = 12, CMB_COLS = 16, CMB_LD = CMB_COLS + 1;
+constexpr size_t SMEM_GEMM_CMB_BYTES = SMEM_GEMM_BYTES + (size_t)CMB_WARPS * 32 * CMB_LD * 4;
+static_assert(SMEM_GEMM_CMB_BYTES <= 227 * 1024, "shared memory of one CTA");
 
 enum { GEMM_GROUPED = 0, GEMM_DENSE_UP = 1, GEMM_DENSE_DOWN = 2 };
 enum { EPI_GELU = 0, EPI_STORE = 1, EPI_COMBINE = 2 };
@@ -253,7 +257,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(ptx::smem_u32(&sh.tfull[a]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh.tempty[a]), 4);
+            ptx::mbar_init(ptx::smem_u32(&sh.tempty[a]), P.epi == EPI_COMBINE ? CMB_WARPS : 4);
         }
         sh.abort_flag = 0;
         sh.bad_offsets = 0;
@@ -374,7 +378,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
             }
         }
-    } else if (warp >= 6) {
+    } else if (warp >= 6 && P.gather) {
         // ------------------------------------------------------------ gather (8 warps, grouped up-projection only)
         // Warps j and j + 4 bring the two halves of the A tiles of the ring stages j, j + 4, ... of this CTA's
         // sequence: per stage, 16 cp.async instructions each, an instruction covering 4 rows x 128 bytes (8 lanes x 16 bytes per row), written in the
@@ -419,8 +423,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 ptx::mbar_arrive(ptx::smem_u32(&sh.full[s]));
             }
         }
-    } else {
-        // ------------------------------------------------------------ epilogue (4 warps)
+    } else if (warp < 6 || P.epi == EPI_COMBINE) {
+        // ------------------------------------------------------------ epilogue (4 warps; 12 with the aggregation)
         const int q = warp & 3;
         int acc = 0;
         uint32_t aph = 0;
@@ -444,65 +448,87 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 // touches the sums once every tile of the previous non-empty expert that covers the same columns has
                 // finished (tiles are handed out in ascending expert order to CTAs that are all resident: the
                 // wait is for work that is already running or done).
+                // Three warps share each quarter of the accumulator's rows (a warp reads TMEM lanes 32 (warp % 4) ..),
+                // taking every third 16-column piece: 12 warps' worth of loads of the old sums are in flight.  A
+                // piece goes from TMEM (lane = row) through a small shared-memory tile into a layout in which 4
+                // neighbouring lanes hold one row's 64 bytes, so that the sums are read and written in full sectors.
                 const int ntn = (P.n_per_expert + BN - 1) / BN, nt = t.n0 / BN;
+                const int slot = warp < 6 ? 0 : 1 + (warp - 6) / 4;
+                float* tp = reinterpret_cast<float*>(smem_raw + (base - raw) + RING_BYTES + SHARED_BYTES) +
+                            (slot * 4 + q) * 32 * CMB_LD;
                 int prev = t.e - 1;
                 while (prev >= 0 && sh.seg1[prev] <= sh.seg0[prev]) --prev;
                 bool ok = true;
                 if (prev >= 0 && warp_has_rows) {
                     if (lane == 0) {
-                        const int target = 4 * ((sh.seg1[prev] - sh.seg0[prev] + BM - 1) / BM);
+                        const int target = CMB_WARPS * ((sh.seg1[prev] - sh.seg0[prev] + BM - 1) / BM);
                         ok = flag_wait_ge(P.tile_done + prev * ntn + nt, target, &sh.abort_flag);
                     }
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 }
                 if (!ok) break;
-                int tok = 0;
+                // this lane's own row (lane = row): token, gate, and whether the expert is the token's first / last
+                int tok = 0, flags = 0;
                 float g = 0.f;
-                bool first = true, last = true;
                 if (valid) {
                     tok = min(max(P.row_token[grow], 0), P.tokens - 1);
                     g = P.row_gate[grow];
                     const uint64_t m = P.sel_mask[tok];
-                    first = (m & ((1ull << t.e) - 1ull)) == 0ull;
-                    last = ((m >> t.e) >> 1) == 0ull;
+                    flags = 4 | ((m & ((1ull << t.e) - 1ull)) == 0ull ? 1 : 0) | (((m >> t.e) >> 1) == 0ull ? 2 : 0);
                 }
-                float* arow = P.acc + (long long)tok * P.n_per_expert + t.out_col0;
-                for (int c = 0; warp_has_rows && c < t.bn; c += 32) {
-                    float4 old[8];
-                    if (valid && !first) {
+                // ... and the same for the four rows this lane serves in the transposed layout: rows rg + 8 i,
+                // 16-byte piece pc of their 64 bytes
+                const int rg = lane >> 2, pc = lane & 3;
+                int tk[4], fl[4];
+                float gt[4];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) old[j] = __ldcg(reinterpret_cast<const float4*>(arow + c) + j);
-                    } else {
+                for (int i = 0; i < 4; ++i) {
+                    tk[i] = __shfl_sync(0xffffffffu, tok, rg + 8 * i);
+                    fl[i] = __shfl_sync(0xffffffffu, flags, rg + 8 * i);
+                    gt[i] = __shfl_sync(0xffffffffu, g, rg + 8 * i);
+                }
+                const int npieces = t.bn / CMB_COLS;
+                auto fetch = [&](int piece, float4 (&o)[4]) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) old[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int i = 0; i < 4; ++i) {
+                        o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (piece < npieces && (fl[i] & 5) == 4)      // a valid row that is not its token's first expert
+                            o[i] = __ldcg(reinterpret_cast<const float4*>(
+                                P.acc + (long long)tk[i] * P.n_per_expert + t.out_col0 + piece * CMB_COLS + pc * 4));
                     }
-                    uint32_t r[32];
-                    ptx::tmem_ld32(taddr + (uint32_t)c, r);
+                };
+                float4 cur[4], nxt[4];
+                if (warp_has_rows) fetch(slot, cur);
+                for (int piece = slot; warp_has_rows && piece < npieces; piece += CMB_WARPS / 4) {
+                    fetch(piece + CMB_WARPS / 4, nxt);
+                    uint32_t r[16];
+                    ptx::tmem_ld16(taddr + (uint32_t)(piece * CMB_COLS), r);
                     ptx::tmem_ld_wait();
-                    if (!valid) continue;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        old[j].x = fmaf(g, __uint_as_float(r[4 * j]), old[j].x);
-                        old[j].y = fmaf(g, __uint_as_float(r[4 * j + 1]), old[j].y);
-                        old[j].z = fmaf(g, __uint_as_float(r[4 * j + 2]), old[j].z);
-                        old[j].w = fmaf(g, __uint_as_float(r[4 * j + 3]), old[j].w);
-                    }
-                    if (last && !P.out_f32) {
-                        uint4 pk[4];
-                        __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
+                    for (int j = 0; j < 16; ++j) tp[lane * CMB_LD + j] = __uint_as_float(r[j]);
+                    __syncwarp();
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            hv[2 * j] = __floats2bfloat162_rn(old[j].x, old[j].y);
-                            hv[2 * j + 1] = __floats2bfloat162_rn(old[j].z, old[j].w);
+                    for (int i = 0; i < 4; ++i) {
+                        const float* src = tp + (rg + 8 * i) * CMB_LD + pc * 4;
+                        float4 v = cur[i];
+                        v.x = fmaf(gt[i], src[0], v.x);
+                        v.y = fmaf(gt[i], src[1], v.y);
+                        v.z = fmaf(gt[i], src[2], v.z);
+                        v.w = fmaf(gt[i], src[3], v.w);
+                        if (!(fl[i] & 4)) continue;
+                        const long long o = (long long)tk[i] * P.n_per_expert + t.out_col0 + piece * CMB_COLS + pc * 4;
+                        if ((fl[i] & 2) && !P.out_f32) {
+                            uint2 pk;
+                            *reinterpret_cast<__nv_bfloat162*>(&pk.x) = __floats2bfloat162_rn(v.x, v.y);
+                            *reinterpret_cast<__nv_bfloat162*>(&pk.y) = __floats2bfloat162_rn(v.z, v.w);
+                            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(P.out) + o) = pk;
+                        } else {
+                            __stcg(reinterpret_cast<float4*>(P.acc + o), v);
                         }
-                        uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) +
-                                                              (long long)tok * P.ld_out + t.out_col0 + c);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) dst[j] = pk[j];
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) __stcg(reinterpret_cast<float4*>(arow + c) + j, old[j]);
                     }
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) cur[i] = nxt[i];
                 }
                 ptx::tc_fence_before();
                 __syncwarp();
@@ -537,8 +563,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     float4* dst = reinterpret_cast<float4*>(static_cast<float*>(P.out) + o);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                             __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                        dst[j] = make_float4(g * __uint_as_float(r[4 * j]), g * __uint_as_float(r[4 * j + 1]),
+                                             g * __uint_as_float(r[4 * j + 2]), g * __uint_as_float(r[4 * j + 3]));
                 } else {
                     uint4 pk[4];
                     __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
@@ -1671,17 +1697,17 @@ dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams&
     DeviceState* st = nullptr;
     DSMOE_TRY(device_state(&st));
     if (!st->attr_gemm) {
-        DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_BYTES));
+        DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_CMB_BYTES));
         st->attr_gemm = true;
     }
     const bool timed = may_time && g_timing.on && g_timing.n < g_timing.cap;
     if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
-    const int threads = P.gather ? GATHER_THREADS : NUM_THREADS;
+    const int threads = (P.gather || P.epi == EPI_COMBINE) ? GATHER_THREADS : NUM_THREADS;
     if (P.epi == EPI_COMBINE) {
         // its epilogues wait for one another's tiles: every CTA must be resident
         void* args[] = {const_cast<CUtensorMap*>(&a), const_cast<BMaps*>(&b), const_cast<GemmParams*>(&P)};
         DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(umma_gemm_kernel), dim3(grid), dim3(threads),
-                                                   args, SMEM_GEMM_BYTES, s));
+                                                   args, SMEM_GEMM_CMB_BYTES, s));
     } else {
         umma_gemm_kernel<<<grid, threads, SMEM_GEMM_BYTES, s>>>(a, b, P);
         DSMOE_CUDA_TRY(cudaGetLastError());
@@ -1828,7 +1854,8 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
     down.mode = GEMM_GROUPED; down.epi = EPI_STORE; down.E = p.E; down.n_per_expert = p.d; down.k_per_expert = p.H;
     down.rows = (int)amax; down.offsets = offsets; down.out = yp; down.ld_out = p.d; down.dev_status = dev_status;
     if (cmb && !cmb->out) {
-        down.row_gate = cmb->row_gate;     // yp[r,:] = gate[r] * (h.W2[e])[r,:], the product taken in fp32
+        down.row_gate = cmb->row_gate;     // yp[r,:] = gate[r] * (h.W2[e])[r,:] in fp32: no rounding before the sum
+        down.out_f32 = 1;
     } else if (cmb) {
         // Eq. 1's weighted sum inside the down-projection's epilogue: no expert-output buffer, no aggregation pass
         down.epi = EPI_COMBINE;

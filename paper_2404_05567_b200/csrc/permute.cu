@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(128) combine_bf16_kernel(const uint4* __restri
         const int r = token_rows[(size_t)t * W + threadIdx.x];
         const bool ok = r >= 0 && r < amax;
         rows_s[threadIdx.x] = ok ? r : 0;
-        gate_s[threadIdx.x] = !ok ? 0.f : row_gate ? row_gate[r] : 1.f;   // no gates: the rows carry them already
+        gate_s[threadIdx.x] = ok ? row_gate[r] : 0.f;
     }
     __syncthreads();
     const int nvec = d / 8;
@@ -119,9 +119,12 @@ __global__ void __launch_bounds__(128) combine_bf16_kernel(const uint4* __restri
     }
 }
 
+// fp32 rows: the plain path's fp32 layers (gates applied here) and the tensor-core path's gate-weighted fp32 expert
+// outputs (row_gate == NULL: only the sum is left to do; the output may be bf16)
+template <bool OUT_BF16>
 __global__ void __launch_bounds__(128) combine_f32_kernel(const float4* __restrict__ yp, const float* __restrict__ row_gate,
                                                           const int32_t* __restrict__ token_rows,
-                                                          const int32_t* __restrict__ k_t, float4* __restrict__ out,
+                                                          const int32_t* __restrict__ k_t, void* __restrict__ out,
                                                           int d, int W, int64_t amax) {
     __shared__ int32_t rows_s[kMaxExperts];
     __shared__ float gate_s[kMaxExperts];
@@ -131,21 +134,35 @@ __global__ void __launch_bounds__(128) combine_f32_kernel(const float4* __restri
         const int r = token_rows[(size_t)t * W + threadIdx.x];
         const bool ok = r >= 0 && r < amax;
         rows_s[threadIdx.x] = ok ? r : 0;
-        gate_s[threadIdx.x] = ok ? row_gate[r] : 0.f;
+        gate_s[threadIdx.x] = !ok ? 0.f : row_gate ? row_gate[r] : 1.f;
     }
     __syncthreads();
     const int nvec = d / 4;
     for (int v = threadIdx.x; v < nvec; v += 128) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int i = 0; i < k; ++i) {
-            const float4 y = __ldg(yp + (size_t)rows_s[i] * nvec + v);
-            const float g = gate_s[i];
-            acc.x = fmaf(g, y.x, acc.x);
-            acc.y = fmaf(g, y.y, acc.y);
-            acc.z = fmaf(g, y.z, acc.z);
-            acc.w = fmaf(g, y.w, acc.w);
+        // four rows' loads are issued before their first use (past the k-th row, row 0 is fetched again and not used)
+        for (int i = 0; i < k; i += 4) {
+            float4 y[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) y[j] = __ldg(yp + (size_t)rows_s[i + j < k ? i + j : 0] * nvec + v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (i + j >= k) continue;
+                const float g = gate_s[i + j];
+                acc.x = fmaf(g, y[j].x, acc.x);
+                acc.y = fmaf(g, y[j].y, acc.y);
+                acc.z = fmaf(g, y[j].z, acc.z);
+                acc.w = fmaf(g, y[j].w, acc.w);
+            }
         }
-        out[(size_t)t * nvec + v] = acc;
+        if (OUT_BF16) {
+            uint2 pk;
+            *reinterpret_cast<__nv_bfloat162*>(&pk.x) = __floats2bfloat162_rn(acc.x, acc.y);
+            *reinterpret_cast<__nv_bfloat162*>(&pk.y) = __floats2bfloat162_rn(acc.z, acc.w);
+            reinterpret_cast<uint2*>(out)[(size_t)t * nvec + v] = pk;
+        } else {
+            reinterpret_cast<float4*>(out)[(size_t)t * nvec + v] = acc;
+        }
     }
 }
 
@@ -190,11 +207,15 @@ dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const floa
 }
 
 dsmoe_status launch_combine(const dsmoe_layer_desc& p, const void* yp, const float* row_gate, const int32_t* token_rows,
-                            const int32_t* k_t, void* out, cudaStream_t s) {
+                            const int32_t* k_t, void* out, cudaStream_t s, bool yp_f32) {
     if (p.T == 0) return DSMOE_OK;
     const int W = width_of(p);
     const int64_t amax = (int64_t)amax_of(p);
-    if (p.dtype == DSMOE_BF16) {
+    if (yp_f32 && p.dtype == DSMOE_BF16 && !p.out_fp32) {
+        combine_f32_kernel<true><<<p.T, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t, out, p.d, W, amax);
+    } else if (yp_f32) {
+        combine_f32_kernel<false><<<p.T, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t, out, p.d, W, amax);
+    } else if (p.dtype == DSMOE_BF16) {
         if (p.out_fp32)
             combine_bf16_kernel<true><<<p.T, 128, 0, s>>>(static_cast<const uint4*>(yp), row_gate, token_rows, k_t, out,
                                                          p.d, W, amax);
@@ -202,8 +223,7 @@ dsmoe_status launch_combine(const dsmoe_layer_desc& p, const void* yp, const flo
             combine_bf16_kernel<false><<<p.T, 128, 0, s>>>(static_cast<const uint4*>(yp), row_gate, token_rows, k_t, out,
                                                           p.d, W, amax);
     } else {
-        combine_f32_kernel<<<p.T, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t,
-                                               static_cast<float4*>(out), p.d, W, amax);
+        combine_f32_kernel<false><<<p.T, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t, out, p.d, W, amax);
     }
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;

@@ -142,7 +142,8 @@ def test_permute_skips_rows_that_inconsistent_offsets_would_put_out_of_range():
     assert np.all(to_np(row_token)[amax:] == -9)
 
 
-# ---------------------------------------------------------------- aggregation inside the down-projection (fuse_combine = 1)
+# ---------------------------------------------------------------- where the aggregation runs: inside the down-projection
+# (fuse_combine = 1) or as a second kernel over fp32 gate-weighted rows (2); 0 lets the library choose by H
 
 FUSED = [
     dict(T=300, d=64, H=64, E=16, mode=gi.MODE_THRESHOLD, eps=0.5),                      # most tokens select nothing
@@ -156,9 +157,10 @@ FUSED = [
 ]
 
 
+@pytest.mark.parametrize("fuse", [1, 2], ids=["inside", "separate"])
 @pytest.mark.parametrize("case", FUSED, ids=[str(i) for i in range(len(FUSED))])
-def test_aggregation_inside_the_down_projection(case):
-    s = gi.LayerSpec(f"fused{FUSED.index(case)}", dtype="bf16", router_gain=5.0, fuse_combine=1, **case)
+def test_aggregation_inside_the_down_projection(case, fuse):
+    s = gi.LayerSpec(f"fused{FUSED.index(case)}", dtype="bf16", router_gain=5.0, fuse_combine=fuse, **case)
     r = layer_parity(s)
     assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
     L = r["layer"]
@@ -170,9 +172,10 @@ def test_aggregation_inside_the_down_projection(case):
         assert (mask == 0).any() and np.all(a[mask == 0] == 0.0)
 
 
-@pytest.mark.parametrize("cfg,kw,n", [("c3", {}, 256), ("c5", dict(eps=0.1), 512)], ids=["c3", "c5_eps0.1"])
-def test_aggregation_inside_the_down_projection_full_size(cfg, kw, n):
-    s = gi.spec(cfg, fuse_combine=1, **kw)
+@pytest.mark.parametrize("cfg,kw,n,fuse", [("c3", {}, 256, 2), ("c5", dict(eps=0.1), 512, 2), ("c5", dict(eps=0.1), 512, 1)],
+                         ids=["c3_separate", "c5_eps0.1_separate", "c5_eps0.1_inside"])
+def test_both_aggregation_paths_full_size(cfg, kw, n, fuse):
+    s = gi.spec(cfg, fuse_combine=fuse, **kw)
     r = layer_parity(s, sample=n)
     assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
     if cfg == "c3":
