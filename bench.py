@@ -252,7 +252,8 @@ def kernels_per_step(s, decode):
     if s.mode == gi.MODE_ALL:
         return router + 2                          # up, down
     # chunk count, finalize, permute index, up, down, and the aggregation unless it runs inside the down-projection
-    fused = s.fuse_combine == 1 or (s.fuse_combine == 0 and s.H >= 1024)      # the library's rule (dsmoe.h)
+    fused = s.fuse_combine == 1 or (s.fuse_combine == 0 and s.mode == gi.MODE_TOPK and s.H >= 1024 and
+                                    s.T * min(s.K, s.E) >= 1024 * s.E)        # the library's rule (dsmoe.h)
     return router + 3 + 2 + (0 if fused else 1)
 
 
@@ -340,9 +341,16 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
             step(0)
         run_step = lambda i, want=False: g.replay()     # noqa: E731
 
-    # ---- device-resident timed region: `value` comes from this loop, which holds nothing but the steps
+    # ---- device-resident timed region.  The library's event pairs around the dominant kernel's launches cost a few
+    # microseconds of stream time per step.  Prefill and dense steps (milliseconds) carry them in the timed loop itself:
+    # the kernel times are then those of the very steps that give `value`.  Decode steps (tens of microseconds) are
+    # timed clean, and the same un-synchronised loop runs once more with the event pairs for the kernel times.
     for i in range(max(warmup, 3)):
         run_step(i)
+    n_pairs = 0 if graph else steps * calls_per_step * timed_per_call
+    events_in_value_loop = n_pairs > 0 and not decode
+    if events_in_value_loop:
+        dm.dsmoe_timing_enable(n_pairs)
     sampler = ClockSampler(sampler_index)
     barrier()
     sampler.start()
@@ -355,12 +363,11 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.finish()
     value, ms_total, world = job_throughput(dist, ms_total, s.T * steps)
-    # ---- the same loop once more, as un-synchronised as the first, with the library's event pairs around the
-    # dominant kernel's launches (an event pair costs a few microseconds of stream time per step, which is why it is
-    # not in the loop that gives `value`); the kernel times fit inside this loop's own step time by construction
-    n_pairs = 0 if graph else steps * calls_per_step * timed_per_call
-    durs, ms_evented = np.zeros(0), None
-    if n_pairs:
+    durs, ms_evented = np.zeros(0), ms_total / steps
+    if events_in_value_loop:
+        durs = np.array(dm.dsmoe_timing_read(n_pairs))
+        dm.dsmoe_timing_enable(0)
+    elif n_pairs:
         dm.dsmoe_timing_enable(n_pairs)
         barrier()
         e0.record()

@@ -91,7 +91,8 @@ typedef struct {
                                     through L2 and is hidden only when the experts are wide);
                                  2: the epilogue stores the gate-weighted outputs as fp32 rows and a
                                     second kernel adds a token's rows;
-                                 0: the library chooses: 1 for H >= 1024, else 2.               */
+                                 0: the library chooses: 1 for a top-K selection with H >= 1024 and
+                                    T*K >= 1024*E (wide experts, many row tiles per expert), else 2. */
 } dsmoe_layer_desc;
 
 /* A void* stands for the caller's cudaStream_t so that this header needs no CUDA include. */
@@ -254,6 +255,36 @@ typedef struct {
 
 dsmoe_status dsmoe_stats(const dsmoe_layer_desc* desc, const float* scores, const uint64_t* mask,
                          dsmoe_selection_stats* stats, dsmoe_stream stream);
+
+/*
+ * Mutual-information loss of the router ("Mutual Information Loss" paragraph, Eq. 4-6) over the T tokens of
+ * the call, natural logarithms:  p(e_i) = mean_t scores[t,i];  H(e) = -sum_i p(e_i) log p(e_i);
+ * H(e|X_t) = -sum_i scores[t,i] log scores[t,i];  L_MI = -H(e) + mean_t H(e|X_t).
+ *   scores [T,E] fp32: read.  loss3 [3] fp32 (device): L_MI, H(e), mean_t H(e|X_t).
+ *   grad [T,E] fp32 or NULL: dL_MI/dscores[t,i] = (log p(e_i) - log scores[t,i]) / T.
+ *   Sums are taken in double precision in a fixed order (bit-reproducible).  T >= 1.
+ *   workspace: at least dsmoe_workspace_size_stages bytes.
+ */
+dsmoe_status dsmoe_mi_loss(const dsmoe_layer_desc* desc, const float* scores, float* loss3, float* grad,
+                           void* workspace, size_t ws_bytes, dsmoe_stream stream);
+
+/*
+ * Gradients of dense training ("Dense Training" paragraph, Eq. 3) for a given gradient dO of the layer
+ * output:  grad S_j = <e_j(X), dO> for every expert j, and grad e_j(X) = S_j dO, which is returned one
+ * linear step further down, at the expert's hidden activation a_j = GeLU(X.W1[j]) (e_j(X) = a_j.W2[j]):
+ * dA[t, j*H + k] = S_j * sum_c dO[t,c] * W2[j][k,c].  With mask (Eq. 2, sparse training: M marks the experts
+ * that were active in the forward pass) both are zero for the other experts.  Activations are recomputed
+ * from x (nothing of the forward pass has to be kept).
+ *   x [T,d], dO [T,d] dtype; W1 [E,d,H], W2 [E,H,d] dtype; scores [T,E] fp32; mask [T] uint64 or NULL: read.
+ *   dS [T,E] fp32; dA [T,E*H] dtype: written.
+ *   packed: NULL, or the buffer dsmoe_pack_weights filled from these weights (bf16): then the tensor cores
+ *   run (W1 may be NULL, W2 is still read in its natural layout) and the workspace must hold
+ *   dsmoe_workspace_size_packed bytes; without it a plain fp32-FMA kernel runs and needs no workspace.
+ */
+dsmoe_status dsmoe_dense_backward(const dsmoe_layer_desc* desc, const void* x, const void* W1, const void* W2,
+                                  const void* packed, const float* scores, const uint64_t* mask, const void* dO,
+                                  float* dS, void* dA, void* workspace, size_t ws_bytes, int32_t* dev_status,
+                                  dsmoe_stream stream);
 
 /*
  * Measurement aid (no counterpart in the paper): a ring of CUDA event pairs on the caller's stream.

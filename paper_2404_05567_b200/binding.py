@@ -24,6 +24,7 @@ EXPORTS = (
     "dsmoe_expert_mlp", "dsmoe_combine", "dsmoe_packed_size", "dsmoe_pack_weights",
     "dsmoe_layer_forward", "dsmoe_layer_forward_host", "dsmoe_timing_enable", "dsmoe_timing_read",
     "dsmoe_select_static", "dsmoe_workspace_size_packed", "dsmoe_workspace_size_stages", "dsmoe_stats",
+    "dsmoe_mi_loss", "dsmoe_dense_backward",
 )
 
 
@@ -189,6 +190,19 @@ def dsmoe_layer_forward_host(desc, x_host, x_dev, Wr, br, W1, W2, packed, out_de
                                           _ptr(workspace),
                                           ctypes.c_size_t(workspace.numel() if workspace is not None else 0),
                                           _ptr(dev_status), _stream(stream)), "dsmoe_layer_forward_host")
+
+
+def dsmoe_mi_loss(desc, scores, loss3, grad, workspace, stream=None):
+    _check(lib().dsmoe_mi_loss(ctypes.byref(desc), _ptr(scores), _ptr(loss3), _ptr(grad), _ptr(workspace),
+                               ctypes.c_size_t(workspace.numel() if workspace is not None else 0), _stream(stream)),
+           "dsmoe_mi_loss")
+
+
+def dsmoe_dense_backward(desc, x, W1, W2, packed, scores, mask, dO, dS, dA, workspace, dev_status=None, stream=None):
+    _check(lib().dsmoe_dense_backward(ctypes.byref(desc), _ptr(x), _ptr(W1), _ptr(W2), _ptr(packed), _ptr(scores),
+                                      _ptr(mask), _ptr(dO), _ptr(dS), _ptr(dA), _ptr(workspace),
+                                      ctypes.c_size_t(workspace.numel() if workspace is not None else 0),
+                                      _ptr(dev_status), _stream(stream)), "dsmoe_dense_backward")
 
 
 def dsmoe_timing_enable(n_pairs: int):

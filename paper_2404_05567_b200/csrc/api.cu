@@ -44,6 +44,7 @@ WsLayout ws_layout(const dsmoe_layer_desc& p) {
     L.batch_k = take(256);               // Threshold-TopK: the batch's K
     L.sync = take(64);                   // grid-barrier counters of the small-T kernel
     L.tile_done = take((size_t)kMaxExperts * ceil_div(p.d, 256) * 4);   // grouped down-projection: finished tiles per (expert, column range)
+    L.mi = take(mi_scratch_bytes());     // mutual-information loss: per-block partial sums
     L.row_token = take(amax * 4);
     L.row_gate = take(amax * 4);
     L.token_rows = take(T * (size_t)width_of(p) * 4);
@@ -59,8 +60,7 @@ WsLayout ws_layout(const dsmoe_layer_desc& p) {
     size_t h_bytes = 0;
     if (umma_supported(p)) {
         h_bytes = amax * p.H * 2;                                   // grouped: [Amax, H]
-        if (T * E * p.H * 2 > h_bytes && (p.mode == DSMOE_SELECT_ALL || p.T <= kSmallMaxT))
-            h_bytes = T * E * p.H * 2;                              // dense forward, small-T: [T, E*H]
+        if (T * E * p.H * 2 > h_bytes) h_bytes = T * E * p.H * 2;       // dense forward and backward, small-T: [T, E*H]
     }
     L.h = take(h_bytes);
     // grouped: the tokens' fp32 running sums [T,d] (aggregation inside the down-projection), or the gate-weighted
@@ -69,6 +69,8 @@ WsLayout ws_layout(const dsmoe_layer_desc& p) {
     // fp32 partial sums of the small-T path: (CTA, 2 column ranges, T, 256)
     L.partial = take(umma_supported(p) && p.T <= kSmallMaxT ? (size_t)kSmallMaxCtas * 2 * T * 256 * 4 : 0);
     L.router = take(router_umma_supported(p) ? router_umma_scratch(p) : 0);   // tensor-core router: split Wr, partial logits
+    // dense backward: the experts' hidden activations go to `h` ([T,E*H]); per-column-tile partial dot products here
+    L.bwd = take(umma_supported(p) ? T * E * ceil_div(p.H, 256) * 4 : 0);
     L.total_packed = off;
     L.total = L.total_plain > L.total_packed ? L.total_plain : L.total_packed;
     return L;
@@ -304,6 +306,36 @@ dsmoe_status dsmoe_stats(const dsmoe_layer_desc* desc, const float* scores, cons
     DSMOE_TRY(check_desc(desc));
     if (!stats || (desc->T > 0 && (!scores || !mask))) return DSMOE_ERR_INVALID_ARG;
     return launch_stats(*desc, scores, mask, stats, (cudaStream_t)stream);
+}
+
+dsmoe_status dsmoe_mi_loss(const dsmoe_layer_desc* desc, const float* scores, float* loss3, float* grad,
+                           void* workspace, size_t ws_bytes, dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    if (desc->T == 0 || !scores || !loss3) return DSMOE_ERR_INVALID_ARG;
+    const WsLayout L = ws_layout(*desc);
+    if (!workspace || ws_bytes < L.stage_total) return DSMOE_ERR_WORKSPACE;
+    return launch_mi_loss(*desc, scores, loss3, grad, static_cast<char*>(workspace) + L.mi, (cudaStream_t)stream);
+}
+
+dsmoe_status dsmoe_dense_backward(const dsmoe_layer_desc* desc, const void* x, const void* W1, const void* W2,
+                                  const void* packed, const float* scores, const uint64_t* mask, const void* dO,
+                                  float* dS, void* dA, void* workspace, size_t ws_bytes, int32_t* dev_status,
+                                  dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    if (desc->T == 0) return DSMOE_OK;
+    if (!x || !W2 || !scores || !dO || !dS || !dA) return DSMOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(W2) || !aligned16(dO) || !aligned16(dA)) return DSMOE_ERR_INVALID_ARG;
+    if (packed && desc->dtype != DSMOE_BF16) return DSMOE_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (packed && umma_supported(*desc)) {
+        const WsLayout L = ws_layout(*desc);
+        if (!workspace || ws_bytes < L.total_packed || !aligned16(workspace)) return DSMOE_ERR_WORKSPACE;
+        char* ws = static_cast<char*>(workspace);
+        return launch_dense_backward(*desc, x, W2, packed, scores, mask, dO, dS, dA, ws + L.h,
+                                     reinterpret_cast<float*>(ws + L.bwd), dev_status, s);
+    }
+    if (!W1 || !aligned16(W1)) return packed ? DSMOE_ERR_UNSUPPORTED : DSMOE_ERR_INVALID_ARG;
+    return launch_dense_backward_plain(*desc, x, W1, W2, scores, mask, dO, dS, dA, s);
 }
 
 dsmoe_status dsmoe_timing_enable(int n_pairs) {

@@ -48,10 +48,10 @@ static inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; 
 //                              sum of the expert outputs), partial (small-T), router (split Wr, partial logits)
 // total_packed = bytes a call with packed weights needs; total = the maximum over both kinds of call.
 struct WsLayout {
-    size_t scores, mask, k_t, counts, offsets, chunk_prefix, batch_k, sync, tile_done, row_token, row_gate, token_rows;
+    size_t scores, mask, k_t, counts, offsets, chunk_prefix, batch_k, sync, tile_done, mi, row_token, row_gate, token_rows;
     size_t stage_total;
     size_t xp, h_plain, yp;                 // plain path
-    size_t h, acc, partial, router;         // tensor-core paths
+    size_t h, acc, partial, router, bwd;    // tensor-core paths
     size_t total_plain, total_packed, total;
 };
 WsLayout ws_layout(const dsmoe_layer_desc& p);
@@ -88,8 +88,13 @@ dsmoe_status launch_combine(const dsmoe_layer_desc& p, const void* yp, const flo
                             const int32_t* token_rows, const int32_t* k_t, void* out, cudaStream_t s,
                             bool yp_f32 = false);
 // Whether dsmoe_layer_forward's tensor-core grouped path aggregates inside the down-projection (see dsmoe.h)
+// The library's own choice (fuse_combine == 0): inside only where it was measured to be as fast as the second
+// kernel -- wide experts (a long enough mainloop to hide the read-modify-write of the sums) and a top-K selection
+// with at least eight row tiles per expert on average (few tiles per expert make consecutive experts' tiles, which
+// must take turns on the same sums, run at the same time).
 static inline bool fuses_combine(const dsmoe_layer_desc& p) {
-    return p.fuse_combine == 1 || (p.fuse_combine == 0 && p.H >= 1024);
+    if (p.fuse_combine != 0) return p.fuse_combine == 1;
+    return p.mode == DSMOE_SELECT_TOPK && p.H >= 1024 && (long long)p.T * width_of(p) >= 1024ll * p.E;
 }
 dsmoe_status launch_pack(const dsmoe_layer_desc& p, const void* W1, const void* W2, void* packed,
                          cudaStream_t s);
@@ -136,5 +141,16 @@ dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const 
 dsmoe_status launch_layer_umma(const dsmoe_layer_desc& p, const void* x, const void* packed, const float* scores,
                                const uint64_t* mask, const int32_t* k_t, int32_t* counts_out, void* out, char* ws,
                                const WsLayout& L, int32_t* dev_status, cudaStream_t s, bool* done);
+
+// ---- training.cu / mlp_umma.cu : the training side (Eq. 2-6)
+size_t mi_scratch_bytes();
+dsmoe_status launch_mi_loss(const dsmoe_layer_desc& p, const float* scores, float* out3, float* grad, char* scratch,
+                            cudaStream_t s);
+dsmoe_status launch_dense_backward_plain(const dsmoe_layer_desc& p, const void* x, const void* W1, const void* W2,
+                                         const float* scores, const uint64_t* mask, const void* dO, float* dS, void* dA,
+                                         cudaStream_t s);
+dsmoe_status launch_dense_backward(const dsmoe_layer_desc& p, const void* x, const void* W2, const void* packed,
+                                   const float* scores, const uint64_t* mask, const void* dO, float* dS, void* dA,
+                                   void* act, float* dot_part, int32_t* dev_status, cudaStream_t s);
 
 }  // namespace dsmoe

@@ -50,7 +50,7 @@ constexpr size_t SMEM_GEMM_CMB_BYTES = SMEM_GEMM_BYTES + (size_t)CMB_WARPS * 32 
 static_assert(SMEM_GEMM_CMB_BYTES <= 227 * 1024, "shared memory of one CTA");
 
 enum { GEMM_GROUPED = 0, GEMM_DENSE_UP = 1, GEMM_DENSE_DOWN = 2 };
-enum { EPI_GELU = 0, EPI_STORE = 1, EPI_COMBINE = 2 };
+enum { EPI_GELU = 0, EPI_STORE = 1, EPI_COMBINE = 2, EPI_BWD = 3 };
 constexpr int kUpUnit = 16;          // small-T up-projection: weight rows per work unit
 constexpr int kUpTileUnits = 16;     // ... and units per tile (256 rows)
 constexpr int kRouterBatch = 12;     // rows of Wr a router thread loads at once
@@ -93,6 +93,14 @@ struct GemmParams {
     float* acc;
     int* tile_done;          // [E][column ranges], zero at launch: epilogue warps that have finished a tile
     int tokens;
+    // B given in its natural layout [E][n][k] (k contiguous) instead of the packed block-major one
+    int b_plain;
+    // backward of the dense forward (epi == EPI_BWD, tiles as in GEMM_DENSE_UP): the accumulator holds
+    // G = dO.W2[e]^T for (token, hidden unit); the epilogue writes out = gate * G (the gradient at the hidden
+    // activation, Eq. 3's S_j dO passed through W2[e]) and the row's partial <act, G> over the tile's columns to
+    // dot_part[(token * E + e) * column_tiles + column_tile] (Eq. 3's <e_j(X), dO>, see launch_dense_backward)
+    const __nv_bfloat16* act;   // [rows, E * n_per_expert] hidden activations GeLU(x.W1[e])
+    float* dot_part;
 };
 
 // Tensor maps of one packed weight tensor [E, n, k] with boxes of 16, 32, 64, 128 and 256 rows: a tile of
@@ -164,12 +172,12 @@ __device__ __forceinline__ int wrow(int kb, int n0, int N) { return kb * N + n0;
 
 // Weight rows [row0, row0 + rows) of expert e (see wrow): power-of-two boxes, largest first.
 __device__ __forceinline__ void load_weight_rows(const BMaps* maps, uint32_t dst, uint32_t bar, int row0, int rows,
-                                                 int e) {
+                                                 int e, int x0 = 0) {
     int done = 0;
 #pragma unroll
     for (int lvl = 4; lvl >= 0; --lvl) {
         if ((rows - done) >= (16 << lvl)) {
-            ptx::tma_load_3d(dst + done * (BK * 2), &maps->m[lvl], bar, 0, row0 + done, e);
+            ptx::tma_load_3d(dst + done * (BK * 2), &maps->m[lvl], bar, x0, row0 + done, e);
             done += 16 << lvl;
         }
     }
@@ -325,9 +333,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (!P.gather) ptx::tma_load_2d(smA + s * A_STAGE_BYTES, &tmA, bar, a_col, t.row0);
                     // full-width tiles take the one 256-row copy directly (measurably faster than walking the
                     // box sizes); only a ragged last column tile needs the decomposition
-                    const int b_row = wrow(b_k / BK, t.n0, P.n_per_expert);
-                    if (t.bn == BN) ptx::tma_load_3d(smB + s * B_STAGE_BYTES, &tmB.m[4], bar, 0, b_row, b_e);
-                    else load_weight_rows(&tmB, smB + s * B_STAGE_BYTES, bar, b_row, t.bn, b_e);
+                    const int b_x = P.b_plain ? b_k : 0;
+                    const int b_row = P.b_plain ? t.n0 : wrow(b_k / BK, t.n0, P.n_per_expert);
+                    if (t.bn == BN) ptx::tma_load_3d(smB + s * B_STAGE_BYTES, &tmB.m[4], bar, b_x, b_row, b_e);
+                    else load_weight_rows(&tmB, smB + s * B_STAGE_BYTES, bar, b_row, t.bn, b_e, b_x);
                     if (++s == STAGES) {
                         s = 0;
                         ph ^= 1u;
@@ -537,6 +546,51 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     __threadfence();                       // the warp's sums are visible before its arrival is
                     atomicAdd(P.tile_done + t.e * ntn + nt, 1);
                 }
+                if (++acc == 2) {
+                    acc = 0;
+                    aph ^= 1u;
+                }
+                continue;
+            }
+            if (P.epi == EPI_BWD) {
+                const bool active = valid && (!P.sel_mask || ((P.sel_mask[grow] >> t.e) & 1ull));   // Eq. 2's mask M
+                const float gs = active ? g : 0.f;
+                float dot = 0.f;
+                for (int c = 0; warp_has_rows && c < t.bn; c += 32) {
+                    const long long o = grow * P.ld_out + t.out_col0 + c;
+                    uint4 av[4];
+                    if (active) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) av[j] = __ldg(reinterpret_cast<const uint4*>(P.act + o) + j);
+                    }
+                    uint32_t r[32];
+                    ptx::tmem_ld32(taddr + (uint32_t)c, r);
+                    ptx::tmem_ld_wait();
+                    if (!valid) continue;
+                    uint4 pk[4];
+                    __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
+                    const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(av);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float g0 = __uint_as_float(r[2 * j]), g1 = __uint_as_float(r[2 * j + 1]);
+                        if (active) {
+                            const float2 a = __bfloat1622float2(ah[j]);
+                            dot = fmaf(a.x, g0, dot);
+                            dot = fmaf(a.y, g1, dot);
+                        }
+                        hv[j] = __floats2bfloat162_rn(gs * g0, gs * g1);
+                    }
+                    uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) + o);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) dst[j] = pk[j];
+                }
+                if (valid) {
+                    const int ntn = (P.n_per_expert + BN - 1) / BN;
+                    P.dot_part[(grow * P.E + t.e) * ntn + t.n0 / BN] = active ? dot : 0.f;
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.tempty[acc]));
                 if (++acc == 2) {
                     acc = 0;
                     aph ^= 1u;
@@ -1601,6 +1655,20 @@ dsmoe_status make_map_3d(CUtensorMap* m, const void* ptr, uint64_t E, uint64_t n
     return r == CUDA_SUCCESS ? DSMOE_OK : DSMOE_ERR_CUDA;
 }
 
+// weights in their natural layout, E matrices [n, k] with k contiguous: bf16 [E][n][k]; box {64 of k, box_n, 1}
+dsmoe_status make_map_3d_plain(CUtensorMap* m, const void* ptr, uint64_t E, uint64_t n, uint64_t k, uint32_t box_n) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return DSMOE_ERR_CUDA;
+    const cuuint64_t dims[3] = {k, n, E};
+    const cuuint64_t strides[2] = {k * 2, n * k * 2};
+    const cuuint32_t box[3] = {BK, box_n, 1};
+    const cuuint32_t es[3] = {1, 1, 1};
+    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DSMOE_OK : DSMOE_ERR_CUDA;
+}
+
 dsmoe_status make_bmaps16(BMaps16* b, const void* ptr, uint64_t E, uint64_t n, uint64_t k) {
     for (int i = 0; i < 16; ++i) DSMOE_TRY(make_map_3d(&b->m[i], ptr, E, n, k, 16u * (i + 1)));
     return DSMOE_OK;
@@ -1664,6 +1732,18 @@ dsmoe_status cached_bmaps(const BMaps** out, const void* ptr, uint64_t E, uint64
     if (!m) {
         BMaps tmp;
         DSMOE_TRY(make_bmaps(&tmp, ptr, E, n, kk));
+        m = g_bmaps.slot(k);
+        *m = tmp;
+    }
+    *out = m;
+    return DSMOE_OK;
+}
+dsmoe_status cached_bmaps_plain(const BMaps** out, const void* ptr, uint64_t E, uint64_t n, uint64_t kk) {
+    const MapKey k{ptr, E, n, kk, 3};
+    BMaps* m = g_bmaps.find(k);
+    if (!m) {
+        BMaps tmp;
+        for (int lvl = 0; lvl < 5; ++lvl) DSMOE_TRY(make_map_3d_plain(&tmp.m[lvl], ptr, E, n, kk, 16u << lvl));
         m = g_bmaps.slot(k);
         *m = tmp;
     }
@@ -1969,6 +2049,50 @@ dsmoe_status launch_layer_umma(const dsmoe_layer_desc& p, const void* x, const v
         DSMOE_TRY(launch_finalize(p, mask, counts, offsets, reinterpret_cast<int32_t*>(ws + L.chunk_prefix), counts_out, s));
     }
     *done = true;
+    return DSMOE_OK;
+}
+
+// dS[t,e] = the column tiles' partial sums added in ascending order
+__global__ void __launch_bounds__(256) bwd_finish_kernel(const float* __restrict__ part, float* __restrict__ dS, long long n,
+                                                         int ntn) {
+    const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (i >= n) return;
+    float v = 0.f;
+    for (int j = 0; j < ntn; ++j) v += part[i * ntn + j];
+    dS[i] = v;
+}
+
+// Gradients of dense training (Eq. 3; Eq. 2 with a mask) on the tensor cores, by recomputation from x:
+//   act = GeLU(x.W1[e])            the dense forward's up-projection without the gate     [T, E*H] bf16
+//   G   = dO.W2[e]^T               one GEMM over d per expert, W2 read in its natural [H, d] layout
+//   dA  = S[t,e] * G,  dS[t,e] = <act[t,e,:], G[t,e,:]>  (= <e_e(x_t), dO_t>)            in that GEMM's epilogue
+dsmoe_status launch_dense_backward(const dsmoe_layer_desc& p, const void* x, const void* W2, const void* packed,
+                                   const float* scores, const uint64_t* mask, const void* dO, float* dS, void* dA,
+                                   void* act, float* dot_part, int32_t* dev_status, cudaStream_t s) {
+    if (p.T == 0) return DSMOE_OK;
+    if (!umma_supported(p)) return DSMOE_ERR_UNSUPPORTED;
+    const __nv_bfloat16* w1t = static_cast<const __nv_bfloat16*>(packed);
+    const CUtensorMap *mX, *mdO;
+    const BMaps *mB1, *mB2;
+    DSMOE_TRY(cached_map_2d(&mX, x, p.T, p.d, BM));
+    DSMOE_TRY(cached_bmaps(&mB1, w1t, p.E, p.H, p.d));
+    DSMOE_TRY(cached_map_2d(&mdO, dO, p.T, p.d, BM));
+    DSMOE_TRY(cached_bmaps_plain(&mB2, W2, p.E, p.H, p.d));
+    const long long ld = (long long)p.E * p.H;
+    GemmParams up{};
+    up.mode = GEMM_DENSE_UP; up.epi = EPI_GELU; up.E = p.E; up.n_per_expert = p.H; up.k_per_expert = p.d; up.rows = p.T;
+    up.out = act; up.ld_out = ld; up.dev_status = dev_status;
+    GemmParams bw = up;
+    bw.epi = EPI_BWD; bw.gate = scores; bw.sel_mask = mask; bw.out = dA; bw.b_plain = 1;
+    bw.act = static_cast<const __nv_bfloat16*>(act); bw.dot_part = dot_part;
+    const int ntn = ceil_div(p.H, BN);
+    const int tiles = ceil_div(p.T, BM) * ntn * p.E;
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    DSMOE_TRY(launch_gemm(*mX, *mB1, up, grid, s));
+    DSMOE_TRY(launch_gemm(*mdO, *mB2, bw, grid, s));
+    const long long n = (long long)p.T * p.E;
+    bwd_finish_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(dot_part, dS, n, ntn);
+    DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
 }
 
