@@ -53,7 +53,14 @@ def _backward_case(s, packed, masked, sample=None):
     dS_g = dS.cpu().numpy() if ids is None else dS.cpu().numpy()[ids]
     dA_g = np_f32(dA).reshape(s.T, s.E, s.H)
     dA_g = dA_g if ids is None else dA_g[ids]
-    e_s, e_a = rel_err(dS_g, dS_ref), rel_err(dA_g.reshape(len(dS_g), -1), dA_ref.reshape(len(dS_g), -1))
+    e_s = rel_err(dS_g, dS_ref)
+    # dA is stored in the layer's type.  For bf16 that last rounding alone is up to 2^-9 of the value, more than the
+    # whole tolerance for an element beyond 5 sigma, so it is allowed for separately: the bar is on
+    # |dA - ref| - 2^-8 |ref| (the rounding of the stored value, with a factor 2 of slack), relative to RMS(ref)
+    a_g, a_r = dA_g.reshape(len(dS_g), -1).astype(np.float64), dA_ref.reshape(len(dS_g), -1)
+    slack = (2.0 ** -8) * np.abs(a_r) if s.dtype == "bf16" else 0.0
+    rms = float(np.sqrt(np.mean(a_r ** 2)))
+    e_a = float(np.max(np.maximum(np.abs(a_g - a_r) - slack, 0.0))) / max(rms, 1e-300)
     record("dense_backward", name=s.name, T=s.T, d=s.d, H=s.H, E=s.E, dtype=s.dtype, packed=bool(L.packed is not None),
            masked=masked, err_dS=e_s, err_dA=e_a, tokens_compared=int(len(dS_g)))
     if masked:
