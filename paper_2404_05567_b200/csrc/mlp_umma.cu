@@ -16,9 +16,8 @@
 // small_layer_kernel: the whole layer for a handful of tokens (decode) in one cooperative launch.
 #include "common.cuh"
 #include "router_device.cuh"
+#include "tensor_maps.cuh"
 #include "umma.cuh"
-
-#include <stdlib.h>
 
 namespace dsmoe {
 
@@ -101,18 +100,6 @@ struct GemmParams {
     // dot_part[(token * E + e) * column_tiles + column_tile] (Eq. 3's <e_j(X), dO>, see launch_dense_backward)
     const __nv_bfloat16* act;   // [rows, E * n_per_expert] hidden activations GeLU(x.W1[e])
     float* dot_part;
-};
-
-// Tensor maps of one packed weight tensor [E, n, k] with boxes of 16, 32, 64, 128 and 256 rows: a tile of
-// any width (a multiple of 16 rows) is fetched with at most five copies, largest first.
-struct BMaps {
-    CUtensorMap m[5];
-};
-
-// ... and, for the small-T up-projection whose tile widths are arbitrary multiples of 16, one map per height
-// 16, 32, ..., 256, so that a tile (or each of its two parts) is a single copy.
-struct BMaps16 {
-    CUtensorMap m[16];
 };
 
 struct Tile {
@@ -1609,169 +1596,6 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 
 // ---------------------------------------------------------------- host side
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-// bf16 [rows, cols] row-major, box {64 cols, box_rows}, 128-byte swizzle
-dsmoe_status make_map_2d(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return DSMOE_ERR_CUDA;
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {BK, box_rows};
-    const cuuint32_t es[2] = {1, 1};
-    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? DSMOE_OK : DSMOE_ERR_CUDA;
-}
-
-// packed weights of E experts, n output columns, reduction length k: bf16 [E][k / 64][n][64], seen as
-// [E][(k / 64) * n][64]; box {64, box_n, 1}, 128-byte swizzle
-dsmoe_status make_map_3d(CUtensorMap* m, const void* ptr, uint64_t E, uint64_t n, uint64_t k, uint32_t box_n) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return DSMOE_ERR_CUDA;
-    const cuuint64_t dims[3] = {BK, (k / BK) * n, E};
-    const cuuint64_t strides[2] = {BK * 2, n * k * 2};
-    const cuuint32_t box[3] = {BK, box_n, 1};
-    const cuuint32_t es[3] = {1, 1, 1};
-    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? DSMOE_OK : DSMOE_ERR_CUDA;
-}
-
-// weights in their natural layout, E matrices [n, k] with k contiguous: bf16 [E][n][k]; box {64 of k, box_n, 1}
-dsmoe_status make_map_3d_plain(CUtensorMap* m, const void* ptr, uint64_t E, uint64_t n, uint64_t k, uint32_t box_n) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return DSMOE_ERR_CUDA;
-    const cuuint64_t dims[3] = {k, n, E};
-    const cuuint64_t strides[2] = {k * 2, n * k * 2};
-    const cuuint32_t box[3] = {BK, box_n, 1};
-    const cuuint32_t es[3] = {1, 1, 1};
-    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? DSMOE_OK : DSMOE_ERR_CUDA;
-}
-
-dsmoe_status make_bmaps16(BMaps16* b, const void* ptr, uint64_t E, uint64_t n, uint64_t k) {
-    for (int i = 0; i < 16; ++i) DSMOE_TRY(make_map_3d(&b->m[i], ptr, E, n, k, 16u * (i + 1)));
-    return DSMOE_OK;
-}
-
-// the five box heights of one packed weight tensor
-dsmoe_status make_bmaps(BMaps* b, const void* ptr, uint64_t E, uint64_t n, uint64_t k) {
-    for (int lvl = 0; lvl < 5; ++lvl) DSMOE_TRY(make_map_3d(&b->m[lvl], ptr, E, n, k, 16u << lvl));
-    return DSMOE_OK;
-}
-
-int sm_count() {
-    DeviceState* st = nullptr;
-    return device_state(&st) == DSMOE_OK ? st->sm_count : 148;   // no device (host-only sizing): the B200's count
-}
-
-// Tensor maps depend only on the buffer and the shape, and encoding one is a driver call of a few microseconds
-// (a layer call needs up to 23): they are encoded once and found again by (address, shape).  A decode loop or a
-// serving loop calls with the same buffers every step.  Not thread-safe, like the rest of the host side.
-struct MapKey {
-    const void* ptr;
-    uint64_t a, b, c;
-    int kind;
-    bool operator==(const MapKey& o) const { return ptr == o.ptr && a == o.a && b == o.b && c == o.c && kind == o.kind; }
-};
-template <typename M, int N>
-struct MapCache {
-    MapKey key[N];
-    M map[N];
-    int n = 0, next = 0;
-    M* find(const MapKey& k) {
-        for (int i = 0; i < n; ++i)
-            if (key[i] == k) return &map[i];
-        return nullptr;
-    }
-    M* slot(const MapKey& k) {
-        const int i = n < N ? n++ : (next++ % N);
-        key[i] = k;
-        return &map[i];
-    }
-};
-MapCache<CUtensorMap, 256> g_maps2d;
-MapCache<BMaps, 128> g_bmaps;
-MapCache<BMaps16, 64> g_bmaps16;
-
-dsmoe_status cached_map_2d(const CUtensorMap** out, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
-    const MapKey k{ptr, rows, cols, box_rows, 0};
-    CUtensorMap* m = g_maps2d.find(k);
-    if (!m) {
-        CUtensorMap tmp;
-        DSMOE_TRY(make_map_2d(&tmp, ptr, rows, cols, box_rows));
-        m = g_maps2d.slot(k);
-        *m = tmp;
-    }
-    *out = m;
-    return DSMOE_OK;
-}
-dsmoe_status cached_bmaps(const BMaps** out, const void* ptr, uint64_t E, uint64_t n, uint64_t kk) {
-    const MapKey k{ptr, E, n, kk, 1};
-    BMaps* m = g_bmaps.find(k);
-    if (!m) {
-        BMaps tmp;
-        DSMOE_TRY(make_bmaps(&tmp, ptr, E, n, kk));
-        m = g_bmaps.slot(k);
-        *m = tmp;
-    }
-    *out = m;
-    return DSMOE_OK;
-}
-dsmoe_status cached_bmaps_plain(const BMaps** out, const void* ptr, uint64_t E, uint64_t n, uint64_t kk) {
-    const MapKey k{ptr, E, n, kk, 3};
-    BMaps* m = g_bmaps.find(k);
-    if (!m) {
-        BMaps tmp;
-        for (int lvl = 0; lvl < 5; ++lvl) DSMOE_TRY(make_map_3d_plain(&tmp.m[lvl], ptr, E, n, kk, 16u << lvl));
-        m = g_bmaps.slot(k);
-        *m = tmp;
-    }
-    *out = m;
-    return DSMOE_OK;
-}
-dsmoe_status cached_bmaps16(const BMaps16** out, const void* ptr, uint64_t E, uint64_t n, uint64_t kk) {
-    const MapKey k{ptr, E, n, kk, 2};
-    BMaps16* m = g_bmaps16.find(k);
-    if (!m) {
-        BMaps16 tmp;
-        DSMOE_TRY(make_bmaps16(&tmp, ptr, E, n, kk));
-        m = g_bmaps16.slot(k);
-        *m = tmp;
-    }
-    *out = m;
-    return DSMOE_OK;
-}
-
-// Optional per-launch timing of the tensor-core kernels (a measurement aid for benchmarks): a ring of CUDA event
-// pairs; every timed launch takes the next pair until the ring is full.  The events sit on the caller's stream, so a
-// benchmark can leave them inside its un-synchronised step loop and read all durations afterwards.
-struct Timing {
-    bool on = false;
-    int n = 0, cap = 0;
-    cudaEvent_t *start = nullptr, *stop = nullptr;
-} g_timing;
-
 dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams& P, int grid, cudaStream_t s,
                          bool may_time = true) {
     DeviceState* st = nullptr;
@@ -1780,8 +1604,8 @@ dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams&
         DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_CMB_BYTES));
         st->attr_gemm = true;
     }
-    const bool timed = may_time && g_timing.on && g_timing.n < g_timing.cap;
-    if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
+    int timed = -1;
+    if (may_time) DSMOE_TRY(timing_begin(s, &timed));
     const int threads = (P.gather || P.epi == EPI_COMBINE) ? GATHER_THREADS : NUM_THREADS;
     if (P.epi == EPI_COMBINE) {
         // its epilogues wait for one another's tiles: every CTA must be resident
@@ -1792,7 +1616,7 @@ dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams&
         umma_gemm_kernel<<<grid, threads, SMEM_GEMM_BYTES, s>>>(a, b, P);
         DSMOE_CUDA_TRY(cudaGetLastError());
     }
-    if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.stop[g_timing.n++], s));
+    DSMOE_TRY(timing_end(s, timed));
     return DSMOE_OK;
 }
 
@@ -1874,35 +1698,6 @@ extern "C" __attribute__((visibility("default"))) int dsmoe_trace_read(unsigned 
     return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(unsigned long long) * 192 * 32);
 }
 #endif
-
-dsmoe_status timing_enable(int n_pairs) {
-    if (n_pairs > g_timing.cap) {
-        cudaEvent_t* a = static_cast<cudaEvent_t*>(realloc(g_timing.start, sizeof(cudaEvent_t) * n_pairs));
-        cudaEvent_t* b = static_cast<cudaEvent_t*>(realloc(g_timing.stop, sizeof(cudaEvent_t) * n_pairs));
-        if (a) g_timing.start = a;
-        if (b) g_timing.stop = b;
-        if (!a || !b) return DSMOE_ERR_CUDA;
-        for (int i = g_timing.cap; i < n_pairs; ++i) {
-            DSMOE_CUDA_TRY(cudaEventCreate(&g_timing.start[i]));
-            DSMOE_CUDA_TRY(cudaEventCreate(&g_timing.stop[i]));
-            g_timing.cap = i + 1;
-        }
-    }
-    g_timing.on = n_pairs > 0;
-    g_timing.n = 0;
-    return DSMOE_OK;
-}
-
-dsmoe_status timing_read(float* ms, int n_max, int* n) {
-    *n = 0;
-    for (int i = 0; i < g_timing.n && i < n_max; ++i) {
-        DSMOE_CUDA_TRY(cudaEventSynchronize(g_timing.stop[i]));
-        DSMOE_CUDA_TRY(cudaEventElapsedTime(&ms[i], g_timing.start[i], g_timing.stop[i]));
-        *n = i + 1;
-    }
-    g_timing.n = 0;
-    return DSMOE_OK;
-}
 
 bool umma_supported(const dsmoe_layer_desc& p) {
     return p.dtype == DSMOE_BF16 && (p.d % 64) == 0 && (p.H % 64) == 0;
@@ -2009,11 +1804,11 @@ dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const 
     DSMOE_CUDA_TRY(cudaMemsetAsync(P.sync, 0, 32, s));
     void* args[] = {const_cast<CUtensorMap*>(mX), const_cast<BMaps16*>(mW1), const_cast<CUtensorMap*>(mHg),
                     const_cast<BMaps*>(mW2), &P};
-    const bool timed = g_timing.on && g_timing.n < g_timing.cap;
-    if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.start[g_timing.n], s));
+    int timed = -1;
+    DSMOE_TRY(timing_begin(s, &timed));
     DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(small_layer_kernel), dim3(G), dim3(SMALL_THREADS),
                                                args, SMEM_BYTES, s));
-    if (timed) DSMOE_CUDA_TRY(cudaEventRecord(g_timing.stop[g_timing.n++], s));
+    DSMOE_TRY(timing_end(s, timed));
     return DSMOE_OK;
 }
 
