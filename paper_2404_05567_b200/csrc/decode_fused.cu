@@ -36,11 +36,19 @@ constexpr int FT_THREADS = 448;
 constexpr int FT_EPI = FT_THREADS - 64;          // router / epilogue threads
 constexpr int FT_N = 16;                         // token columns of every MMA
 constexpr int FT_UNIT = 16;                      // hidden units per work unit = reduction length of one down-projection MMA
-constexpr int FT_XBYTES = FT_N * 128;            // one 64-wide block of the tokens: 16 rows of 128 bytes
-constexpr int FT_SLOT = FT_XBYTES + 128 * 128;   // ring slot: tokens' block + 128 rows of W1, or 512 32-byte rows of W2
-constexpr int FT_STAGES = 8;
-constexpr int FT_RING = FT_STAGES * FT_SLOT;     // 144 KB in flight per SM
-constexpr int FT_DOWN_ROWS = 512;                // output columns per down-projection slot
+// The copy engine has only a few copies per SM under way at a time, whatever their size (about 4.5 per microsecond
+// from HBM), so every copy is made as large as a ring slot: up to 32 KB, which four slots turn into the memory's
+// full rate.  A narrow up-projection tile therefore brings several 64-wide blocks of d per copy, and a
+// down-projection copy brings up to 1024 output columns of one hidden unit.  The tokens are not copied per slot at
+// all: the router warps put them into shared memory once, as the MMA's N operand.
+constexpr int FT_SLOT = 32 * 1024;
+#ifndef DSMOE_FUSED_RING_SLOTS
+#define DSMOE_FUSED_RING_SLOTS 4
+#endif
+constexpr int FT_STAGES = DSMOE_FUSED_RING_SLOTS;
+constexpr int FT_RING = FT_STAGES * FT_SLOT;
+constexpr int FT_XBLOCK = 8 * 128;               // one 64-wide block of the tokens in shared memory: 8 rows of 128 bytes
+constexpr int FT_MAXTILES = 16;
 constexpr int FT_HG_BYTES = kFusedMaxUnits * FT_N * 32;
 constexpr int FT_TMEM_COLS = 512;
 constexpr int FT_ROUTER_BATCH = 12;              // rows of Wr a router thread loads at once
@@ -71,15 +79,32 @@ struct FShared {
     volatile int abort_flag;
     volatile int geo_ready;
     int n_act, u0, u1;                   // this CTA's units [u0, u1) of the n_act * H / 16 of the selected experts
+    // ... cut at the expert boundaries into up-projection tiles of at most 8 units (128 hidden units, the MMA's M):
+    // expert, first unit inside the expert, units, first unit counted from u0
+    int ntiles, tile_e[FT_MAXTILES], tile_iu0[FT_MAXTILES], tile_len[FT_MAXTILES], tile_ul0[FT_MAXTILES];
+    int nchain;                          // accumulators per tile (see the MMA issuer)
     int active[kMaxExperts];             // the selected experts, ascending
     uint64_t mask_s[kFusedMaxT];
     float score_s[kFusedMaxT][kMaxExperts];
+#ifdef DSMOE_TRACE
+    unsigned long long trace[32];
+#endif
 };
+#ifdef DSMOE_TRACE
+// Diagnostic build only (-DDSMOE_TRACE): per-CTA time stamps (globaltimer ns) of the kernel's milestones.
+__device__ unsigned long long g_trace_fused[192][32];
+#define TRACE(i) sh.trace[i] = ptx::globaltimer_ns()
+#else
+#define TRACE(i)
+#endif
 constexpr int FT_SHARED_BYTES = 4096;
 static_assert(sizeof(FShared) <= FT_SHARED_BYTES, "FShared must fit its slot");
-constexpr size_t FT_SMEM_BYTES = 1024 + (size_t)FT_RING + FT_HG_BYTES + FT_SHARED_BYTES + FT_RED_FLOATS * 4;
-static_assert(FT_SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
-static_assert(kFusedMaxT * FT_EPI * 16 <= FT_RING, "the router's scratch borrows the ring");
+// ring | tokens (d / 64 + 1 blocks) | gated activations | FShared | scratch of the final sum
+constexpr size_t ft_smem_bytes(int d) {
+    return 1024 + (size_t)FT_RING + (size_t)(d / 64 + 1) * FT_XBLOCK + FT_HG_BYTES + FT_SHARED_BYTES + FT_RED_FLOATS * 4;
+}
+static_assert(ft_smem_bytes(4096) <= 227 * 1024, "shared memory of one CTA");
+static_assert(kFusedMaxT * 16 * kMaxExperts * 4 <= FT_RING, "the router's scratch borrows the ring");
 
 __device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f)); }
 
@@ -136,20 +161,21 @@ __device__ __forceinline__ bool wait_geo(FShared& sh) {
 }
 
 __global__ void __launch_bounds__(FT_THREADS, 1)
-fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ BMaps16 tmW1,
-                    const __grid_constant__ BMapsK16 tmW2, const FusedParams P) {
+fused_decode_kernel(const __grid_constant__ BMapsUp tmW1, const __grid_constant__ BMapsDown tmW2, const FusedParams P) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    const uint32_t ring = base, hg_addr = base + FT_RING;
-    uint8_t* hg = smem + FT_RING;
-    FShared& sh = *reinterpret_cast<FShared*>(smem + FT_RING + FT_HG_BYTES);
-    float* red = reinterpret_cast<float*>(smem + FT_RING + FT_HG_BYTES + FT_SHARED_BYTES);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, T = P.T, E = P.E;
     const int upe = P.H / FT_UNIT;                       // units per expert
     const int nkb = P.d / 64;
+    const uint32_t xs_bytes = (uint32_t)(nkb + 1) * FT_XBLOCK;
+    const uint32_t ring = base, xs_addr = base + FT_RING, hg_addr = xs_addr + xs_bytes;
+    uint8_t* xs = smem + FT_RING;
+    uint8_t* hg = xs + xs_bytes;
+    FShared& sh = *reinterpret_cast<FShared*>(hg + FT_HG_BYTES);
+    float* red = reinterpret_cast<float*>(hg + FT_HG_BYTES + FT_SHARED_BYTES);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < FT_STAGES; ++s) {
@@ -161,9 +187,12 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         ptx::mbar_init(ptx::smem_u32(&sh.d2_full), 1);
         sh.abort_flag = 0;
         sh.geo_ready = 0;
+#ifdef DSMOE_TRACE
+        for (int i = 0; i < 32; ++i) sh.trace[i] = 0;
+        TRACE(0);
+#endif
         ptx::fence_barrier_init();
-        ptx::prefetch_tensormap(&tmX);
-        ptx::prefetch_tensormap(&tmW2.m[2]);
+        ptx::prefetch_tensormap(&tmW2.m);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), FT_TMEM_COLS);
@@ -178,59 +207,49 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         // ------------------------------------------------------------ TMA producer
         if (lane == 0 && wait_geo(sh)) {
             const uint64_t wpol = ptx::policy_evict_first();    // weights are read once: first to leave L2
-            const int u0 = sh.u0, u1 = sh.u1, nu = u1 - u0;
+            const int u0 = sh.u0, nu = sh.u1 - sh.u0;
             int s = 0;
             uint32_t ph = 0;
             bool alive = true;
-            // up-projection: M tiles of up to 8 units (128 hidden units), every 64-wide block of d
-            for (int mu0 = u0; alive && mu0 < u1; mu0 += 8) {
-                const int mu1 = min(u1, mu0 + 8);
-                for (int kb = 0; kb < nkb; ++kb) {
+            TRACE(3);
+            // up-projection: tile by tile, kbp reduction blocks per copy
+            for (int ti = 0; alive && ti < sh.ntiles; ++ti) {
+                const int len = sh.tile_len[ti], kbp = tmW1.kbp[len - 1];
+                for (int g = 0; g * kbp < nkb; ++g) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
                         alive = false;
                         break;
                     }
-                    const uint32_t bar = ptx::smem_u32(&sh.full[s]), slot = ring + s * FT_SLOT;
-                    ptx::mbar_expect_tx(bar, (uint32_t)(FT_XBYTES + (mu1 - mu0) * FT_UNIT * 128));
-                    ptx::tma_load_2d(slot, &tmX, bar, kb * 64, 0);
-                    // the tile's units, expert by expert (a run of units inside one expert is one copy)
-                    int off = 0;
-                    for (int u = mu0; u < mu1;) {
-                        const int ei = u / upe, iu = u % upe, len = min(mu1 - u, upe - iu);
-                        ptx::tma_load_3d_hint(slot + FT_XBYTES + off * (FT_UNIT * 128), &tmW1.m[len - 1], bar, 0,
-                                              wrow(kb, iu * FT_UNIT, P.H), sh.active[ei], wpol);
-                        off += len;
-                        u += len;
-                    }
+                    const uint32_t bar = ptx::smem_u32(&sh.full[s]);
+                    ptx::mbar_expect_tx(bar, (uint32_t)(kbp * len * FT_UNIT * 128));     // blocks past d arrive as zeros
+                    ptx::tma_load_4d_hint(ring + s * FT_SLOT, &tmW1.m[len - 1], bar, 0, sh.tile_iu0[ti] * FT_UNIT, g * kbp,
+                                          sh.tile_e[ti], wpol);
                     if (++s == FT_STAGES) {
                         s = 0;
                         ph ^= 1u;
                     }
                 }
             }
-            // down-projection: unit by unit, 512 output columns per slot
+            TRACE(14);
+            // down-projection: unit by unit, `ch` chunks of 256 output columns per copy
+            const int nch = P.d / 256, ch = tmW2.ch;
             for (int j = 0; alive && j < nu; ++j) {
                 const int u = u0 + j, e = sh.active[u / upe], hid = (u % upe) * FT_UNIT;
-                const int kb = hid / 64, sub = hid % 64;
-                for (int r = 0; r < P.d; r += FT_DOWN_ROWS) {
-                    const int rows = min(FT_DOWN_ROWS, P.d - r);
+                for (int cg = 0; cg * ch < nch; ++cg) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
                         alive = false;
                         break;
                     }
-                    const uint32_t bar = ptx::smem_u32(&sh.full[s]), slot = ring + s * FT_SLOT;
-                    ptx::mbar_expect_tx(bar, (uint32_t)rows * 32u);
-                    for (int done = 0; done < rows;) {
-                        const int rem = rows - done, lvl = rem >= 256 ? 2 : rem >= 128 ? 1 : 0;
-                        ptx::tma_load_3d_hint(slot + done * 32, &tmW2.m[lvl], bar, sub, wrow(kb, r + done, P.d), e, wpol);
-                        done += 64 << lvl;
-                    }
+                    const uint32_t bar = ptx::smem_u32(&sh.full[s]);
+                    ptx::mbar_expect_tx(bar, (uint32_t)(ch * 256 * 32));
+                    ptx::tma_load_5d_hint(ring + s * FT_SLOT, &tmW2.m, bar, hid % 64, 0, cg * ch, hid / 64, e, wpol);
                     if (++s == FT_STAGES) {
                         s = 0;
                         ph ^= 1u;
                     }
                 }
             }
+            TRACE(15);
             if (!alive) {
                 const uint64_t t0 = ptx::globaltimer_ns();   // copies already issued still land in this CTA's smem
                 while (ptx::globaltimer_ns() - t0 < 200000ull) {
@@ -240,25 +259,39 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0 && wait_geo(sh)) {
-            const int u0 = sh.u0, u1 = sh.u1, nu = u1 - u0;
+            const int nu = sh.u1 - sh.u0;
             const uint32_t idesc = ptx::make_idesc_bf16(128, FT_N);
             int s = 0;
             uint32_t ph = 0;
             bool alive = nu > 0;
-            // D1[m][k, t] = sum over d of W1 rows (M) x tokens (N); tile m sits at TMEM columns 16 m ..
-            int m = 0;
-            for (int mu0 = u0; alive && mu0 < u1; mu0 += 8, ++m) {
-                for (int kb = 0; kb < nkb; ++kb) {
+            // D1[tile][k, t] = sum over d of W1 rows (M) x tokens (N).  The M operand is read 128 rows deep whatever the
+            // tile's height: what lies beyond it in shared memory only reaches TMEM lanes that nobody looks at.
+            // Likewise the tokens' rows 8..15 (the next block's bytes).  These MMAs are tiny (128 x 16 x 16) and an
+            // MMA waits for the previous one into the same accumulator, so a tile's reduction over d is spread over
+            // `nchain` accumulators (64-wide block kb goes to accumulator kb % nchain, at TMEM columns
+            // 16 (tile nchain + kb % nchain) ..), which the epilogue adds up.
+            const int nchain = sh.nchain;
+            for (int ti = 0; alive && ti < sh.ntiles; ++ti) {
+                const int len = sh.tile_len[ti], kbp = tmW1.kbp[len - 1];
+                for (int g = 0; g * kbp < nkb; ++g) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&sh.full[s]), ph, &sh.abort_flag)) {
                         alive = false;
                         break;
                     }
                     ptx::tc_fence_after();
+#ifdef DSMOE_TRACE
+                    if (sh.trace[4] == 0) TRACE(4);
+#endif
                     const uint32_t slot = ring + s * FT_SLOT;
+                    for (int kbi = 0; kbi < kbp && g * kbp + kbi < nkb; ++kbi) {
+                        const int kb = g * kbp + kbi;
+                        const uint32_t a0 = slot + kbi * len * (FT_UNIT * 128), b0 = xs_addr + kb * FT_XBLOCK;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        ptx::umma_bf16(tmem_base + (uint32_t)(m * FT_N), ptx::make_desc_k_sw128(slot + FT_XBYTES + k * 32),
-                                       ptx::make_desc_k_sw128(slot + k * 32), idesc, (uint32_t)((kb | k) != 0));
+                        for (int k = 0; k < 4; ++k)
+                            ptx::umma_bf16(tmem_base + (uint32_t)((ti * nchain + kb % nchain) * FT_N),
+                                           ptx::make_desc_k_sw128(a0 + k * 32), ptx::make_desc_k_sw128(b0 + k * 32), idesc,
+                                           (uint32_t)(kb >= nchain || k != 0));
+                    }
                     ptx::umma_commit(ptx::smem_u32(&sh.empty[s]));
                     if (++s == FT_STAGES) {
                         s = 0;
@@ -266,6 +299,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                     }
                 }
             }
+            TRACE(5);
             if (alive) {
                 ptx::umma_commit(ptx::smem_u32(&sh.d1_full));
                 // the gated activations in shared memory (and D1 read out of TMEM: D2 takes its place)
@@ -273,17 +307,17 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                 ptx::tc_fence_after();
             }
             // D2[c][col, t] += W2 rows of unit j (M = 128 output columns of chunk c, K = 16) x hg of unit j (N)
+            const int nch = P.d / 256, ch = tmW2.ch;
             for (int j = 0; alive && j < nu; ++j) {
-                for (int r = 0; r < P.d; r += FT_DOWN_ROWS) {
-                    const int rows = min(FT_DOWN_ROWS, P.d - r);
+                for (int cg = 0; cg * ch < nch; ++cg) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&sh.full[s]), ph, &sh.abort_flag)) {
                         alive = false;
                         break;
                     }
                     ptx::tc_fence_after();
                     const uint32_t slot = ring + s * FT_SLOT;
-                    for (int c = 0; c * 128 < rows; ++c)
-                        ptx::umma_bf16(tmem_base + (uint32_t)((r / 128 + c) * FT_N), make_desc_k_sw32(slot + c * 4096),
+                    for (int c = 0; c < 2 * ch && (cg * ch * 2 + c) * 128 < P.d; ++c)
+                        ptx::umma_bf16(tmem_base + (uint32_t)((cg * ch * 2 + c) * FT_N), make_desc_k_sw32(slot + c * 4096),
                                        make_desc_k_sw32(hg_addr + j * (FT_N * 32)), idesc, (uint32_t)(j != 0));
                     ptx::umma_commit(ptx::smem_u32(&sh.empty[s]));
                     if (++s == FT_STAGES) {
@@ -292,76 +326,100 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                     }
                 }
             }
+            TRACE(8);
             if (alive) ptx::umma_commit(ptx::smem_u32(&sh.d2_full));
         }
     } else {
         // ------------------------------------------------------------ router, epilogues, final sum (12 warps)
         const int etid = (int)threadIdx.x - 64;
 #define FT_SYNC() asm volatile("bar.sync 1, %0;" ::"n"(FT_EPI) : "memory")
-        // ---- router: logits of every token.  A row of Wr (E floats) is covered by E/4 neighbouring threads with one
-        // 16-byte load each; a thread keeps its four experts' sums over every rpp-th row, for every token.
+        // ---- the tokens as the up-projection's N operand: per 64-wide block of d, 8 rows of 128 bytes in the 128-byte
+        // swizzle (16-byte piece c of row t sits at piece c ^ t); rows T.. are zero
+        for (int i = etid; i < nkb * 64; i += FT_EPI) {
+            const int kb = i >> 6, t = (i >> 3) & 7, c = i & 7;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (t < T) v = __ldg(reinterpret_cast<const uint4*>(P.x + (size_t)t * P.d + kb * 64) + c);
+            *reinterpret_cast<uint4*>(xs + kb * FT_XBLOCK + t * 128 + ((c ^ t) << 4)) = v;
+        }
+        // ---- router, step 1: the reduction over d of every token is cut into KS slices, one CTA per (token, slice).
+        // A row of Wr (E floats) is covered by E/4 neighbouring threads with one 16-byte load each; a thread keeps its
+        // four experts' sums over every rpp-th row of the slice; all its loads are in flight at once.
         {
+            int KS = 1;
+            while (KS < 16 && KS * 2 * T <= G) KS *= 2;
             const int quads = (E + 3) / 4, rpp = FT_EPI / quads;
-            const int qd = etid % quads, r0 = etid / quads;
-            float4 acc[kFusedMaxT];
+            if ((int)blockIdx.x < T * KS) {
+                const int t = blockIdx.x / KS, sl = blockIdx.x % KS;
+                const int klen = (P.d + KS - 1) / KS, kbeg = sl * klen, kend = min(P.d, kbeg + klen);
+                const __nv_bfloat16* __restrict__ xr = P.x + (size_t)t * P.d;
+                const int qd = etid % quads, r0 = etid / quads;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (r0 < rpp) {
+                    if ((E & 3) == 0) {
+                        for (int kb = kbeg + r0; kb < kend; kb += FT_ROUTER_BATCH * rpp) {
+                            float4 w[FT_ROUTER_BATCH];
+                            float xs[FT_ROUTER_BATCH];
 #pragma unroll
-            for (int t = 0; t < kFusedMaxT; ++t) acc[t] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (r0 < rpp) {
-                if ((E & 3) == 0) {
-                    for (int kb = r0; kb < P.d; kb += FT_ROUTER_BATCH * rpp) {
-                        float4 w[FT_ROUTER_BATCH];
+                            for (int j = 0; j < FT_ROUTER_BATCH; ++j) {
+                                const int k = kb + j * rpp;
+                                const bool ok = k < kend;
+                                w[j] = ok ? __ldg(reinterpret_cast<const float4*>(P.Wr + (size_t)k * E) + qd)
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+                                xs[j] = ok ? __bfloat162float(xr[k]) : 0.f;
+                            }
 #pragma unroll
-                        for (int j = 0; j < FT_ROUTER_BATCH; ++j) {
-                            const int k = kb + j * rpp;
-                            w[j] = k < P.d ? __ldg(reinterpret_cast<const float4*>(P.Wr + (size_t)k * E) + qd)
-                                           : make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-#pragma unroll
-                        for (int j = 0; j < FT_ROUTER_BATCH; ++j) {
-                            const int k = kb + j * rpp;
-#pragma unroll
-                            for (int t = 0; t < kFusedMaxT; ++t) {
-                                if (t < T && k < P.d) {
-                                    const float xv = __bfloat162float(P.x[(size_t)t * P.d + k]);
-                                    acc[t].x = fmaf(xv, w[j].x, acc[t].x);
-                                    acc[t].y = fmaf(xv, w[j].y, acc[t].y);
-                                    acc[t].z = fmaf(xv, w[j].z, acc[t].z);
-                                    acc[t].w = fmaf(xv, w[j].w, acc[t].w);
-                                }
+                            for (int j = 0; j < FT_ROUTER_BATCH; ++j) {
+                                acc.x = fmaf(xs[j], w[j].x, acc.x);
+                                acc.y = fmaf(xs[j], w[j].y, acc.y);
+                                acc.z = fmaf(xs[j], w[j].z, acc.z);
+                                acc.w = fmaf(xs[j], w[j].w, acc.w);
                             }
                         }
-                    }
-                } else {
-                    const int e0 = qd * 4;
-                    for (int k = r0; k < P.d; k += rpp) {
-                        const float* w = P.Wr + (size_t)k * E + e0;
-                        const float w0 = __ldg(w), w1 = e0 + 1 < E ? __ldg(w + 1) : 0.f, w2 = e0 + 2 < E ? __ldg(w + 2) : 0.f,
-                                    w3 = e0 + 3 < E ? __ldg(w + 3) : 0.f;
-#pragma unroll
-                        for (int t = 0; t < kFusedMaxT; ++t) {
-                            if (t < T) {
-                                const float xv = __bfloat162float(P.x[(size_t)t * P.d + k]);
-                                acc[t].x = fmaf(xv, w0, acc[t].x);
-                                acc[t].y = fmaf(xv, w1, acc[t].y);
-                                acc[t].z = fmaf(xv, w2, acc[t].z);
-                                acc[t].w = fmaf(xv, w3, acc[t].w);
-                            }
+                    } else {
+                        const int e0 = qd * 4;
+                        for (int k = kbeg + r0; k < kend; k += rpp) {
+                            const float xv = __bfloat162float(xr[k]);
+                            const float* w = P.Wr + (size_t)k * E + e0;
+                            acc.x = fmaf(xv, __ldg(w), acc.x);
+                            if (e0 + 1 < E) acc.y = fmaf(xv, __ldg(w + 1), acc.y);
+                            if (e0 + 2 < E) acc.z = fmaf(xv, __ldg(w + 2), acc.z);
+                            if (e0 + 3 < E) acc.w = fmaf(xv, __ldg(w + 3), acc.w);
                         }
                     }
                 }
+                // the threads' sums meet in shared memory (the ring is idle until the partition is known); the slice's
+                // sum per expert goes to global memory, where every CTA will read it (the partial-output buffer is free
+                // until the very end)
+                reinterpret_cast<float4*>(smem)[etid] = acc;
+                FT_SYNC();
+                if (etid < E) {
+                    const float* sf = reinterpret_cast<const float*>(smem);
+                    float v = 0.f;
+                    for (int r = 0; r < rpp; ++r) v += sf[(r * quads + (etid >> 2)) * 4 + (etid & 3)];
+                    P.partial[((size_t)t * KS + sl) * kMaxExperts + etid] = v;
+                }
             }
-            // the threads' sums meet in shared memory (the ring is idle until the partition is known) and are added
-            // per (token, expert) in a fixed order
-            float4* scratch = reinterpret_cast<float4*>(smem);
-#pragma unroll
-            for (int t = 0; t < kFusedMaxT; ++t)
-                if (t < T) scratch[t * FT_EPI + etid] = acc[t];
+            if (etid == 0) TRACE(1);
             FT_SYNC();
-            const float* sf = reinterpret_cast<const float*>(smem);
+            if (etid == 0) {
+                grid_arrive(P.sync, 1);
+                if (!grid_wait(P.sync, 1, G, &sh.abort_flag)) sh.abort_flag = 1;
+                TRACE(13);
+            }
+            FT_SYNC();
+            // ---- router, step 2, in EVERY CTA: the slices' sums of every token are fetched in one go into shared memory
+            // and added per (token, expert) in ascending slice order: the same arithmetic everywhere, hence the same
+            // scores, selection and partition -- nothing more to agree on
+            float* stage = reinterpret_cast<float*>(smem);
+            for (int i = etid; i < T * KS * E; i += FT_EPI) {
+                const int e = i % E, ts = i / E;
+                stage[ts * kMaxExperts + e] = __ldcg(P.partial + (size_t)ts * kMaxExperts + e);
+            }
+            FT_SYNC();
             for (int item = etid; item < T * E; item += FT_EPI) {
                 const int t = item / E, e = item % E;
                 float v = P.br ? P.br[e] : 0.f;
-                for (int r = 0; r < rpp; ++r) v += sf[((size_t)t * FT_EPI + r * quads + (e >> 2)) * 4 + (e & 3)];
+                for (int sl = 0; sl < KS; ++sl) v += stage[(t * KS + sl) * kMaxExperts + e];
                 sh.score_s[t][e] = v;
             }
             FT_SYNC();
@@ -397,8 +455,21 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                 const long long U = (long long)n * upe;
                 sh.u0 = (int)(U * blockIdx.x / G);
                 sh.u1 = (int)(U * (blockIdx.x + 1) / G);
+                int nt = 0;
+                for (int u = sh.u0; u < sh.u1 && nt < FT_MAXTILES;) {
+                    const int iu = u % upe, len = min(8, min(sh.u1 - u, upe - iu));
+                    sh.tile_e[nt] = sh.active[u / upe];
+                    sh.tile_iu0[nt] = iu;
+                    sh.tile_len[nt] = len;
+                    sh.tile_ul0[nt] = u - sh.u0;
+                    ++nt;
+                    u += len;
+                }
+                sh.ntiles = nt;
+                sh.nchain = max(1, min(min(4, nkb), FT_TMEM_COLS / FT_N / max(nt, 1)));
                 __threadfence_block();
                 sh.geo_ready = 1;
+                TRACE(2);
             }
             if (P.counts_out && blockIdx.x == 0 && etid < E) {
                 int n = 0;
@@ -407,7 +478,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             }
             FT_SYNC();
         }
-        const int u0 = sh.u0, u1 = sh.u1, nu = u1 - u0;
+        const int nu = sh.u1 - sh.u0;
         const int q = warp & 3, grp = (warp - 2) >> 2;       // TMEM lanes 32 q ..; three warps share a quarter
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         float* mine = P.partial + (size_t)blockIdx.x * T * P.d;
@@ -418,19 +489,27 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             if (!dead && !ptx::mbar_wait(ptx::smem_u32(&sh.d1_full), 0u, &sh.abort_flag)) dead = true;
             dead = __any_sync(0xffffffffu, dead);
             ptx::tc_fence_after();
-            for (int m = grp; !dead && m * 8 < nu; m += 3) {
-                uint32_t r[16];
-                ptx::tmem_ld16(tmem_base + (uint32_t)(m * FT_N) + lane_base, r);
-                ptx::tmem_ld_wait();
-                const int hr = q * 32 + lane, ul = m * 8 + hr / FT_UNIT, kk = hr % FT_UNIT;
-                if (ul < nu) {
-                    const int e = sh.active[(u0 + ul) / upe];
+            if (etid == 0) TRACE(6);
+            for (int ti = grp; !dead && ti < sh.ntiles; ti += 3) {
+                float r[16];
+#pragma unroll
+                for (int t = 0; t < 16; ++t) r[t] = 0.f;
+                for (int c = 0; c < sh.nchain; ++c) {
+                    uint32_t rc[16];
+                    ptx::tmem_ld16(tmem_base + (uint32_t)((ti * sh.nchain + c) * FT_N) + lane_base, rc);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) r[t] += __uint_as_float(rc[t]);
+                }
+                const int hr = q * 32 + lane, kk = hr % FT_UNIT;
+                if (hr < sh.tile_len[ti] * FT_UNIT) {
+                    const int ul = sh.tile_ul0[ti] + hr / FT_UNIT, e = sh.tile_e[ti];
                     uint8_t* dst = hg + ul * (FT_N * 32) + (kk & 7) * 2;
 #pragma unroll
                     for (int t = 0; t < FT_N; ++t) {
                         float v = 0.f;
                         if (t < kFusedMaxT && t < T && ((sh.mask_s[t] >> e) & 1ull))
-                            v = sh.score_s[t][e] * gelu_erf(__uint_as_float(r[t]));
+                            v = sh.score_s[t][e] * gelu_erf(r[t]);
                         *reinterpret_cast<__nv_bfloat16*>(dst + t * 32 + (((kk >> 3) ^ ((t >> 2) & 1)) << 4)) = __float2bfloat16_rn(v);
                     }
                 }
@@ -438,11 +517,15 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             ptx::tc_fence_before();
             ptx::fence_proxy_async();           // the tensor core reads what these threads wrote
             FT_SYNC();
-            if (etid == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.hg_ready));
+            if (etid == 0) {
+                ptx::mbar_arrive(ptx::smem_u32(&sh.hg_ready));
+                TRACE(7);
+            }
             // ---- this CTA's partial output: D2 -> global memory
             if (!dead && !ptx::mbar_wait(ptx::smem_u32(&sh.d2_full), 0u, &sh.abort_flag)) dead = true;
             dead = __any_sync(0xffffffffu, dead);
             ptx::tc_fence_after();
+            if (etid == 0) TRACE(9);
             for (int c = grp; !dead && c * 128 < P.d; c += 3) {
                 uint32_t r[16];
                 ptx::tmem_ld16(tmem_base + (uint32_t)(c * FT_N) + lane_base, r);
@@ -461,8 +544,10 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         // ---- grid barrier, then out[t,c] = the CTAs' partial outputs added in ascending CTA order
         FT_SYNC();
         if (etid == 0) {
+            TRACE(10);
             grid_arrive(P.sync, 0);
             if (!grid_wait(P.sync, 0, G, &sh.abort_flag)) sh.abort_flag = 1;
+            TRACE(11);
         }
         FT_SYNC();
         if (!sh.abort_flag) {
@@ -512,6 +597,12 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, FT_TMEM_COLS);
     }
+#ifdef DSMOE_TRACE
+    if (threadIdx.x == 0 && blockIdx.x < 192) {
+        TRACE(12);
+        for (int i = 0; i < 32; ++i) g_trace_fused[blockIdx.x][i] = sh.trace[i];
+    }
+#endif
     if (threadIdx.x == 0 && sh.abort_flag) {
         atomicExch(P.sync + 4, 1);
         if (P.dev_status) *P.dev_status = DSMOE_ERR_TIMEOUT;
@@ -520,11 +611,17 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 
 }  // namespace
 
+#ifdef DSMOE_TRACE
+extern "C" __attribute__((visibility("default"))) int dsmoe_trace_read_fused(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_trace_fused, sizeof(unsigned long long) * 192 * 32);
+}
+#endif
+
 bool fused_decode_supported(const dsmoe_layer_desc& p) {
     const int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
     if (!umma_supported(p) || p.T < 1 || p.T > kFusedMaxT || p.T > G) return false;
     if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK) return false;            // its K needs a pass over the batch first
-    if (p.d > 4096) return false;                                       // d / 128 accumulators of 16 columns in TMEM
+    if (p.d > 4096 || p.d % 256) return false;       // d / 128 accumulators of 16 columns in TMEM; W2 copied in chunks of 256 columns
     return ((long long)p.E * (p.H / FT_UNIT) + G - 1) / G <= kFusedMaxUnits;
 }
 
@@ -535,18 +632,16 @@ dsmoe_status launch_layer_fused_decode(const dsmoe_layer_desc& p, const void* x,
     DeviceState* st = nullptr;
     DSMOE_TRY(device_state(&st));
     if (!st->attr_fused) {
-        DSMOE_CUDA_TRY(cudaFuncSetAttribute(fused_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FT_SMEM_BYTES));
+        DSMOE_CUDA_TRY(cudaFuncSetAttribute(fused_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ft_smem_bytes(4096)));
         st->attr_fused = true;
     }
     const __nv_bfloat16* w1t = static_cast<const __nv_bfloat16*>(packed);
     const __nv_bfloat16* w2t = w1t + (size_t)p.E * p.H * p.d;
     const int G = sm_count() < kSmallMaxCtas ? sm_count() : kSmallMaxCtas;
-    const CUtensorMap* mX;
-    const BMaps16* mW1;
-    const BMapsK16* mW2;
-    DSMOE_TRY(cached_map_2d(&mX, x, p.T, p.d, FT_N));          // rows beyond T read as zeros
-    DSMOE_TRY(cached_bmaps16(&mW1, w1t, p.E, p.H, p.d));
-    DSMOE_TRY(cached_bmaps_k16(&mW2, w2t, p.E, p.d, p.H));
+    const BMapsUp* mW1;
+    const BMapsDown* mW2;
+    DSMOE_TRY(cached_bmaps_up(&mW1, w1t, p.E, p.H, p.d));
+    DSMOE_TRY(cached_bmaps_down(&mW2, w2t, p.E, p.d, p.H));
     FusedParams P;
     P.T = p.T; P.d = p.d; P.H = p.H; P.E = p.E;
     P.x = static_cast<const __nv_bfloat16*>(x);
@@ -563,11 +658,11 @@ dsmoe_status launch_layer_fused_decode(const dsmoe_layer_desc& p, const void* x,
     P.sync = reinterpret_cast<int*>(ws + L.sync);
     P.dev_status = dev_status;
     DSMOE_CUDA_TRY(cudaMemsetAsync(P.sync, 0, 32, s));
-    void* args[] = {const_cast<CUtensorMap*>(mX), const_cast<BMaps16*>(mW1), const_cast<BMapsK16*>(mW2), &P};
+    void* args[] = {const_cast<BMapsUp*>(mW1), const_cast<BMapsDown*>(mW2), &P};
     int timed = -1;
     DSMOE_TRY(timing_begin(s, &timed));
     DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(fused_decode_kernel), dim3(G), dim3(FT_THREADS),
-                                               args, FT_SMEM_BYTES, s));
+                                               args, ft_smem_bytes(p.d), s));
     DSMOE_TRY(timing_end(s, timed));
     return DSMOE_OK;
 }
