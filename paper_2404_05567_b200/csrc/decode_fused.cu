@@ -68,7 +68,8 @@ struct FusedParams {
     float* partial;          // [grid][T][d]
     void* out;
     int out_f32;
-    int* sync;               // 8 ints, zero at launch: grid-barrier counter [0] and an abort flag [4]
+    int* sync;               // 8 ints, zero at launch: grid-barrier counters [0], [1] and an abort flag [4]
+    int simt_up;             // up-projection on the CUDA cores (T <= 4) instead of the tensor cores
     int32_t* dev_status;
 };
 
@@ -271,7 +272,7 @@ fused_decode_kernel(const __grid_constant__ BMapsUp tmW1, const __grid_constant_
             // `nchain` accumulators (64-wide block kb goes to accumulator kb % nchain, at TMEM columns
             // 16 (tile nchain + kb % nchain) ..), which the epilogue adds up.
             const int nchain = sh.nchain;
-            for (int ti = 0; alive && ti < sh.ntiles; ++ti) {
+            for (int ti = 0; alive && !P.simt_up && ti < sh.ntiles; ++ti) {
                 const int len = sh.tile_len[ti], kbp = tmW1.kbp[len - 1];
                 for (int g = 0; g * kbp < nkb; ++g) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&sh.full[s]), ph, &sh.abort_flag)) {
@@ -299,9 +300,19 @@ fused_decode_kernel(const __grid_constant__ BMapsUp tmW1, const __grid_constant_
                     }
                 }
             }
+            if (P.simt_up) {
+                // the CUDA cores took the up-projection's copies off the ring: the down-projection's follow them
+                int n_up = 0;
+                for (int ti = 0; ti < sh.ntiles; ++ti) {
+                    const int kbp = tmW1.kbp[sh.tile_len[ti] - 1];
+                    n_up += (nkb + kbp - 1) / kbp;
+                }
+                s = n_up % FT_STAGES;
+                ph = (uint32_t)(n_up / FT_STAGES) & 1u;
+            }
             TRACE(5);
             if (alive) {
-                ptx::umma_commit(ptx::smem_u32(&sh.d1_full));
+                if (!P.simt_up) ptx::umma_commit(ptx::smem_u32(&sh.d1_full));
                 // the gated activations in shared memory (and D1 read out of TMEM: D2 takes its place)
                 if (!ptx::mbar_wait(ptx::smem_u32(&sh.hg_ready), 0u, &sh.abort_flag)) alive = false;
                 ptx::tc_fence_after();
@@ -333,13 +344,29 @@ fused_decode_kernel(const __grid_constant__ BMapsUp tmW1, const __grid_constant_
         // ------------------------------------------------------------ router, epilogues, final sum (12 warps)
         const int etid = (int)threadIdx.x - 64;
 #define FT_SYNC() asm volatile("bar.sync 1, %0;" ::"n"(FT_EPI) : "memory")
-        // ---- the tokens as the up-projection's N operand: per 64-wide block of d, 8 rows of 128 bytes in the 128-byte
-        // swizzle (16-byte piece c of row t sits at piece c ^ t); rows T.. are zero
-        for (int i = etid; i < nkb * 64; i += FT_EPI) {
-            const int kb = i >> 6, t = (i >> 3) & 7, c = i & 7;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (t < T) v = __ldg(reinterpret_cast<const uint4*>(P.x + (size_t)t * P.d + kb * 64) + c);
-            *reinterpret_cast<uint4*>(xs + kb * FT_XBLOCK + t * 128 + ((c ^ t) << 4)) = v;
+        // ---- the tokens in shared memory.  For the tensor cores: the up-projection's N operand, per 64-wide block of d
+        // 8 rows of 128 bytes in the 128-byte swizzle (16-byte piece c of row t sits at piece c ^ t), rows T.. zero.
+        // For the CUDA cores (simt_up): fp32, per (block, token) the low halves of the eight 8-element pieces (16 bytes
+        // each, 128 bytes in all), then the high halves, so that 8 lanes read them without bank conflicts.
+        if (P.simt_up) {
+            for (int i = etid; i < nkb * T * 8; i += FT_EPI) {
+                const int c = i & 7, kt = i >> 3, kb = kt / T, t = kt % T;
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(P.x + (size_t)t * P.d + kb * 64) + c);
+                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+                const float2 a = __bfloat1622float2(h2[0]), b = __bfloat1622float2(h2[1]), cc = __bfloat1622float2(h2[2]),
+                             dd = __bfloat1622float2(h2[3]);
+                float4* dst = reinterpret_cast<float4*>(xs + (size_t)kt * 256 + c * 16);
+                dst[0] = make_float4(a.x, a.y, b.x, b.y);
+                dst[8] = make_float4(cc.x, cc.y, dd.x, dd.y);
+            }
+            for (int i = etid; i < FT_HG_BYTES / 16; i += FT_EPI) reinterpret_cast<uint4*>(hg)[i] = make_uint4(0u, 0u, 0u, 0u);
+        } else {
+            for (int i = etid; i < nkb * 64; i += FT_EPI) {
+                const int kb = i >> 6, t = (i >> 3) & 7, c = i & 7;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (t < T) v = __ldg(reinterpret_cast<const uint4*>(P.x + (size_t)t * P.d + kb * 64) + c);
+                *reinterpret_cast<uint4*>(xs + kb * FT_XBLOCK + t * 128 + ((c ^ t) << 4)) = v;
+            }
         }
         // ---- router, step 1: the reduction over d of every token is cut into KS slices, one CTA per (token, slice).
         // A row of Wr (E floats) is covered by E/4 neighbouring threads with one 16-byte load each; a thread keeps its
@@ -486,6 +513,91 @@ fused_decode_kernel(const __grid_constant__ BMapsUp tmW1, const __grid_constant_
         if (nu > 0) {
             // ---- GeLU and gate: D1 -> shared memory, as the down-projection's token operand (16 rows of 32 bytes per
             // unit, the 32-byte swizzle written by hand)
+            if (P.simt_up) {
+                // Few tokens: the MMA would read 128 rows of weights per instruction at its fixed pace whatever the
+                // number of tokens (about 128 cycles for 4 KB, less for a narrower tile), which is slower than the
+                // memory delivers them.  The CUDA cores keep up: a row of 64 weights is read by 8 lanes (16 bytes
+                // each), a warp takes 4 rows at a time, every lane keeps fp32 sums for its rows and every token.
+                const int w = warp - 2, g = lane >> 3, c = lane & 7;
+                int sl = 0;
+                uint32_t sph = 0;
+                for (int ti = 0; ti < sh.ntiles; ++ti) {
+                    const int len = sh.tile_len[ti], rows = len * FT_UNIT, kbp = tmW1.kbp[len - 1];
+                    float acc[3][4];
+#pragma unroll
+                    for (int i = 0; i < 3; ++i)
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) acc[i][t] = 0.f;
+                    for (int g0 = 0; g0 * kbp < nkb; ++g0) {
+                        if (!dead && !ptx::mbar_wait(ptx::smem_u32(&sh.full[sl]), sph, &sh.abort_flag)) dead = true;
+                        const uint8_t* slot = smem + sl * FT_SLOT;
+                        for (int kbi = 0; !dead && kbi < kbp && g0 * kbp + kbi < nkb; ++kbi) {
+                            const int kb = g0 * kbp + kbi;
+                            float4 xlo[4], xhi[4];
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) {
+                                if (t < T) {
+                                    const float4* xp = reinterpret_cast<const float4*>(xs + (size_t)(kb * T + t) * 256 + c * 16);
+                                    xlo[t] = xp[0];
+                                    xhi[t] = xp[8];
+                                }
+                            }
+#pragma unroll
+                            for (int i = 0; i < 3; ++i) {
+                                const int r = 4 * (w + 12 * i) + g;
+                                if (r < rows) {
+                                    const uint4 wv = *reinterpret_cast<const uint4*>(slot + (size_t)kbi * rows * 128 + r * 128 +
+                                                                                     ((c ^ (r & 7)) << 4));
+                                    const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&wv);
+                                    const float2 w0 = __bfloat1622float2(h2[0]), w1 = __bfloat1622float2(h2[1]),
+                                                 w2 = __bfloat1622float2(h2[2]), w3 = __bfloat1622float2(h2[3]);
+#pragma unroll
+                                    for (int t = 0; t < 4; ++t) {
+                                        if (t < T) {
+                                            float a = acc[i][t];
+                                            a = fmaf(w0.x, xlo[t].x, a);
+                                            a = fmaf(w0.y, xlo[t].y, a);
+                                            a = fmaf(w1.x, xlo[t].z, a);
+                                            a = fmaf(w1.y, xlo[t].w, a);
+                                            a = fmaf(w2.x, xhi[t].x, a);
+                                            a = fmaf(w2.y, xhi[t].y, a);
+                                            a = fmaf(w3.x, xhi[t].z, a);
+                                            a = fmaf(w3.y, xhi[t].w, a);
+                                            acc[i][t] = a;
+                                        }
+                                    }
+                                }
+                            }
+                        }
+                        FT_SYNC();                                   // every warp is done with the slot
+                        if (etid == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.empty[sl]));
+                        if (++sl == FT_STAGES) {
+                            sl = 0;
+                            sph ^= 1u;
+                        }
+                    }
+                    // the 8 lanes of a row add their sums; lane c = t writes token t's gated activation
+                    const int e = sh.tile_e[ti];
+#pragma unroll
+                    for (int i = 0; i < 3; ++i) {
+                        const int r = 4 * (w + 12 * i) + g;
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            float v = acc[i][t];
+                            v += __shfl_xor_sync(0xffffffffu, v, 1);
+                            v += __shfl_xor_sync(0xffffffffu, v, 2);
+                            v += __shfl_xor_sync(0xffffffffu, v, 4);
+                            if (c == t && t < T && r < rows) {
+                                const int ul = sh.tile_ul0[ti] + r / FT_UNIT, kk = r % FT_UNIT;
+                                const float gate = ((sh.mask_s[t] >> e) & 1ull) ? sh.score_s[t][e] : 0.f;
+                                *reinterpret_cast<__nv_bfloat16*>(hg + ul * (FT_N * 32) + t * 32 + ((kk >> 3) << 4) + (kk & 7) * 2) =
+                                    __float2bfloat16_rn(gate * gelu_erf(v));          // rows 0..3: the swizzle leaves them in place
+                            }
+                        }
+                    }
+                }
+                if (etid == 0) TRACE(6);
+            } else {
             if (!dead && !ptx::mbar_wait(ptx::smem_u32(&sh.d1_full), 0u, &sh.abort_flag)) dead = true;
             dead = __any_sync(0xffffffffu, dead);
             ptx::tc_fence_after();
@@ -513,6 +625,7 @@ fused_decode_kernel(const __grid_constant__ BMapsUp tmW1, const __grid_constant_
                         *reinterpret_cast<__nv_bfloat16*>(dst + t * 32 + (((kk >> 3) ^ ((t >> 2) & 1)) << 4)) = __float2bfloat16_rn(v);
                     }
                 }
+            }
             }
             ptx::tc_fence_before();
             ptx::fence_proxy_async();           // the tensor core reads what these threads wrote
@@ -657,6 +770,10 @@ dsmoe_status launch_layer_fused_decode(const dsmoe_layer_desc& p, const void* x,
     P.out_f32 = p.out_fp32 ? 1 : 0;
     P.sync = reinterpret_cast<int*>(ws + L.sync);
     P.dev_status = dev_status;
+#ifndef DSMOE_FUSED_SIMT_MAX_T
+#define DSMOE_FUSED_SIMT_MAX_T 4
+#endif
+    P.simt_up = p.T <= (DSMOE_FUSED_SIMT_MAX_T < 4 ? DSMOE_FUSED_SIMT_MAX_T : 4) ? 1 : 0;
     DSMOE_CUDA_TRY(cudaMemsetAsync(P.sync, 0, 32, s));
     void* args[] = {const_cast<BMapsUp*>(mW1), const_cast<BMapsDown*>(mW2), &P};
     int timed = -1;
