@@ -45,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     sources = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     headers = sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + [os.path.join(ROOT, "include", "dsmoe.h")]
     extra = ["-Xptxas", "-v"] if verbose else []
-    extra += os.environ.get("DSMOE_NVCC_EXTRA", "").split()      # e.g. -DDSMOE_FUSED_DECODE_MAX_T=8 for a tuning build
+    extra += os.environ.get("DSMOE_NVCC_EXTRA", "").split()      # e.g. -DDSMOE_SMALL_INFLIGHT=196608 for a tuning build
     jobs = []
     objs = []
     for src in sources:

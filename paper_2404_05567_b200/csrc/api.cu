@@ -67,10 +67,7 @@ WsLayout ws_layout(const dsmoe_layer_desc& p) {
     // expert outputs [Amax,d] in fp32 (separate aggregation)
     L.acc = take(!umma_supported(p) ? 0 : fuses_combine(p) ? T * p.d * 4 : amax * p.d * 4);
     // fp32 partial sums of the small-T path: (CTA, 2 column ranges, T, 256)
-    // ... or of the few-token kernel: (CTA, T, d)
-    size_t part = umma_supported(p) && p.T <= kSmallMaxT ? (size_t)kSmallMaxCtas * 2 * T * 256 * 4 : 0;
-    if (umma_supported(p) && p.T <= kFusedMaxT && (size_t)kSmallMaxCtas * T * p.d * 4 > part) part = (size_t)kSmallMaxCtas * T * p.d * 4;
-    L.partial = take(part);
+    L.partial = take(umma_supported(p) && p.T <= kSmallMaxT ? (size_t)kSmallMaxCtas * 2 * T * 256 * 4 : 0);
     L.router = take(router_umma_supported(p) ? router_umma_scratch(p) : 0);   // tensor-core router: split Wr, partial logits
     // dense backward: the experts' hidden activations go to `h` ([T,E*H]); per-column-tile partial dot products here
     L.bwd = take(umma_supported(p) ? T * E * ceil_div(p.H, 256) * 4 : 0);
@@ -244,11 +241,6 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     float* row_gate = reinterpret_cast<float*>(ws + L.row_gate);
     int32_t* token_rows = reinterpret_cast<int32_t*>(ws + L.token_rows);
 
-#ifndef DSMOE_FUSED_DECODE_MAX_T
-#define DSMOE_FUSED_DECODE_MAX_T 7
-#endif
-    if (fast && p.T <= DSMOE_FUSED_DECODE_MAX_T && fused_decode_supported(p))
-        return launch_layer_fused_decode(p, x, Wr, br, packed, scores, mask, k_t, counts_out, out, ws, L, dev_status, s);
     if (fast && small_supported(p))
         return launch_layer_small(p, x, Wr, br, packed, scores, mask, k_t, counts_out, out, ws, L, dev_status, s);
 

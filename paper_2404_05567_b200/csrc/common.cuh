@@ -15,8 +15,6 @@ constexpr int kMaxExperts = 64;
 constexpr int kChunk = 32;   // tokens per ballot chunk in the grouping kernels
 constexpr int kSmallMaxT = 128;      // the small-T (decode) path keeps all tokens in one 128-row MMA tile
 constexpr int kSmallMaxCtas = 192;   // upper bound on that path's grid (sizes its partial-sum buffer)
-constexpr int kFusedMaxT = 8;        // the few-token kernel (decode_fused.cu): tokens it takes ...
-constexpr int kFusedMaxUnits = 32;   // ... and 16-wide hidden units one CTA may own
 
 #define DSMOE_CUDA_TRY(expr)                                  \
     do {                                                      \
@@ -63,7 +61,7 @@ WsLayout ws_layout(const dsmoe_layer_desc& p);
 constexpr int kMaxDeviceSlots = 64;
 struct DeviceState {
     int sm_count = 0;
-    bool attr_gemm = false, attr_small = false, attr_fused = false, attr_router_f32 = false, attr_router_bf16 = false;
+    bool attr_gemm = false, attr_small = false, attr_router_f32 = false, attr_router_bf16 = false;
 };
 dsmoe_status device_state(DeviceState** out, int* device = nullptr);   // of the current device
 
@@ -143,14 +141,6 @@ dsmoe_status launch_layer_small(const dsmoe_layer_desc& p, const void* x, const 
 dsmoe_status launch_layer_umma(const dsmoe_layer_desc& p, const void* x, const void* packed, const float* scores,
                                const uint64_t* mask, const int32_t* k_t, int32_t* counts_out, void* out, char* ws,
                                const WsLayout& L, int32_t* dev_status, cudaStream_t s, bool* done);
-
-// ---- decode_fused.cu : whole layer for up to kFusedMaxT tokens, one cooperative launch, no hand-over between CTAs
-// from the up- to the down-projection
-bool fused_decode_supported(const dsmoe_layer_desc& p);
-dsmoe_status launch_layer_fused_decode(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
-                                       const void* packed, float* scores, uint64_t* mask, int32_t* k_t,
-                                       int32_t* counts_out, void* out, char* ws, const WsLayout& L, int32_t* dev_status,
-                                       cudaStream_t s);
 
 // ---- training.cu / mlp_umma.cu : the training side (Eq. 2-6)
 size_t mi_scratch_bytes();

@@ -156,61 +156,6 @@ dsmoe_status cached_bmaps16(const BMaps16** out, const void* ptr, uint64_t E, ui
 }
 
 
-static dsmoe_status encode(CUtensorMap* m, int rank, const void* ptr, const cuuint64_t* dims, const cuuint64_t* strides,
-                           const cuuint32_t* box, CUtensorMapSwizzle swz) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return DSMOE_ERR_CUDA;
-    const cuuint32_t es[5] = {1, 1, 1, 1, 1};
-    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), dims, strides, box, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? DSMOE_OK : DSMOE_ERR_CUDA;
-}
-
-static MapCache<BMapsUp, 64> g_bmaps_up;
-static MapCache<BMapsDown, 64> g_bmaps_down;
-
-dsmoe_status cached_bmaps_up(const BMapsUp** out, const void* ptr, uint64_t E, uint64_t n, uint64_t kk) {
-    const MapKey k{ptr, E, n, kk, 4};
-    BMapsUp* m = g_bmaps_up.find(k);
-    if (!m) {
-        BMapsUp tmp;
-        const uint64_t nkb = kk / kTileK;
-        for (int len = 1; len <= 8; ++len) {
-            uint32_t kbp = 1;
-            while (kbp * 2 * len * 16 * 128 <= 32768 && kbp * 2 <= nkb) kbp *= 2;
-            const cuuint64_t dims[4] = {kTileK, n, nkb, E};
-            const cuuint64_t strides[3] = {kTileK * 2, n * kTileK * 2, n * kk * 2};
-            const cuuint32_t box[4] = {kTileK, (cuuint32_t)(16 * len), kbp, 1};
-            DSMOE_TRY(encode(&tmp.m[len - 1], 4, ptr, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B));
-            tmp.kbp[len - 1] = (int)kbp;
-        }
-        m = g_bmaps_up.slot(k);
-        *m = tmp;
-    }
-    *out = m;
-    return DSMOE_OK;
-}
-
-// n (output columns) must be a multiple of 256
-dsmoe_status cached_bmaps_down(const BMapsDown** out, const void* ptr, uint64_t E, uint64_t n, uint64_t kk) {
-    const MapKey k{ptr, E, n, kk, 5};
-    BMapsDown* m = g_bmaps_down.find(k);
-    if (!m) {
-        BMapsDown tmp;
-        const uint64_t nch = n / 256;
-        tmp.ch = (int)(nch < 4 ? nch : 4);
-        const cuuint64_t dims[5] = {kTileK, 256, nch, kk / kTileK, E};
-        const cuuint64_t strides[4] = {kTileK * 2, 256 * kTileK * 2, n * kTileK * 2, n * kk * 2};
-        const cuuint32_t box[5] = {16, 256, (cuuint32_t)tmp.ch, 1, 1};
-        DSMOE_TRY(encode(&tmp.m, 5, ptr, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_32B));
-        m = g_bmaps_down.slot(k);
-        *m = tmp;
-    }
-    *out = m;
-    return DSMOE_OK;
-}
-
 // Optional per-launch timing of the tensor-core kernels (a measurement aid for benchmarks): a ring of CUDA event
 // pairs; every timed launch takes the next pair until the ring is full.  The events sit on the caller's stream, so a
 // benchmark can leave them inside its un-synchronised step loop and read all durations afterwards.

@@ -24,21 +24,6 @@ struct BMaps16 {
 };
 
 
-// The few-token kernel's views of the packed weights.  The copy engine handles only a few copies per SM at a time
-// whatever their size (measured: about 4.5 copies per microsecond and SM from HBM), so a narrow tile must not cost
-// one copy per 64-wide reduction block: its copies span several blocks.
-//   up    W1 as [E][d/64][H][64]: one copy = `kbp[len-1]` reduction blocks of a run of `len` 16-row units (<= 32 KB)
-//   down  W2 as [E][H/64][d/256][256][64] in slices of 16 reduction elements (32-byte rows, 32-byte swizzle): one
-//         copy = `ch` chunks of 256 output columns of one 16-wide hidden unit (<= 32 KB)
-struct BMapsUp {
-    CUtensorMap m[8];
-    int kbp[8];
-};
-struct BMapsDown {
-    CUtensorMap m;
-    int ch;
-};
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -51,8 +36,6 @@ dsmoe_status cached_map_2d(const CUtensorMap** out, const void* ptr, uint64_t ro
 // packed weights [E][k / 64][n][64]
 dsmoe_status cached_bmaps(const BMaps** out, const void* ptr, uint64_t E, uint64_t n, uint64_t k);
 dsmoe_status cached_bmaps16(const BMaps16** out, const void* ptr, uint64_t E, uint64_t n, uint64_t k);
-dsmoe_status cached_bmaps_up(const BMapsUp** out, const void* ptr, uint64_t E, uint64_t n, uint64_t k);
-dsmoe_status cached_bmaps_down(const BMapsDown** out, const void* ptr, uint64_t E, uint64_t n, uint64_t k);
 // weights in their natural layout [E][n][k], k contiguous
 dsmoe_status cached_bmaps_plain(const BMaps** out, const void* ptr, uint64_t E, uint64_t n, uint64_t k);
 

@@ -1,4 +1,4 @@
-"""Phase timeline of the two decode kernels (a developer's diagnostic).
+"""Phase timeline of the decode kernel (a developer's diagnostic).
 
     python -m paper_2404_05567_b200.trace [--T 1] [--d 2048] [--H 1024] [--E 32] [--eps 0.03] [--reps 20]
 
@@ -21,11 +21,6 @@ import torch
 from . import binding
 from .build import CSRC, NVCC_FLAGS, PKG, ROOT, _nvcc
 
-FUSED_NAMES = {0: "CTA starts", 1: "router: slice sums written", 13: "router: grid barrier passed", 2: "router: partition known", 3: "producer: first copy issued",
-               4: "MMA issuer: first tile in shared memory", 14: "producer: last up-projection copy issued",
-               5: "MMA issuer: up-projection issued", 6: "epilogue: up-projection complete", 7: "epilogue: gated activations in shared memory",
-               15: "producer: last copy issued", 8: "MMA issuer: down-projection issued", 9: "epilogue: down-projection complete",
-               10: "partial output written", 11: "grid barrier passed", 12: "CTA ends"}
 SMALL_NAMES = {0: "CTA starts", 12: "router: first loads", 13: "router: slice sums done", 1: "router: at grid barrier",
                14: "router: grid barrier passed", 2: "router: partition known", 4: "MMA issuer: first tile in shared memory",
                3: "producer: up-projection issued", 28: "epilogue: first accumulator complete", 7: "epilogue: hg written, at grid barrier",
@@ -54,17 +49,19 @@ def main():
     ap.add_argument("--H", type=int, default=1024)
     ap.add_argument("--E", type=int, default=32)
     ap.add_argument("--eps", type=float, default=0.03)
+    ap.add_argument("--topk", type=int, default=0, help="select exactly this many experts per token instead of the threshold")
     ap.add_argument("--reps", type=int, default=20)
     a = ap.parse_args()
     binding.LIB_PATH = build_trace_lib()
     binding._lib = None
     dm = binding
     torch.manual_seed(0)
-    desc = dm.make_desc(a.T, a.d, a.H, a.E, dm.BF16, dm.SELECT_THRESHOLD, eps=a.eps)
+    desc = (dm.make_desc(a.T, a.d, a.H, a.E, dm.BF16, dm.SELECT_TOPK, K=a.topk) if a.topk
+            else dm.make_desc(a.T, a.d, a.H, a.E, dm.BF16, dm.SELECT_THRESHOLD, eps=a.eps))
     x = torch.randn(a.T, a.d, device="cuda").bfloat16()
     Wr = torch.randn(a.d, a.E, device="cuda") * 0.02
     layers = []
-    for _ in range(4):
+    for _ in range(8):
         W1 = (torch.randn(a.E, a.d, a.H, device="cuda") * 0.02).bfloat16()
         W2 = (torch.randn(a.E, a.H, a.d, device="cuda") * 0.02).bfloat16()
         pk = torch.empty(dm.dsmoe_packed_size(desc), dtype=torch.uint8, device="cuda")
@@ -75,12 +72,12 @@ def main():
     counts = torch.zeros(64, dtype=torch.int32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     for i in range(a.reps):
-        dm.dsmoe_layer_forward(desc, x, Wr, None, None, None, layers[i % 4], out, None, counts, ws, status)
+        dm.dsmoe_layer_forward(desc, x, Wr, None, None, None, layers[i % 8], out, None, counts, ws, status)
     torch.cuda.synchronize()
     print(f"T={a.T} d={a.d} H={a.H} E={a.E}: {int((counts[:a.E] > 0).sum())} experts selected, device status {int(status.item())}")
     L = dm.lib()
     buf = (ctypes.c_ulonglong * (192 * 32))()
-    for reader, names in (("dsmoe_trace_read_fused", FUSED_NAMES), ("dsmoe_trace_read", SMALL_NAMES)):
+    for reader, names in (("dsmoe_trace_read", SMALL_NAMES),):
         if not hasattr(L, reader) or getattr(L, reader)(buf) != 0:
             continue
         tr = np.frombuffer(buf, dtype=np.uint64).reshape(192, 32).astype(np.int64)
@@ -88,7 +85,7 @@ def main():
         if not live.any():
             continue
         t0 = tr[live, 0].min()
-        print(f"-- {reader[len('dsmoe_trace_read'):] or '_small'} kernel, last launch, {int(live.sum())} CTAs; microseconds after the first CTA's start: median / min / max")
+        print(f"-- small_layer_kernel, last launch, {int(live.sum())} CTAs; microseconds after the first CTA's start: median / min / max")
         for idx, name in names.items():
             col = tr[live, idx]
             col = col[col > 0]

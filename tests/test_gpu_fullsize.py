@@ -182,16 +182,15 @@ def test_both_aggregation_paths_full_size(cfg, kw, n, fuse):
         assert r["err"] <= TOL_BF16
 
 
-# ---------------------------------------------------------------- the few-token kernel (up to 7 tokens: one launch, no
-# hand-over between CTAs from the up- to the down-projection)
+# ---------------------------------------------------------------- a handful of tokens (a decoding step of a few sequences)
 
 FEW = [
     dict(T=1, d=2048, H=1024, E=32, mode=gi.MODE_THRESHOLD, eps=0.03),
     dict(T=3, d=512, H=256, E=16, mode=gi.MODE_TOPK, K=2),
     dict(T=7, d=320, H=192, E=8, mode=gi.MODE_ALL),                          # ragged column tiles of the down-projection
-    dict(T=5, d=4096, H=512, E=32, mode=gi.MODE_THRESHOLD, eps=0.03),        # every accumulator column of TMEM in use
-    dict(T=2, d=128, H=64, E=64, mode=gi.MODE_TOPK, K=3),                    # 4 units per expert: tiles cross experts
-    dict(T=4, d=64, H=6144, E=8, mode=gi.MODE_ALL),                          # 21 units per CTA: three M tiles
+    dict(T=5, d=4096, H=512, E=32, mode=gi.MODE_THRESHOLD, eps=0.03),
+    dict(T=2, d=128, H=64, E=64, mode=gi.MODE_TOPK, K=3),                    # tiles cross several experts
+    dict(T=4, d=64, H=6144, E=8, mode=gi.MODE_ALL),                          # wide experts, short reductions
     dict(T=6, d=256, H=128, E=33, mode=gi.MODE_THRESHOLD, eps=0.02, zipf_s=1.1),   # E % 4 != 0: the router's scalar loads
     dict(T=7, d=256, H=128, E=8, mode=gi.MODE_THRESHOLD, eps=0.999),         # nothing selected: zeros
     dict(T=1, d=64, H=64, E=1, mode=gi.MODE_ALL),
@@ -200,7 +199,7 @@ FEW = [
 
 
 @pytest.mark.parametrize("case", FEW, ids=[str(i) for i in range(len(FEW))])
-def test_few_token_kernel(case):
+def test_few_tokens(case):
     s = gi.LayerSpec(f"few{FEW.index(case)}", dtype="bf16", router_gain=3.0, **case)
     r = layer_parity(s)
     assert r["err_rows"] <= TOL_BF16 and r["err"] <= TOL_BF16, (r["err_rows"], r["err"])
