@@ -41,9 +41,11 @@ WORKLOADS = {
     "c3_separate": ("c3", dict(fuse_combine=2)),   # aggregation as a second kernel instead of inside the down-projection (see dsmoe.h)
     "c5": ("c5", dict(eps=0.01)),
     # output-token throughput as the paper measures it ("GPU Inference Analysis"): a decode loop in which layer i's
-    # output is layer i+1's input, 24 distinct layers (Table tab:model_arch: N_layer = 24 .. 36); W2 is drawn 16 times
-    # larger so that the activations keep their scale from layer to layer without the model's normalisation layers
-    "decode_loop_t8": ("c2", dict(T=8, w2_gain=16.0)), "decode_loop_t32": ("c2", dict(T=32, w2_gain=16.0)),
+    # output is layer i+1's input, 24 distinct layers (Table tab:model_arch: N_layer = 24 .. 36).  Between two layers
+    # the activations are brought back to unit RMS by one elementwise multiply (a torch op standing in for the model's
+    # normalisation layer, which is not part of this library), so that every layer's router sees inputs of the scale
+    # the threshold was calibrated on
+    "decode_loop_t8": ("c2", dict(T=8)), "decode_loop_t32": ("c2", dict(T=32)),
 }
 for _e in (0.0, 0.01, 0.05, 0.1, 0.2):
     WORKLOADS[f"c5_eps{_e}"] = ("c5", dict(eps=_e))
@@ -294,6 +296,7 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
         dm.dsmoe_layer_forward(desc, src, Wr_d, br_d, None, None, packed[i % n_layers], dst,
                                mask if want else None, counts if want else None, ws, status)
 
+    scales = []                                   # loop workloads: 1 / RMS of each layer's output (set by the pre-pass)
     if loop:
         def step(i, want=False):
             # one decoding step of a 24-layer stack: x -> layer 0 -> layer 1 -> ... (each layer its own weights)
@@ -301,6 +304,8 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
             for layer in range(n_layers):
                 dst = act[1 + layer % 2]
                 layer_call(layer, src, dst, want and layer == 0)
+                if scales:
+                    dst.mul_(scales[layer])
                 src = dst
     else:
         def step(i, want=False):
@@ -312,6 +317,20 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
     cnt = counts[:s.E].cpu().numpy()
     A = int(cnt.sum())
     n_act = int((cnt > 0).sum())
+    n_act_layers, rms_layers = [n_act], []
+    if loop:
+        # what each layer of the stack really selects on the activations it gets (outside the timed region)
+        n_act_layers, src = [], x_d
+        for layer in range(n_layers):
+            dst = act[1 + layer % 2]
+            layer_call(layer, src, dst, True)
+            torch.cuda.synchronize()
+            n_act_layers.append(int((counts[:s.E] > 0).sum().item()))
+            rms = dst.float().pow(2).mean().sqrt()
+            rms_layers.append(float(rms.item()))
+            scales.append((1.0 / rms).to(torch.bfloat16))
+            dst.mul_(scales[-1])
+            src = dst
     # selection statistics of this batch (stage calls, outside the timed region)
     scores = torch.empty((s.T, s.E), dtype=torch.float32, device="cuda")
     dm.dsmoe_router(desc, x_d, Wr_d, br_d, scores)
@@ -382,13 +401,14 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
 
     step_s = ms_total * 1e-3 / steps
     res = dict(value=value, ms_per_step=ms_total / steps, clocks=clocks, A=A, active_experts=n_act, stats=stats,
+               active_experts_per_layer=n_act_layers if loop else None, activation_rms_per_layer=rms_layers if loop else None,
                launches_per_step=kernels_per_step(s, decode) * calls_per_step, spec=s)
     if len(durs):
         durs = durs.reshape(steps, calls_per_step * timed_per_call)
         kernel_ms = float(durs.sum(axis=1).mean())        # time inside the dominant kernel per step
         capped = "sw_power_cap" in clocks["reasons"] or (clocks["sm_mhz"] and clocks["sm_max_mhz"] and
                                                           clocks["sm_mhz"] < 0.9 * clocks["sm_max_mhz"])
-        weight_bytes = 2.0 * n_act * s.d * s.H * 2.0 * calls_per_step
+        weight_bytes = 2.0 * sum(n_act_layers) * s.d * s.H * 2.0 * (1 if loop else calls_per_step)
         flops = 4.0 * A * s.d * s.H * calls_per_step
         if decode:
             # selected experts' weights (W1 and W2), each byte once, all inside one launch of small_layer_kernel
@@ -397,7 +417,7 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
             roof["frac"] = roof["achieved"] / roof["peak"]
             roof["frac_nominal"] = roof["achieved"] / NOMINAL["hbm"]
             roof["step_frac"] = weight_bytes / step_s / 1e9 / roof["peak"]
-            roof["algorithmic_per_launch"] = weight_bytes / calls_per_step
+            roof["algorithmic_per_launch"] = weight_bytes / calls_per_step      # loop workloads: the mean over the layers
         else:
             # both projections: two launches of umma_gemm_kernel per step.  Peak: the burst figure unless the clock
             # samples of this very region show the power cap (then the sustained one applies)
@@ -595,6 +615,8 @@ def main():
                 also.append({"workload": other, "value": r["value"], "unit": "tokens/s", "ms_per_step": r["ms_per_step"],
                              "steps": k, "roofline": r.get("roofline"), "clocks": r["clocks"], "assignments": r["A"],
                              "active_experts": r["active_experts"],
+                             "active_experts_per_layer": r["active_experts_per_layer"],
+                             "activation_rms_per_layer": r["activation_rms_per_layer"],
                              "near_threshold_1e-6": r["stats"]["near_threshold"]})
             line["also"] = also
     print(json.dumps(line))

@@ -208,3 +208,51 @@ def test_paper_shaped_prefill_topk(name, d, H, K):
     r = layer_parity(s, sample=256)
     assert r["A"] == 2048 * K
     assert r["err_rows"] <= TOL_BF16 and r["err"] <= TOL_BF16, (r["err_rows"], r["err"])
+
+
+# ---------------------------------------------------------------- the scaled models of the paper's speed test (Table tab:scaled)
+# DS-MoE-10B / 14B / 19B: 32 experts of width 640 / 768 / 896 at model width 5120 / 6144 / 7168, top-K 4.
+
+SCALED_SHAPES = [("10b", 5120, 640), ("14b", 6144, 768), ("19b", 7168, 896)]
+
+
+@pytest.mark.parametrize("name,d,H", SCALED_SHAPES, ids=[p[0] for p in SCALED_SHAPES])
+@pytest.mark.parametrize("T", [1, 32, 1024])
+def test_scaled_model_shapes(name, d, H, T):
+    s = gi.LayerSpec(f"scaled_{name}_t{T}", T=T, d=d, H=H, E=32, dtype="bf16", mode=gi.MODE_TOPK, K=4, router_gain=2.0)
+    r = layer_parity(s, sample=64 if T > 64 else None)
+    assert r["A"] == T * 4
+    assert r["err_rows"] <= TOL_BF16 and r["err"] <= TOL_BF16, (r["err_rows"], r["err"])
+
+
+# ---------------------------------------------------------------- a stack of layers: layer i's output is layer i + 1's input
+# (output-token throughput as the "GPU Inference Analysis" section measures it).  Every layer of the stack is checked
+# against the oracle on the very activations the previous layer produced on the GPU.
+
+@pytest.mark.parametrize("T", [1, 8, 40, 300])
+def test_stack_of_layers_feeding_one_another(T):
+    n_layers = 6
+    s = gi.LayerSpec(f"stack_t{T}", T=T, d=512, H=256, E=16, dtype="bf16", mode=gi.MODE_THRESHOLD, eps=0.04,
+                     router_gain=2.0, w2_gain=64.0)
+    x = gi.tokens(s)
+    x_d = None
+    rms = []
+    for layer in range(n_layers):
+        L = Layer(s, layer=layer)
+        if x_d is not None:
+            L.x_d, L.x = x_d, to_np(x_d)                      # the previous layer's bf16 output, bit for bit
+        out32 = L.forward(out_fp32=True).cpu().numpy()
+        out16 = L.forward(out_fp32=False)
+        assert torch.equal(out16, torch.from_numpy(out32).cuda().to(torch.bfloat16))
+        mask_gpu = to_np(L.mask)[:T].view(np.uint64)
+        S = oracle.router_scores(L.x, L.Wr, L.br)
+        mask_ref, _ = oracle.select(S, s.mode, s.eps, s.eps_normalized, s.K, s.min_k)
+        from harness import check_mask_against_oracle, rel_err_rows
+        check_mask_against_oracle(s, S, mask_gpu, mask_ref)
+        ref = oracle.layer(L.x, L.W1, L.W2, S, mask_gpu)
+        assert rel_err_rows(out32, ref) <= TOL_BF16
+        rms.append(float(np.sqrt(np.mean(ref ** 2))))
+        x_d = out16.clone()
+    from harness import record
+    record("layer_stack", T=T, layers=n_layers, rms_per_layer=rms)
+    assert all(np.isfinite(rms)) and rms[-1] > 0.0
