@@ -233,7 +233,7 @@ def test_scaled_model_shapes(name, d, H, T):
 def test_stack_of_layers_feeding_one_another(T):
     n_layers = 6
     s = gi.LayerSpec(f"stack_t{T}", T=T, d=512, H=256, E=16, dtype="bf16", mode=gi.MODE_THRESHOLD, eps=0.04,
-                     router_gain=2.0, w2_gain=64.0)
+                     router_gain=2.0, w2_gain=32.0)
     x = gi.tokens(s)
     x_d = None
     rms = []
