@@ -62,6 +62,7 @@ constexpr int kMaxDeviceSlots = 64;
 struct DeviceState {
     int sm_count = 0;
     bool attr_gemm = false, attr_small = false, attr_router_f32 = false, attr_router_bf16 = false;
+    int max_pairs = -1;   // CTA pairs of umma_gemm_kernel that can be resident at once; -1 not asked yet, 0 pairs unavailable
 };
 dsmoe_status device_state(DeviceState** out, int* device = nullptr);   // of the current device
 

@@ -14,6 +14,9 @@
 //   DENSE_DOWN  out[t,:] = sum over (e,j) of that h times W2[e][j,:] -- the router-weighted sum of
 //               Eq. 1 folded into the reduction dimension, so no grouping and no aggregation pass
 // small_layer_kernel: the whole layer for a handful of tokens (decode) in one cooperative launch.
+#include <climits>
+#include <cstdlib>
+
 #include "common.cuh"
 #include "router_device.cuh"
 #include "tensor_maps.cuh"
@@ -47,6 +50,24 @@ constexpr size_t SMEM_GEMM_BYTES = 1024 + (size_t)RING_BYTES + SHARED_BYTES;   /
 constexpr int CMB_WARPS = 12, CMB_COLS = 16, CMB_LD = CMB_COLS + 1;
 constexpr size_t SMEM_GEMM_CMB_BYTES = SMEM_GEMM_BYTES + (size_t)CMB_WARPS * 32 * CMB_LD * 4;
 static_assert(SMEM_GEMM_CMB_BYTES <= 227 * 1024, "shared memory of one CTA");
+
+// umma_gemm_kernel comes in two forms.  Alone, a CTA computes 128 x 256 tiles from a ring of 4 slots of 16 + 32 KB.
+// As a pair (a cluster of two CTAs, tcgen05 .cta_group::2), the two compute a 256 x 256 tile: each holds its own 128
+// rows of A and half of the B tile's rows, the even CTA issues MMAs that read both CTAs' shared memory and write
+// 128 accumulator rows into each CTA's tensor memory.  A slot is then 16 + 16 KB, so the ring holds 6 of them, and
+// a CTA brings 32 KB from L2 per 64-wide reduction block instead of 48 KB.
+#ifndef DSMOE_PAIR_GW
+#define DSMOE_PAIR_GW 6
+#endif
+template <bool PAIR>
+struct Geo {
+    static constexpr int ST = PAIR ? 6 : STAGES;                             // ring slots
+    static constexpr int B_BYTES = PAIR ? B_STAGE_BYTES / 2 : B_STAGE_BYTES; // this CTA's part of a B tile
+    static constexpr int GW = PAIR ? DSMOE_PAIR_GW : GATHER_WARPS;           // warps that gather rows of A
+    static constexpr int MT = PAIR ? 2 * BM : BM;                            // rows of a tile
+    static_assert(ST * (A_STAGE_BYTES + B_BYTES) == RING_BYTES, "both forms fill the same ring");
+    static_assert(GW % ST == 0 && ST <= MAX_STAGES, "whole warps per slot");
+};
 
 enum { GEMM_GROUPED = 0, GEMM_DENSE_UP = 1, GEMM_DENSE_DOWN = 2 };
 enum { EPI_GELU = 0, EPI_STORE = 1, EPI_COMBINE = 2, EPI_BWD = 3 };
@@ -103,7 +124,8 @@ struct GemmParams {
 };
 
 struct Tile {
-    int row0, rows_valid, e, n0, bn, nk, out_col0;
+    int row0, rows_valid, e, n0, bn, nk, out_col0;   // rows_valid <= 0: this CTA's half of a pair's tile lies past the rows
+    int row_safe;                                    // a row that exists (stands in for rows past the end)
 };
 
 // small_layer_kernel: the selected experts and the work partition and ring geometry that follow from them
@@ -120,7 +142,6 @@ struct Shared {
     uint32_t tmem_base;
     volatile int abort_flag;
     int bad_offsets;
-    int rowtok[GATHER_WARPS][BM / (GATHER_WARPS / STAGES)];                   // umma_gemm_kernel, gathered A: the source row of each tile row, per gathering warp
     int tile_prefix[kMaxExperts + 1];
     int seg0[kMaxExperts], seg1[kMaxExperts];
     unsigned long long active_mask;
@@ -134,8 +155,13 @@ struct Shared {
     volatile int spec_issued, spec_stop;   // producer -> MMA issuer: ring slots filled under geo[0]; no more will be
     volatile int up_arrived;               // epilogue -> producer: this CTA has arrived at the barrier between the projections
     volatile int mma_drained;              // MMA issuer -> producer: those slots are consumed, the ring is idle
-    float gate_s[BM], gate2_s[BM];
-    uint64_t mask_s[BM];                   // small_layer_kernel: every token's selection word
+    union {
+        int rowtok[(DSMOE_PAIR_GW > 8 ? DSMOE_PAIR_GW / 2 : 6) * BM];                // umma_gemm_kernel, gathered A: the source row of each tile row, per gathering warp
+        struct {                           // small_layer_kernel: router gates and every token's selection word
+            float gate_s[BM], gate2_s[BM];
+            uint64_t mask_s[BM];
+        };
+    };
 #ifdef DSMOE_TRACE
     unsigned long long trace[32];
 #endif
@@ -146,11 +172,42 @@ static_assert(sizeof(Shared) <= SHARED_BYTES, "Shared must fit its slot");
 // Diagnostic build only (-DDSMOE_TRACE): per-CTA time stamps (globaltimer ns) of small_layer_kernel's milestones.
 __device__ unsigned long long g_trace[192][32];
 #define TRACE(i) sh.trace[i] = ptx::globaltimer_ns()
+// ... and of umma_gemm_kernel: clock cycles its roles spent waiting, per CTA, for the last launch of each kind
+// (0 router logits, 1 up-projection, 2 down-projection or backward): [0] MMA issuer in all, [1] of these waiting for
+// operands, [2] for a free accumulator; [3] producer in all, [4] of these waiting for a free slot; [5] first epilogue
+// warp in all, [6] of these waiting for an accumulator; [7] tiles
+__device__ long long g_gemm_trace[3][192][8];
+#define GTRACE_T0(v) const long long v = clock64()
+#define GTRACE_ADD(slot, v) gtr[slot] += clock64() - (v)
 #else
 #define TRACE(i)
+#define GTRACE_T0(v)
+#define GTRACE_ADD(slot, v)
 #endif
 
-__device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f)); }
+// GeLU(v) = v Phi(v) with the exact Phi (the erf form, not the tanh form).  Phi comes from Abramowitz & Stegun's
+// rational approximation 7.1.28, erfc(z) = (1 + a1 z + ... + a6 z^6)^-16 with |error| <= 3e-7 for z >= 0 -- three
+// orders below the bf16 rounding of the result: Phi(v) = erfc(|v| / sqrt 2) / 2 for v < 0 and 1 minus that for
+// v >= 0, so the negative tail has no cancellation.  Six FMAs, one reciprocal, four squarings: about half the
+// instructions of erff, which matters because the GeLU epilogue of a tile costs the CUDA cores nearly as many issue
+// slots as its mainloop costs the tensor core.
+__device__ __forceinline__ float gelu_erf(float v) {
+    const float z = fabsf(v) * 0.70710678118654752440f;
+    float p = fmaf(z, 0.0000430638f, 0.0002765672f);
+    p = fmaf(z, p, 0.0001520143f);
+    p = fmaf(z, p, 0.0092705272f);
+    p = fmaf(z, p, 0.0422820123f);
+    p = fmaf(z, p, 0.0705230784f);
+    p = fmaf(z, p, 1.f);
+    float q;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(q) : "f"(p));   // p >= 1: one unit in the last place is plenty
+    q *= q;
+    q *= q;
+    q *= q;
+    q *= q;
+    const float tail = 0.5f * q;                    // Phi(-|v|)
+    return v * (v < 0.f ? tail : 1.f - tail);
+}
 
 // The packed weights are block-major along the reduction: [E][k / 64][n][64], so the tile (64 k, rows n0..) of
 // reduction block kb is the `rows` consecutive 128-byte rows starting at wrow(kb, n0, N) of a [E][(K/64)*N][64]
@@ -158,26 +215,33 @@ __device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.f + er
 __device__ __forceinline__ int wrow(int kb, int n0, int N) { return kb * N + n0; }
 
 // Weight rows [row0, row0 + rows) of expert e (see wrow): power-of-two boxes, largest first.
+template <bool PAIR = false>
 __device__ __forceinline__ void load_weight_rows(const BMaps* maps, uint32_t dst, uint32_t bar, int row0, int rows,
                                                  int e, int x0 = 0) {
     int done = 0;
 #pragma unroll
     for (int lvl = 4; lvl >= 0; --lvl) {
         if ((rows - done) >= (16 << lvl)) {
-            ptx::tma_load_3d(dst + done * (BK * 2), &maps->m[lvl], bar, x0, row0 + done, e);
+            if (PAIR) ptx::tma_load_3d_pair(dst + done * (BK * 2), &maps->m[lvl], bar, x0, row0 + done, e);
+            else ptx::tma_load_3d(dst + done * (BK * 2), &maps->m[lvl], bar, x0, row0 + done, e);
             done += 16 << lvl;
         }
     }
 }
 
+template <bool PAIR>
 __device__ __forceinline__ int total_tiles(const GemmParams& P, const Shared& sh) {
+    constexpr int MT = Geo<PAIR>::MT;
     const int ntn = (P.n_per_expert + BN - 1) / BN;
     if (P.mode == GEMM_GROUPED) return sh.tile_prefix[P.E];
-    const int mt = (P.rows + BM - 1) / BM;
+    const int mt = (P.rows + MT - 1) / MT;
     return P.mode == GEMM_DENSE_UP ? mt * ntn * P.E : mt * ntn;
 }
 
-__device__ __forceinline__ Tile decode_tile(const GemmParams& P, const Shared& sh, int id) {
+// Tile `id` as CTA `half` (0, or 1 for the odd CTA of a pair) sees it: its own 128 rows, the whole column range.
+template <bool PAIR>
+__device__ __forceinline__ Tile decode_tile(const GemmParams& P, const Shared& sh, int id, int half) {
+    constexpr int MT = Geo<PAIR>::MT;
     Tile t;
     const int kbpe = P.k_per_expert / BK;
     if (P.mode == GEMM_GROUPED) {
@@ -185,20 +249,22 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& P, const Shared& s
         while (e + 1 < P.E && id >= sh.tile_prefix[e + 1]) ++e;
         const int local = id - sh.tile_prefix[e];
         const int cnt = sh.seg1[e] - sh.seg0[e];
-        const int mtiles = (cnt + BM - 1) / BM;
+        const int mtiles = (cnt + MT - 1) / MT;
         const int nt = local / mtiles, mt = local % mtiles;
         t.e = e;
-        t.row0 = sh.seg0[e] + mt * BM;
+        t.row0 = sh.seg0[e] + mt * MT + half * BM;
         t.rows_valid = min(BM, sh.seg1[e] - t.row0);
+        t.row_safe = sh.seg0[e];
         t.n0 = nt * BN;
         t.nk = kbpe;
         t.out_col0 = t.n0;
     } else {
-        const int mtiles = (P.rows + BM - 1) / BM;
+        const int mtiles = (P.rows + MT - 1) / MT;
         const int ntn = (P.n_per_expert + BN - 1) / BN;
         const int mt = id % mtiles, rest = id / mtiles;
-        t.row0 = mt * BM;
+        t.row0 = mt * MT + half * BM;
         t.rows_valid = min(BM, P.rows - t.row0);
+        t.row_safe = 0;
         if (P.mode == GEMM_DENSE_UP) {
             t.e = rest / ntn;
             t.n0 = (rest % ntn) * BN;
@@ -235,24 +301,39 @@ __device__ __forceinline__ bool flag_wait_ge(const int* flag, int target, volati
     }
 }
 
-__global__ void __launch_bounds__(GATHER_THREADS, 1)
+// A barrier of this CTA that (in a pair) the other CTA or its tensor core also signals
+template <bool PAIR>
+__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    return PAIR ? ptx::mbar_wait_cluster(bar, parity, abort_flag) : ptx::mbar_wait(bar, parity, abort_flag);
+}
+
+template <bool PAIR>
+__global__ void __launch_bounds__((PAIR && NUM_THREADS + 32 * DSMOE_PAIR_GW > GATHER_THREADS) ? NUM_THREADS + 32 * DSMOE_PAIR_GW : GATHER_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ BMaps tmB, const GemmParams P) {
+    constexpr int ST = Geo<PAIR>::ST, B_BYTES = Geo<PAIR>::B_BYTES, GW = Geo<PAIR>::GW, MT = Geo<PAIR>::MT;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;             // 128-byte swizzle wants 1024-byte aligned tiles
-    const uint32_t smA = base, smB = base + STAGES * A_STAGE_BYTES;
+    const uint32_t smA = base, smB = base + ST * A_STAGE_BYTES;
     Shared& sh = *reinterpret_cast<Shared*>(smem_raw + (base - raw) + RING_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // pair: `half` is this CTA's place in it (0 issues the MMAs and owns the barriers both CTAs signal); the pair
+    // walks the tiles pair_id, pair_id + pairs, ...
+    const int half = PAIR ? (int)ptx::cluster_ctarank() : 0;
+    const int first_tile = PAIR ? (int)blockIdx.x / 2 : (int)blockIdx.x;
+    const int tile_step = PAIR ? (int)gridDim.x / 2 : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&sh.full[s]), P.gather ? 1 + 32 * (GATHER_WARPS / STAGES) : 1);   // + one arrival per thread of the gathering warps
+        for (int s = 0; s < ST; ++s) {
+            // the producer's arrival (pair: the even CTA's) + one per gathering warp of the slot (pair: of either CTA)
+            const int gather_arrivals = (PAIR ? 2 : 1) * (GW / ST);
+            ptx::mbar_init(ptx::smem_u32(&sh.full[s]), P.gather ? 1 + gather_arrivals : 1);
             ptx::mbar_init(ptx::smem_u32(&sh.empty[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(ptx::smem_u32(&sh.tfull[a]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh.tempty[a]), P.epi == EPI_COMBINE ? CMB_WARPS : 4);
+            ptx::mbar_init(ptx::smem_u32(&sh.tempty[a]), (P.epi == EPI_COMBINE ? CMB_WARPS : 4) * (PAIR ? 2 : 1));
         }
         sh.abort_flag = 0;
         sh.bad_offsets = 0;
@@ -277,19 +358,25 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         int run = 0;
         for (int e = 0; e < P.E; ++e) {
             sh.tile_prefix[e] = run;
-            run += ((sh.seg1[e] - sh.seg0[e] + BM - 1) / BM) * ntn;
+            run += ((sh.seg1[e] - sh.seg0[e] + MT - 1) / MT) * ntn;
         }
         sh.tile_prefix[P.E] = run;
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), TMEM_COLS);
-        ptx::tmem_relinquish();
+        if (PAIR) {
+            ptx::tmem_alloc_pair(ptx::smem_u32(&sh.tmem_base), TMEM_COLS);
+            ptx::tmem_relinquish_pair();
+        } else {
+            ptx::tmem_alloc(ptx::smem_u32(&sh.tmem_base), TMEM_COLS);
+            ptx::tmem_relinquish();
+        }
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    if (PAIR) ptx::cluster_sync();      // both CTAs' barriers and tensor memory exist before either signals the other
+    else __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = sh.tmem_base;
-    const int ntiles = total_tiles(P, sh);
+    const int ntiles = total_tiles<PAIR>(P, sh);
     const int kbpe = P.k_per_expert / BK;
 
     if (warp == 0) {
@@ -298,15 +385,24 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int s = 0;
             uint32_t ph = 0;
             bool alive = true;
-            for (int id = blockIdx.x; id < ntiles && alive; id += gridDim.x) {
-                const Tile t = decode_tile(P, sh, id);
+#ifdef DSMOE_TRACE
+            long long gtr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
+            GTRACE_T0(t_all);
+            for (int id = first_tile; id < ntiles && alive; id += tile_step) {
+                const Tile t = decode_tile<PAIR>(P, sh, id, half);
                 for (int i = 0; i < t.nk; ++i) {
-                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
+                    GTRACE_T0(t_w);
+                    if (!bar_wait<PAIR>(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
                         alive = false;
                         break;
                     }
-                    const uint32_t bar = ptx::smem_u32(&sh.full[s]);
-                    ptx::mbar_expect_tx(bar, (P.gather ? 0u : (uint32_t)A_STAGE_BYTES) + (uint32_t)t.bn * BK * 2);
+                    GTRACE_ADD(4, t_w);
+                    // pair: the bytes of both CTAs' copies are counted at the even CTA's barrier, which its producer arms
+                    const uint32_t bar = PAIR ? ptx::map_to_cta(ptx::smem_u32(&sh.full[s]), 0) : ptx::smem_u32(&sh.full[s]);
+                    const uint32_t bytes = (P.gather ? 0u : (uint32_t)A_STAGE_BYTES) + (uint32_t)t.bn * BK * 2;
+                    if (!PAIR) ptx::mbar_expect_tx(bar, bytes);
+                    else if (half == 0) ptx::mbar_expect_tx(ptx::smem_u32(&sh.full[s]), bytes + (P.gather ? 0u : (uint32_t)A_STAGE_BYTES));
                     int a_col, b_e, b_k;
                     if (P.mode == GEMM_DENSE_DOWN) {
                         b_e = i / kbpe;
@@ -317,19 +413,35 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         b_k = i * BK;
                         a_col = b_k;
                     }
-                    if (!P.gather) ptx::tma_load_2d(smA + s * A_STAGE_BYTES, &tmA, bar, a_col, t.row0);
-                    // full-width tiles take the one 256-row copy directly (measurably faster than walking the
-                    // box sizes); only a ragged last column tile needs the decomposition
+                    if (!P.gather) {
+                        if (PAIR) ptx::tma_load_2d_pair(smA + s * A_STAGE_BYTES, &tmA, bar, a_col, t.row0);
+                        else ptx::tma_load_2d(smA + s * A_STAGE_BYTES, &tmA, bar, a_col, t.row0);
+                    }
+                    // full-width tiles take the one 256-row copy (pair: this CTA's 128 rows) directly (measurably
+                    // faster than walking the box sizes); only a ragged last column tile needs the decomposition
                     const int b_x = P.b_plain ? b_k : 0;
-                    const int b_row = P.b_plain ? t.n0 : wrow(b_k / BK, t.n0, P.n_per_expert);
-                    if (t.bn == BN) ptx::tma_load_3d(smB + s * B_STAGE_BYTES, &tmB.m[4], bar, b_x, b_row, b_e);
-                    else load_weight_rows(&tmB, smB + s * B_STAGE_BYTES, bar, b_row, t.bn, b_e, b_x);
-                    if (++s == STAGES) {
+                    const int b_rows = PAIR ? t.bn / 2 : t.bn;
+                    const int b_row = (P.b_plain ? t.n0 : wrow(b_k / BK, t.n0, P.n_per_expert)) + half * b_rows;
+                    if (t.bn == BN) {
+                        if (PAIR) ptx::tma_load_3d_pair(smB + s * B_BYTES, &tmB.m[3], bar, b_x, b_row, b_e);
+                        else ptx::tma_load_3d(smB + s * B_BYTES, &tmB.m[4], bar, b_x, b_row, b_e);
+                    } else {
+                        load_weight_rows<PAIR>(&tmB, smB + s * B_BYTES, bar, b_row, b_rows, b_e, b_x);
+                    }
+                    if (++s == ST) {
                         s = 0;
                         ph ^= 1u;
                     }
                 }
             }
+#ifdef DSMOE_TRACE
+            GTRACE_ADD(3, t_all);
+            if (blockIdx.x < 192) {
+                long long* g = g_gemm_trace[P.epi == EPI_GELU ? 1 : (P.n_per_expert <= 192 ? 0 : 2)][blockIdx.x];
+                g[3] = gtr[3];
+                g[4] = gtr[4];
+            }
+#endif
             if (!alive) {
                 // copies already issued still land in this CTA's shared memory: give them time
                 const uint64_t t0 = ptx::globaltimer_ns();
@@ -339,84 +451,133 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (lane == 0 && half == 0) {
             int s = 0, acc = 0;
             uint32_t ph = 0, aph = 0;
             bool alive = true;
-            for (int id = blockIdx.x; id < ntiles && alive; id += gridDim.x) {
-                const Tile t = decode_tile(P, sh, id);
-                if (!ptx::mbar_wait(ptx::smem_u32(&sh.tempty[acc]), aph ^ 1u, &sh.abort_flag)) break;
+#ifdef DSMOE_TRACE
+            long long gtr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
+            GTRACE_T0(t_all);
+            for (int id = first_tile; id < ntiles && alive; id += tile_step) {
+                const Tile t = decode_tile<PAIR>(P, sh, id, 0);
+                GTRACE_T0(t_acc);
+                if (!bar_wait<PAIR>(ptx::smem_u32(&sh.tempty[acc]), aph ^ 1u, &sh.abort_flag)) break;
+                GTRACE_ADD(2, t_acc);
+#ifdef DSMOE_TRACE
+                gtr[7] += 1;
+#endif
                 ptx::tc_fence_after();
-                const uint32_t idesc = ptx::make_idesc_bf16(BM, (uint32_t)t.bn);
+                const uint32_t idesc = ptx::make_idesc_bf16(MT, (uint32_t)t.bn);
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 for (int i = 0; i < t.nk; ++i) {
-                    if (!ptx::mbar_wait(ptx::smem_u32(&sh.full[s]), ph, &sh.abort_flag)) {
+                    GTRACE_T0(t_w);
+                    if (!bar_wait<PAIR>(ptx::smem_u32(&sh.full[s]), ph, &sh.abort_flag)) {
                         alive = false;
                         break;
                     }
+                    GTRACE_ADD(1, t_w);
                     ptx::tc_fence_after();
-                    const uint32_t a0 = smA + s * A_STAGE_BYTES, b0 = smB + s * B_STAGE_BYTES;
+                    const uint32_t a0 = smA + s * A_STAGE_BYTES, b0 = smB + s * B_BYTES;
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        ptx::umma_bf16(d_tmem, ptx::make_desc_k_sw128(a0 + k * 32), ptx::make_desc_k_sw128(b0 + k * 32),
-                                       idesc, (uint32_t)((i | k) != 0));
-                    ptx::umma_commit(ptx::smem_u32(&sh.empty[s]));   // slot reusable once these MMAs have read it
-                    if (++s == STAGES) {
+                    for (int k = 0; k < BK / 16; ++k) {
+                        if (PAIR)
+                            ptx::umma_bf16_pair(d_tmem, ptx::make_desc_k_sw128(a0 + k * 32), ptx::make_desc_k_sw128(b0 + k * 32),
+                                                idesc, (uint32_t)((i | k) != 0));
+                        else
+                            ptx::umma_bf16(d_tmem, ptx::make_desc_k_sw128(a0 + k * 32), ptx::make_desc_k_sw128(b0 + k * 32),
+                                           idesc, (uint32_t)((i | k) != 0));
+                    }
+                    // slot reusable once these MMAs have read it (pair: in both CTAs)
+                    if (PAIR) {
+                        ptx::umma_commit_pair(ptx::smem_u32(&sh.empty[s]));
+                        ptx::umma_commit_pair(ptx::map_to_cta(ptx::smem_u32(&sh.empty[s]), 1));
+                    } else {
+                        ptx::umma_commit(ptx::smem_u32(&sh.empty[s]));
+                    }
+                    if (++s == ST) {
                         s = 0;
                         ph ^= 1u;
                     }
                 }
                 if (!alive) break;
-                ptx::umma_commit(ptx::smem_u32(&sh.tfull[acc]));      // accumulator complete
+                // accumulator complete (pair: each CTA's epilogue reads its own 128 rows)
+                if (PAIR) {
+                    ptx::umma_commit_pair(ptx::smem_u32(&sh.tfull[acc]));
+                    ptx::umma_commit_pair(ptx::map_to_cta(ptx::smem_u32(&sh.tfull[acc]), 1));
+                } else {
+                    ptx::umma_commit(ptx::smem_u32(&sh.tfull[acc]));
+                }
                 if (++acc == 2) {
                     acc = 0;
                     aph ^= 1u;
                 }
             }
+#ifdef DSMOE_TRACE
+            GTRACE_ADD(0, t_all);
+            if (blockIdx.x < 192) {
+                long long* g = g_gemm_trace[P.epi == EPI_GELU ? 1 : (P.n_per_expert <= 192 ? 0 : 2)][blockIdx.x];
+                g[0] = gtr[0];
+                g[1] = gtr[1];
+                g[2] = gtr[2];
+                g[7] = gtr[7];
+            }
+#endif
         }
     } else if (warp >= 6 && P.gather) {
-        // ------------------------------------------------------------ gather (8 warps, grouped up-projection only)
-        // Warps j and j + 4 bring the two halves of the A tiles of the ring stages j, j + 4, ... of this CTA's
-        // sequence: per stage, 16 cp.async instructions each, an instruction covering 4 rows x 128 bytes (8 lanes x 16 bytes per row), written in the
-        // 128-byte-swizzle order the MMA descriptors expect (chunk c of row r sits at chunk c ^ (r % 8)).  It then
-        // waits for its copies, makes them visible to the tensor core's proxy and arrives at the stage's barrier;
-        // while it waits, the other three warps' stages are in flight.
-        constexpr int PARTS = GATHER_WARPS / STAGES, ROWS = BM / PARTS;   // warps per stage, rows per warp
-        const int team = (warp - 6) % STAGES, part = (warp - 6) / STAGES;
-        int* rowtok = sh.rowtok[warp - 6];
+        // ------------------------------------------------------------ gather (grouped up-projection only)
+        // Alone, 8 warps: warps j and j + 4 bring the two halves of the A tiles of the ring stages j, j + 4, ... of
+        // this CTA's sequence; in a pair, 6 warps: warp j brings the whole A tile of the stages j, j + 6, ....  An
+        // instruction covers 4 rows x 128 bytes (8 lanes x 16 bytes per row), written in the 128-byte-swizzle order
+        // the MMA descriptors expect (chunk c of row r sits at chunk c ^ (r % 8)).  The warp then waits for its
+        // copies, makes them visible to the tensor core's proxy and arrives at the stage's barrier; while it
+        // waits, the other warps' stages are in flight.
+        if (warp >= 6 + GW) goto teardown;
+        constexpr int PARTS = GW / ST, ROWS = BM / PARTS;   // warps per stage, rows per warp
+        const int team = (warp - 6) % ST, part = (warp - 6) / ST;
+        int* rowtok = sh.rowtok + (warp - 6) * ROWS;
         const int lr = lane >> 3, lc = lane & 7;
         int n = 0;                       // stages of the sequence seen so far
         bool alive = true;
-        for (int id = blockIdx.x; id < ntiles && alive; id += gridDim.x) {
-            const Tile t = decode_tile(P, sh, id);
+        for (int id = first_tile; id < ntiles && alive; id += tile_step) {
+            const Tile t = decode_tile<PAIR>(P, sh, id, half);
             __syncwarp();
 #pragma unroll
             for (int j = 0; j < ROWS / 32; ++j) {
                 const int r = part * ROWS + lane + 32 * j;
-                const int tok = P.gather[t.row0 + (r < t.rows_valid ? r : 0)];   // rows past the segment: nobody reads them
+                const int tok = P.gather[r < t.rows_valid ? t.row0 + r : t.row_safe];   // rows past the segment: nobody reads them
                 rowtok[lane + 32 * j] = min(max(tok, 0), P.gather_rows - 1);
             }
             __syncwarp();
+            // this lane's rows (4 jj + lane / 8 of the warp's share): where they start in the source, in 16-byte units
+            uint32_t src_off[ROWS / 4];
+#pragma unroll
+            for (int jj = 0; jj < ROWS / 4; ++jj)
+                src_off[jj] = (uint32_t)(((size_t)rowtok[jj * 4 + lr] * P.k_per_expert * 2) >> 4);
             for (int i = 0; i < t.nk; ++i, ++n) {
-                if ((n & (STAGES - 1)) != team) continue;
-                const int s = n & (STAGES - 1);
-                const uint32_t ph = (uint32_t)(n / STAGES) & 1u;
-                if (!ptx::mbar_wait(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
+                if (n % ST != team) continue;
+                const int s = n % ST;
+                const uint32_t ph = (uint32_t)(n / ST) & 1u;
+                if (!bar_wait<PAIR>(ptx::smem_u32(&sh.empty[s]), ph ^ 1u, &sh.abort_flag)) {
                     alive = false;
                     break;
                 }
                 const uint32_t dst0 = smA + s * A_STAGE_BYTES;
                 const char* src0 = static_cast<const char*>(P.gather_src) + (size_t)i * (BK * 2) + lc * 16;
-#pragma unroll 8
+#pragma unroll
                 for (int jj = 0; jj < ROWS / 4; ++jj) {
                     const int rl = jj * 4 + lr, r = part * ROWS + rl;
                     ptx::cp_async16(dst0 + (uint32_t)r * (BK * 2) + (uint32_t)((lc ^ (r & 7)) << 4),
-                                    src0 + (size_t)rowtok[rl] * P.k_per_expert * 2);
+                                    src0 + ((size_t)src_off[jj] << 4));
                 }
                 ptx::cp_async_commit();
                 ptx::cp_async_wait<0>();
                 ptx::fence_proxy_async();
-                ptx::mbar_arrive(ptx::smem_u32(&sh.full[s]));
+                __syncwarp();              // every lane's rows are in place and fenced: one arrival for the warp
+                if (lane == 0) {
+                    if (PAIR) ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&sh.full[s]), 0));
+                    else ptx::mbar_arrive(ptx::smem_u32(&sh.full[s]));
+                }
             }
         }
     } else if (warp < 6 || P.epi == EPI_COMBINE) {
@@ -424,10 +585,21 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int q = warp & 3;
         int acc = 0;
         uint32_t aph = 0;
-        for (int id = blockIdx.x; id < ntiles; id += gridDim.x) {
-            const Tile t = decode_tile(P, sh, id);
+        // pair: the accumulators are free again once both CTAs' epilogues have read them; the even CTA's issuer waits
+        const auto release_acc = [&](int a) {
+            if (PAIR) ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&sh.tempty[a]), 0));
+            else ptx::mbar_arrive(ptx::smem_u32(&sh.tempty[a]));
+        };
+#ifdef DSMOE_TRACE
+        long long gtr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
+        GTRACE_T0(t_all);
+        for (int id = first_tile; id < ntiles; id += tile_step) {
+            const Tile t = decode_tile<PAIR>(P, sh, id, half);
             // the TMEM reads below are warp-collective: the warp leaves as one
-            if (__any_sync(0xffffffffu, !ptx::mbar_wait(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag))) break;
+            GTRACE_T0(t_w);
+            if (__any_sync(0xffffffffu, !bar_wait<PAIR>(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag))) break;
+            GTRACE_ADD(6, t_w);
             ptx::tc_fence_after();
             const int row = q * 32 + lane;
             const bool valid = row < t.rows_valid;
@@ -457,7 +629,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 bool ok = true;
                 if (prev >= 0 && warp_has_rows) {
                     if (lane == 0) {
-                        const int target = CMB_WARPS * ((sh.seg1[prev] - sh.seg0[prev] + BM - 1) / BM);
+                        const int target = CMB_WARPS * (PAIR ? 2 : 1) * ((sh.seg1[prev] - sh.seg0[prev] + MT - 1) / MT);
                         ok = flag_wait_ge(P.tile_done + prev * ntn + nt, target, &sh.abort_flag);
                     }
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -529,7 +701,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    ptx::mbar_arrive(ptx::smem_u32(&sh.tempty[acc]));
+                    release_acc(acc);
                     __threadfence();                       // the warp's sums are visible before its arrival is
                     atomicAdd(P.tile_done + t.e * ntn + nt, 1);
                 }
@@ -577,7 +749,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.tempty[acc]));
+                if (lane == 0) release_acc(acc);
                 if (++acc == 2) {
                     acc = 0;
                     aph ^= 1u;
@@ -619,20 +791,31 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.tempty[acc]));
+            if (lane == 0) release_acc(acc);
             if (++acc == 2) {
                 acc = 0;
                 aph ^= 1u;
             }
         }
+#ifdef DSMOE_TRACE
+        GTRACE_ADD(5, t_all);
+        if (warp == 2 && lane == 0 && blockIdx.x < 192) {
+            long long* g = g_gemm_trace[P.epi == EPI_GELU ? 1 : (P.n_per_expert <= 192 ? 0 : 2)][blockIdx.x];
+            g[5] = gtr[5];
+            g[6] = gtr[6];
+        }
+#endif
     }
 
     // ---------------------------------------------------------------- teardown
+teardown:
     ptx::tc_fence_before();
-    __syncthreads();
+    if (PAIR) ptx::cluster_sync();      // neither CTA frees tensor memory or leaves while the other may still use or signal it
+    else __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+        if (PAIR) ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
+        else ptx::tmem_dealloc(tmem_base, TMEM_COLS);
     }
     if (threadIdx.x == 0 && P.dev_status) {
         if (sh.abort_flag) *P.dev_status = DSMOE_ERR_TIMEOUT;
@@ -1596,24 +1779,77 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 
 // ---------------------------------------------------------------- host side
 
+// DSMOE_GEMM_PAIR=0 in the environment keeps umma_gemm_kernel to single CTAs, =1 pairs wherever the shapes allow
+// (tuning aid); unset, launch_gemm decides.
+int pair_override() {
+    const char* e = getenv("DSMOE_GEMM_PAIR");     // read at every launch: a test switches it between calls
+    return e && *e ? atoi(e) : -1;
+}
+
+// pair_tiles: an upper bound of the number of 256-row tiles (INT_MAX where only the device knows, as in the grouped
+// modes); 0 = never pair (the caller's shapes do not allow it).
 dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams& P, int grid, cudaStream_t s,
-                         bool may_time = true) {
+                         bool may_time = true, int pair_tiles = 0) {
     DeviceState* st = nullptr;
     DSMOE_TRY(device_state(&st));
     if (!st->attr_gemm) {
-        DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_CMB_BYTES));
+        DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_CMB_BYTES));
+        DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_CMB_BYTES));
         st->attr_gemm = true;
     }
+    int threads = (P.gather || P.epi == EPI_COMBINE) ? GATHER_THREADS : NUM_THREADS;
+    const size_t smem = P.epi == EPI_COMBINE ? SMEM_GEMM_CMB_BYTES : SMEM_GEMM_BYTES;
+    if (st->max_pairs < 0) {
+        // how many clusters of two CTAs fit the device at once (the persistent kernel launches no more)
+        cudaLaunchConfig_t q{};
+        q.gridDim = dim3(2 * (st->sm_count / 2));
+        q.blockDim = dim3(GATHER_THREADS);
+        q.dynamicSmemBytes = SMEM_GEMM_CMB_BYTES;
+        cudaLaunchAttribute qa[1];
+        qa[0].id = cudaLaunchAttributeClusterDimension;
+        qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+        q.attrs = qa; q.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, umma_gemm_kernel<true>, &q) != cudaSuccess) {
+            cudaGetLastError();
+            n = 0;
+        }
+        st->max_pairs = n < st->sm_count / 2 ? n : st->sm_count / 2;
+    }
+    // Measured (C3, C4 and the paper's shapes): pairs gain 3 to 8 % where a long mainloop runs against a light
+    // epilogue (plain stores after a reduction of 1024 or more), lose up to 9 % under the GeLU and gathering
+    // up-projections and on short reductions, and change nothing under the aggregating epilogue.
+    bool pair = pair_tiles > 0 && st->max_pairs > 0 && (P.n_per_expert % 64) == 0;
+    if (pair_override() == 0) pair = false;
+    else if (pair && pair_override() != 1)
+        pair = P.epi == EPI_STORE && pair_tiles >= st->max_pairs && (P.mode == GEMM_DENSE_DOWN || P.k_per_expert >= 1024);
     int timed = -1;
     if (may_time) DSMOE_TRY(timing_begin(s, &timed));
-    const int threads = (P.gather || P.epi == EPI_COMBINE) ? GATHER_THREADS : NUM_THREADS;
-    if (P.epi == EPI_COMBINE) {
+    if (pair) {
+        if (P.gather) threads = NUM_THREADS + 32 * Geo<true>::GW;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(2 * (pair_tiles < st->max_pairs ? pair_tiles : st->max_pairs));
+        cfg.blockDim = dim3(threads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = s;
+        cudaLaunchAttribute at[2];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        int na = 1;
+        if (P.epi == EPI_COMBINE) {      // its epilogues wait for one another's tiles: every CTA must be resident
+            at[na].id = cudaLaunchAttributeCooperative;
+            at[na].val.cooperative = 1;
+            ++na;
+        }
+        cfg.attrs = at; cfg.numAttrs = na;
+        DSMOE_CUDA_TRY(cudaLaunchKernelEx(&cfg, umma_gemm_kernel<true>, a, b, P));
+    } else if (P.epi == EPI_COMBINE) {
         // its epilogues wait for one another's tiles: every CTA must be resident
         void* args[] = {const_cast<CUtensorMap*>(&a), const_cast<BMaps*>(&b), const_cast<GemmParams*>(&P)};
-        DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(umma_gemm_kernel), dim3(grid), dim3(threads),
-                                                   args, SMEM_GEMM_CMB_BYTES, s));
+        DSMOE_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(umma_gemm_kernel<false>), dim3(grid), dim3(threads),
+                                                   args, smem, s));
     } else {
-        umma_gemm_kernel<<<grid, threads, SMEM_GEMM_BYTES, s>>>(a, b, P);
+        umma_gemm_kernel<false><<<grid, threads, smem, s>>>(a, b, P);
         DSMOE_CUDA_TRY(cudaGetLastError());
     }
     DSMOE_TRY(timing_end(s, timed));
@@ -1697,6 +1933,9 @@ dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const 
 extern "C" __attribute__((visibility("default"))) int dsmoe_trace_read(unsigned long long* out) {
     return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(unsigned long long) * 192 * 32);
 }
+extern "C" __attribute__((visibility("default"))) int dsmoe_gemm_trace_read(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_gemm_trace, sizeof(long long) * 3 * 192 * 8);
+}
 #endif
 
 bool umma_supported(const dsmoe_layer_desc& p) {
@@ -1744,8 +1983,12 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
         down.tokens = p.T;
         DSMOE_CUDA_TRY(cudaMemsetAsync(cmb->tile_done, 0, (size_t)p.E * ceil_div(p.d, BN) * sizeof(int), s));
     }
-    DSMOE_TRY(launch_gemm(*mA1, *mB1, up, sm_count(), s));
-    DSMOE_TRY(launch_gemm(*mA2, *mB2, down, sm_count(), s));
+    // 256-row tiles (CTA pairs) waste little only where experts hold many rows; the host knows their number for a
+    // top-K selection alone (an upper bound otherwise), so only there may the launches pair on their own
+    const long long known = p.mode == DSMOE_SELECT_TOPK ? (long long)p.T * (p.K < p.E ? p.K : p.E) : 0;
+    const int pair_tiles = known >= 1024ll * p.E ? INT_MAX : (pair_override() == 1 ? INT_MAX : 0);
+    DSMOE_TRY(launch_gemm(*mA1, *mB1, up, sm_count(), s, true, pair_tiles));
+    DSMOE_TRY(launch_gemm(*mA2, *mB2, down, sm_count(), s, true, pair_tiles));
     return DSMOE_OK;
 }
 
@@ -1836,8 +2079,9 @@ dsmoe_status launch_layer_umma(const dsmoe_layer_desc& p, const void* x, const v
     down.rows = p.T; down.out = out; down.ld_out = p.d; down.out_f32 = p.out_fp32 ? 1 : 0; down.dev_status = dev_status;
     const int mt = ceil_div(p.T, BM);
     const int tiles_up = mt * ceil_div(p.H, BN) * p.E, tiles_down = mt * ceil_div(p.d, BN);
-    DSMOE_TRY(launch_gemm(*mA1, *mB1, up, tiles_up < sm_count() ? tiles_up : sm_count(), s));
-    DSMOE_TRY(launch_gemm(*mA2, *mB2, down, tiles_down < sm_count() ? tiles_down : sm_count(), s));
+    const int mt2 = ceil_div(p.T, 2 * BM);
+    DSMOE_TRY(launch_gemm(*mA1, *mB1, up, tiles_up < sm_count() ? tiles_up : sm_count(), s, true, mt2 * ceil_div(p.H, BN) * p.E));
+    DSMOE_TRY(launch_gemm(*mA2, *mB2, down, tiles_down < sm_count() ? tiles_down : sm_count(), s, true, mt2 * ceil_div(p.d, BN)));
     if (counts_out) {
         int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
         int32_t* offsets = reinterpret_cast<int32_t*>(ws + L.offsets);
@@ -1883,8 +2127,9 @@ dsmoe_status launch_dense_backward(const dsmoe_layer_desc& p, const void* x, con
     const int ntn = ceil_div(p.H, BN);
     const int tiles = ceil_div(p.T, BM) * ntn * p.E;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    DSMOE_TRY(launch_gemm(*mX, *mB1, up, grid, s));
-    DSMOE_TRY(launch_gemm(*mdO, *mB2, bw, grid, s));
+    const int pair_tiles = ceil_div(p.T, 2 * BM) * ntn * p.E;
+    DSMOE_TRY(launch_gemm(*mX, *mB1, up, grid, s, true, pair_tiles));
+    DSMOE_TRY(launch_gemm(*mdO, *mB2, bw, grid, s, true, pair_tiles));
     const long long n = (long long)p.T * p.E;
     bwd_finish_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(dot_part, dS, n, ntn);
     DSMOE_CUDA_TRY(cudaGetLastError());
