@@ -261,7 +261,11 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& P, const Shared& s
     } else {
         const int mtiles = (P.rows + MT - 1) / MT;
         const int ntn = (P.n_per_expert + BN - 1) / BN;
-        const int mt = id % mtiles, rest = id / mtiles;
+        // Dense up: row tiles fastest, so the CTAs running at one time share an expert's weight tile.  Dense down: column
+        // ranges fastest, so they share a few row tiles of A (every expert's hidden activations, far larger than L2,
+        // which would otherwise stream from DRAM once per column range) and all of the weights.
+        const bool n_first = P.mode == GEMM_DENSE_DOWN;
+        const int mt = n_first ? id / ntn : id % mtiles, rest = n_first ? id % ntn : id / mtiles;
         t.row0 = mt * MT + half * BM;
         t.rows_valid = min(BM, P.rows - t.row0);
         t.row_safe = 0;

@@ -1,11 +1,16 @@
-"""Phase timeline of the decode kernel (a developer's diagnostic).
+"""Where the kernels' time goes (a developer's diagnostic).
 
     python -m paper_2404_05567_b200.trace [--T 1] [--d 2048] [--H 1024] [--E 32] [--eps 0.03] [--reps 20]
+    python -m paper_2404_05567_b200.trace --gemm prefill|dense [--fuse 0|1|2] [--pairs 0|1]
 
-Builds the library once more with -DDSMOE_TRACE into ``libdsmoe_trace.so`` (the kernels then record
-``globaltimer`` stamps of their milestones per CTA), runs one decode-shaped layer a few times on random
-inputs, and prints, per milestone, the median / minimum / maximum over the CTAs of the time since the
-first CTA started, in microseconds.  Nothing here is part of the product path.
+Builds the library once more with -DDSMOE_TRACE into ``libdsmoe_trace.so``.  Without ``--gemm``: the decode kernel
+records ``globaltimer`` stamps of its milestones per CTA; one decode-shaped layer runs a few times on random inputs and
+the tool prints, per milestone, the median / minimum / maximum over the CTAs of the time since the first CTA
+started, in microseconds.  With ``--gemm``: the roles of the tensor-core GEMM kernel (MMA issuer, TMA producer, first
+epilogue warp) count the clock cycles they spend waiting; a prefill-shaped (T=8192, d=3072, H=1536, top-K 12) or
+dense-forward-shaped (T=16384, d=2048, H=1024, all 32 experts) layer runs a few times and the tool prints, per launch
+of the layer, the median share of each role's time spent in each wait.  ``--pairs`` forces the kernel's form (single
+CTAs / CTA pairs) instead of the library's own choice.  Nothing here is part of the product path.
 """
 from __future__ import annotations
 
@@ -42,6 +47,46 @@ def build_trace_lib() -> str:
     return out
 
 
+def gemm_waits(a):
+    if a.pairs is not None:
+        os.environ["DSMOE_GEMM_PAIR"] = str(a.pairs)
+    dm = binding
+    torch.manual_seed(0)
+    if a.gemm == "dense":
+        T, d, H, E = 16384, 2048, 1024, 32
+        desc = dm.make_desc(T, d, H, E, dm.BF16, dm.SELECT_ALL)
+    else:
+        T, d, H, E = 8192, 3072, 1536, 32
+        desc = dm.make_desc(T, d, H, E, dm.BF16, dm.SELECT_TOPK, K=12, fuse_combine=a.fuse)
+    x = torch.randn(T, d, device="cuda").bfloat16()
+    Wr = torch.randn(d, E, device="cuda") * 0.02
+    W1 = (torch.randn(E, d, H, device="cuda") * 0.02).bfloat16()
+    W2 = (torch.randn(E, H, d, device="cuda") * 0.02).bfloat16()
+    pk = torch.empty(dm.dsmoe_packed_size(desc), dtype=torch.uint8, device="cuda")
+    dm.dsmoe_pack_weights(desc, W1, W2, pk)
+    ws = torch.empty(dm.dsmoe_workspace_size_packed(desc), dtype=torch.uint8, device="cuda")
+    out = torch.empty(T, d, dtype=torch.bfloat16, device="cuda")
+    counts = torch.zeros(64, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for _ in range(a.reps):
+        dm.dsmoe_layer_forward(desc, x, Wr, None, None, None, pk, out, None, counts, ws, status)
+    torch.cuda.synchronize()
+    buf = (ctypes.c_longlong * (3 * 192 * 8))()
+    if dm.lib().dsmoe_gemm_trace_read(buf) != 0:
+        raise RuntimeError("dsmoe_gemm_trace_read failed")
+    g = np.array(buf[:], dtype=np.float64).reshape(3, 192, 8)
+    print(f"{a.gemm}: T={T} d={d} H={H} E={E}, pairs {'library' if a.pairs is None else a.pairs}, device status {int(status.item())}")
+    print("-- umma_gemm_kernel, last launch of each kind; medians over the CTAs that hold the role")
+    for k, name in enumerate(("router logits", "up-projection", "down-projection")):
+        mm, pr, ep = g[k][g[k][:, 0] > 0], g[k][g[k][:, 3] > 0], g[k][g[k][:, 5] > 0]
+        if not len(mm):
+            continue
+        print(f"{name:16s} MMA issuers {len(mm):3d}: {np.median(mm[:, 0]):9.0f} clk in all, {np.median(mm[:, 7]):4.0f} tiles; "
+              f"waiting for operands {100 * np.median(mm[:, 1] / mm[:, 0]):5.1f} %, for a free accumulator {100 * np.median(mm[:, 2] / mm[:, 0]):5.1f} %"
+              f" | producers {len(pr):3d}: waiting for a free slot {100 * np.median(pr[:, 4] / pr[:, 3]):5.1f} %"
+              f" | epilogue warps: waiting for an accumulator {100 * np.median(ep[:, 6] / ep[:, 5]):5.1f} %")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--T", type=int, default=1)
@@ -51,9 +96,15 @@ def main():
     ap.add_argument("--eps", type=float, default=0.03)
     ap.add_argument("--topk", type=int, default=0, help="select exactly this many experts per token instead of the threshold")
     ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--gemm", choices=["prefill", "dense"], default=None, help="wait-time shares of the GEMM kernel's roles instead")
+    ap.add_argument("--fuse", type=int, default=0, help="--gemm prefill: the layer's fuse_combine (0 library's choice, 1 inside, 2 separate)")
+    ap.add_argument("--pairs", type=int, default=None, help="--gemm: 0 single CTAs, 1 CTA pairs wherever the shapes allow")
     a = ap.parse_args()
     binding.LIB_PATH = build_trace_lib()
     binding._lib = None
+    if a.gemm:
+        a.reps = min(a.reps, 5)
+        return gemm_waits(a)
     dm = binding
     torch.manual_seed(0)
     desc = (dm.make_desc(a.T, a.d, a.H, a.E, dm.BF16, dm.SELECT_TOPK, K=a.topk) if a.topk
