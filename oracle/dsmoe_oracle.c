@@ -17,6 +17,8 @@
  *              whose gradients are Eq. 3   ("Dense Training" paragraph)
  *   training   the gradients of Eq. 2 and Eq. 3 for a given output gradient, and
  *              the mutual-information loss of the router (Eq. 4-6)
+ *   attention  the mixture-of-attention-heads layer: per-expert query heads and
+ *              output projections over shared keys and values       (Eq. 7-8)
  *
  * Readings where the paper is silent (each also listed in the design notes):
  * router h is linear (x.Wr + b); GeLU is the exact erf form; expert MLPs carry
@@ -335,6 +337,80 @@ void oracle_dense_backward(const void *x, const void *W1, const void *W2, int dt
         }
         free(hbuf);
         free(y);
+    }
+}
+
+/*
+ * Mixture-of-attention-heads layer ("Mixture of Attention Head" paragraph, Eq. 7-8), for a list of tokens.
+ * Expert i owns n_head query heads and their output projections; keys and values are shared by all experts:
+ * head j of every expert attends to key/value head j.  For token t (the n-th token of its sequence has cache
+ * position pos[t]: it sees keys 0..pos[t] of its sequence's cache):
+ *
+ *   Q_ij   = x_t . Wq[i][:, j*dh : (j+1)*dh]                                   (Eq. 7, first half)
+ *   a_ij   = softmax_l( scale * <Q_ij, K[seq][j][l]> , l = 0..pos[t] ) . V[seq][j][0..pos[t]]
+ *   O_t    = sum_{i in mask[t], ascending} scores[t,i] * sum_j a_ij . Wo[i][j*dh : (j+1)*dh, :]   (Eq. 8)
+ *
+ * Readings: Eq. 7 prints no scale under the softmax; it is an argument here (the usual 1/sqrt(dh), or 1).  The
+ * projections carry no biases.  Nothing is rounded between the steps.
+ * Layouts: Wq[E][d][n_head*dh], Wo[E][n_head*dh][d], Kc and Vc [n_seq][n_head][L][dh], all of the layer's type;
+ * tok_seq[t] (NULL: all 0) and pos[t] are int32.  out is double [n_tokens, d].
+ */
+void oracle_moa_layer(const void *x, const void *Wq, const void *Wo, const void *Kc, const void *Vc, int dtype,
+                      const float *scores, const uint64_t *mask, const int32_t *tok_seq, const int32_t *pos,
+                      const int64_t *token_ids, int64_t n_tokens, int64_t d, int64_t n_head, int64_t dh, int64_t E,
+                      int64_t L, double scale, double *out) {
+    const int64_t H = n_head * dh;
+#pragma omp parallel
+    {
+        double *q = (double *)malloc(sizeof(double) * (size_t)dh);
+        double *a = (double *)malloc(sizeof(double) * (size_t)dh);
+        double *w = (double *)malloc(sizeof(double) * (size_t)(L > 0 ? L : 1));
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t i = 0; i < n_tokens; ++i) {
+            const int64_t t = token_ids ? token_ids[i] : i;
+            const int64_t sq = tok_seq ? tok_seq[t] : 0;
+            const int64_t last = pos[t];
+            double *o = out + i * d;
+            for (int64_t c = 0; c < d; ++c) o[c] = 0.0;
+            for (int64_t e = 0; e < E; ++e) {
+                if (!((mask[t] >> e) & 1)) continue;
+                const double s = (double)scores[t * E + e];
+                for (int64_t j = 0; j < n_head; ++j) {
+                    for (int64_t c = 0; c < dh; ++c) q[c] = 0.0;
+                    for (int64_t k = 0; k < d; ++k) {
+                        const double xv = load_val(x, dtype, (size_t)(t * d + k));
+                        const size_t wrow = (size_t)((e * d + k) * H + j * dh);
+                        for (int64_t c = 0; c < dh; ++c) q[c] += xv * load_val(Wq, dtype, wrow + (size_t)c);
+                    }
+                    const size_t kv0 = (size_t)(((sq * n_head + j) * L) * dh);
+                    double mx = -INFINITY;
+                    for (int64_t l = 0; l <= last; ++l) {
+                        double dot = 0.0;
+                        for (int64_t c = 0; c < dh; ++c) dot += q[c] * load_val(Kc, dtype, kv0 + (size_t)(l * dh + c));
+                        w[l] = scale * dot;
+                        mx = w[l] > mx ? w[l] : mx;
+                    }
+                    double den = 0.0;
+                    for (int64_t l = 0; l <= last; ++l) {
+                        w[l] = exp(w[l] - mx);
+                        den += w[l];
+                    }
+                    for (int64_t c = 0; c < dh; ++c) a[c] = 0.0;
+                    for (int64_t l = 0; l <= last; ++l) {
+                        const double p = w[l] / den;
+                        for (int64_t c = 0; c < dh; ++c) a[c] += p * load_val(Vc, dtype, kv0 + (size_t)(l * dh + c));
+                    }
+                    for (int64_t r = 0; r < dh; ++r) {
+                        const double ar = s * a[r];
+                        const size_t orow = (size_t)((e * H + j * dh + r) * d);
+                        for (int64_t c = 0; c < d; ++c) o[c] += ar * load_val(Wo, dtype, orow + (size_t)c);
+                    }
+                }
+            }
+        }
+        free(q);
+        free(a);
+        free(w);
     }
 }
 

@@ -21,7 +21,7 @@ _lib = None
 MODE_THRESHOLD, MODE_TOPK, MODE_ALL, MODE_THRESHOLD_TOPK = 0, 1, 2, 3
 
 __all__ = [
-    "build", "router_scores", "select", "group", "layer", "expert_rows", "combine", "mi_loss", "dense_backward",
+    "build", "router_scores", "select", "group", "layer", "expert_rows", "combine", "mi_loss", "dense_backward", "moa_layer",
     "num_threads", "MODE_THRESHOLD", "MODE_TOPK", "MODE_ALL", "MODE_THRESHOLD_TOPK",
 ]
 
@@ -131,6 +131,33 @@ def layer(x, W1, W2, scores, mask, token_ids=None) -> np.ndarray:
     out = np.empty((n, d), dtype=np.float64)
     _load().oracle_layer(_p(x), _p(W1), _p(W2), dt, _p(S), _p(mask), _p(ids), ctypes.c_int64(n),
                          ctypes.c_int64(d), ctypes.c_int64(H), ctypes.c_int64(E), _p(out))
+    return out
+
+
+def moa_layer(x, Wq, Wo, Kc, Vc, scores, mask, pos, n_head, scale, tok_seq=None, token_ids=None) -> np.ndarray:
+    """Mixture-of-attention-heads layer (Eq. 7-8), float64:
+    O[t] = sum_{i selected} S[t,i] sum_j softmax(scale Q_ij K_j^T) V_j Wo_ij over keys 0..pos[t] of the token's sequence.
+
+    Wq [E, d, n_head*dh], Wo [E, n_head*dh, d], Kc and Vc [n_seq, n_head, L, dh]."""
+    x, Wq, Wo, Kc, Vc = _c(x), _c(Wq), _c(Wo), _c(Kc), _c(Vc)
+    S = _c(scores, np.float32)
+    mask = _c(mask, np.uint64)
+    pos = _c(pos, np.int32)
+    T, d = x.shape
+    E, d1, H = Wq.shape
+    n_seq, nh, L, dh = Kc.shape
+    assert d1 == d and Wo.shape == (E, H, d) and S.shape == (T, E) and nh == n_head and H == n_head * dh
+    assert Vc.shape == Kc.shape and pos.shape == (T,) and pos.min(initial=0) >= 0 and pos.max(initial=0) < L
+    dt = _dtype_code(x)
+    assert all(_dtype_code(a) == dt for a in (Wq, Wo, Kc, Vc))
+    seq = None if tok_seq is None else _c(tok_seq, np.int32)
+    assert seq is None or (seq.shape == (T,) and seq.min(initial=0) >= 0 and seq.max(initial=0) < n_seq)
+    ids = None if token_ids is None else _c(token_ids, np.int64)
+    n = T if ids is None else ids.shape[0]
+    out = np.empty((n, d), dtype=np.float64)
+    _load().oracle_moa_layer(_p(x), _p(Wq), _p(Wo), _p(Kc), _p(Vc), dt, _p(S), _p(mask), _p(seq), _p(pos), _p(ids),
+                             ctypes.c_int64(n), ctypes.c_int64(d), ctypes.c_int64(n_head), ctypes.c_int64(dh),
+                             ctypes.c_int64(E), ctypes.c_int64(L), ctypes.c_double(scale), _p(out))
     return out
 
 
