@@ -287,6 +287,39 @@ dsmoe_status dsmoe_dense_backward(const dsmoe_layer_desc* desc, const void* x, c
                                   dsmoe_stream stream);
 
 /*
+ * The mixture-of-attention-heads layer ("Mixture of Attention Head" paragraph, Eq. 7-8): the model's other MoE
+ * block.  Expert i owns n_head query heads and their output projections; keys and values are shared by all experts,
+ * head j of every expert attending to key/value head j.  For token t, which sees keys 0..pos[t] of its sequence's cache:
+ *
+ *   Q_ij = x_t . Wq[i][:, j*dh:(j+1)*dh]              a_ij = softmax_l(scale <Q_ij, K[seq][j][l]>) . V[seq][j]
+ *   O_t  = sum over the selected experts i (ascending) of S[t,i] * sum_j a_ij . Wo[i][j*dh:(j+1)*dh, :]
+ *
+ * It is the feed-forward layer's pipeline with attention in place of GeLU: desc describes it with E = the number of
+ * attention experts and H = n_head * d_head; router, selection (desc->mode ...), grouping and the router-weighted sum
+ * are those of dsmoe_layer_forward.  Eq. 7 prints no scale under the softmax: `scale` is the caller's (1/sqrt(d_head)
+ * in the usual form).  No biases.  Queries and attention outputs are rounded to bf16 between the steps.
+ *
+ * args (host struct, read during the call): Kc, Vc  device, bf16 [n_seq][n_head][L][d_head]; tok_seq  device int32 [T],
+ * the sequence of each token, or NULL (all 0); pos  device int32 [T], 0 <= pos[t] < L.
+ * packed   device: dsmoe_pack_weights(desc, Wq, Wo, packed) with Wq [E][d][H], Wo [E][H][d].
+ * x, Wr, br, out, mask_out, counts_out, workspace (dsmoe_workspace_size_packed(desc) bytes), dev_status: as for
+ * dsmoe_layer_forward.  Supported: bf16, d and H multiples of 64, d_head a multiple of 32 up to 256, L up to
+ * 12000; DSMOE_ERR_UNSUPPORTED otherwise.  A tok_seq or pos entry out of range is clamped and reported as
+ * DSMOE_ERR_INVALID_ARG in *dev_status.
+ */
+typedef struct dsmoe_moa_args {
+    int32_t n_head, n_seq, L;
+    float scale;
+    const void* Kc;
+    const void* Vc;
+    const int32_t* tok_seq;
+    const int32_t* pos;
+} dsmoe_moa_args;
+dsmoe_status dsmoe_moa_forward(const dsmoe_layer_desc* desc, const dsmoe_moa_args* args, const void* x, const float* Wr,
+                               const float* br, const void* packed, void* out, uint64_t* mask_out, int32_t* counts_out,
+                               void* workspace, size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream);
+
+/*
  * Measurement aid (no counterpart in the paper): a ring of CUDA event pairs on the caller's stream.
  * After dsmoe_timing_enable(n_pairs) (n_pairs > 0; events are created here, so call it outside any
  * timed region), every launch of an expert-MLP tensor-core kernel (the two grouped or dense GEMMs of

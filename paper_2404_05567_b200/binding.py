@@ -24,7 +24,7 @@ EXPORTS = (
     "dsmoe_expert_mlp", "dsmoe_combine", "dsmoe_packed_size", "dsmoe_pack_weights",
     "dsmoe_layer_forward", "dsmoe_layer_forward_host", "dsmoe_timing_enable", "dsmoe_timing_read",
     "dsmoe_select_static", "dsmoe_workspace_size_packed", "dsmoe_workspace_size_stages", "dsmoe_stats",
-    "dsmoe_mi_loss", "dsmoe_dense_backward",
+    "dsmoe_mi_loss", "dsmoe_dense_backward", "dsmoe_moa_forward",
 )
 
 
@@ -33,6 +33,11 @@ class LayerDesc(ctypes.Structure):
                 ("dtype", ctypes.c_int32), ("mode", ctypes.c_int32), ("eps", ctypes.c_float),
                 ("eps_normalized", ctypes.c_int32), ("K", ctypes.c_int32), ("min_k", ctypes.c_int32),
                 ("out_fp32", ctypes.c_int32), ("fuse_combine", ctypes.c_int32)]
+
+
+class MoaArgs(ctypes.Structure):
+    _fields_ = [("n_head", ctypes.c_int32), ("n_seq", ctypes.c_int32), ("L", ctypes.c_int32), ("scale", ctypes.c_float),
+                ("Kc", ctypes.c_void_p), ("Vc", ctypes.c_void_p), ("tok_seq", ctypes.c_void_p), ("pos", ctypes.c_void_p)]
 
 
 class DsmoeError(RuntimeError):
@@ -203,6 +208,18 @@ def dsmoe_dense_backward(desc, x, W1, W2, packed, scores, mask, dO, dS, dA, work
                                       _ptr(mask), _ptr(dO), _ptr(dS), _ptr(dA), _ptr(workspace),
                                       ctypes.c_size_t(workspace.numel() if workspace is not None else 0),
                                       _ptr(dev_status), _stream(stream)), "dsmoe_dense_backward")
+
+
+def dsmoe_moa_forward(desc, n_head, scale, Kc, Vc, tok_seq, pos, x, Wr, br, packed, out, mask_out, counts_out, workspace,
+                      dev_status=None, stream=None):
+    """Mixture-of-attention-heads layer (Eq. 7-8).  Kc, Vc: [n_seq, n_head, L, d_head] bf16 tensors."""
+    n_seq, nh, L, _ = Kc.shape
+    assert nh == n_head and Vc.shape == Kc.shape
+    args = MoaArgs(int(n_head), int(n_seq), int(L), float(scale), _ptr(Kc), _ptr(Vc), _ptr(tok_seq), _ptr(pos))
+    _check(lib().dsmoe_moa_forward(ctypes.byref(desc), ctypes.byref(args), _ptr(x), _ptr(Wr), _ptr(br), _ptr(packed),
+                                   _ptr(out), _ptr(mask_out), _ptr(counts_out), _ptr(workspace),
+                                   ctypes.c_size_t(workspace.numel() if workspace is not None else 0),
+                                   _ptr(dev_status), _stream(stream)), "dsmoe_moa_forward")
 
 
 def dsmoe_timing_enable(n_pairs: int):

@@ -338,6 +338,54 @@ dsmoe_status dsmoe_dense_backward(const dsmoe_layer_desc* desc, const void* x, c
     return launch_dense_backward_plain(*desc, x, W1, W2, scores, mask, dO, dS, dA, s);
 }
 
+dsmoe_status dsmoe_moa_forward(const dsmoe_layer_desc* desc, const dsmoe_moa_args* args, const void* x, const float* Wr,
+                               const float* br, const void* packed, void* out, uint64_t* mask_out, int32_t* counts_out,
+                               void* workspace, size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream) {
+    DSMOE_TRY(check_desc(desc));
+    const dsmoe_layer_desc& p = *desc;
+    if (p.T == 0) return DSMOE_OK;
+    if (!args || !x || !Wr || !out || !packed || !args->Kc || !args->Vc || !args->pos) return DSMOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(Wr) || !aligned16(out) || !aligned16(packed) || !aligned16(args->Kc) || !aligned16(args->Vc))
+        return DSMOE_ERR_INVALID_ARG;
+    if (args->n_seq <= 0 || args->L <= 0) return DSMOE_ERR_INVALID_ARG;
+    if (p.dtype != DSMOE_BF16 || !moa_supported(p, args->n_head, args->L)) return DSMOE_ERR_UNSUPPORTED;
+    const WsLayout L = ws_layout(p);
+    if (!workspace || ws_bytes < L.total_packed || !aligned16(workspace)) return DSMOE_ERR_WORKSPACE;
+    char* ws = static_cast<char*>(workspace);
+    cudaStream_t s = (cudaStream_t)stream;
+    float* scores = reinterpret_cast<float*>(ws + L.scores);
+    uint64_t* mask = mask_out ? mask_out : reinterpret_cast<uint64_t*>(ws + L.mask);
+    int32_t* k_t = reinterpret_cast<int32_t*>(ws + L.k_t);
+    int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+    int32_t* offsets = reinterpret_cast<int32_t*>(ws + L.offsets);
+    int32_t* chunk_prefix = reinterpret_cast<int32_t*>(ws + L.chunk_prefix);
+    int32_t* row_token = reinterpret_cast<int32_t*>(ws + L.row_token);
+    float* row_gate = reinterpret_cast<float*>(ws + L.row_gate);
+    int32_t* token_rows = reinterpret_cast<int32_t*>(ws + L.token_rows);
+    const MoaCore core{args->n_head, args->n_seq, args->L, args->scale, args->Kc, args->Vc, args->tok_seq, args->pos};
+
+    // router, selection and grouping as in dsmoe_layer_forward's grouped path (also when every expert is selected)
+    dsmoe_layer_desc pr = p;
+    if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK) pr.mode = DSMOE_SELECT_THRESHOLD;
+    if (router_umma_supported(p))
+        DSMOE_TRY(launch_router_umma(pr, x, Wr, br, scores, mask, k_t, ws + L.router, dev_status, s));
+    else
+        DSMOE_TRY(launch_router(pr, x, Wr, br, scores, mask, k_t, s));
+    if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK)
+        DSMOE_TRY(launch_select(p, scores, mask, k_t, s, reinterpret_cast<int*>(ws + L.batch_k)));
+    DSMOE_TRY(launch_finalize(p, mask, counts, offsets, chunk_prefix, counts_out, s));
+    if (fuses_combine(p)) {
+        DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, nullptr, s, out));
+        const CombineArgs cmb{row_token, row_gate, mask, reinterpret_cast<float*>(ws + L.acc),
+                              reinterpret_cast<int*>(ws + L.tile_done), out};
+        return launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, nullptr, dev_status, s, x, row_token, &cmb, &core);
+    }
+    DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, nullptr, s));
+    const CombineArgs gated{row_token, row_gate, nullptr, nullptr, nullptr, nullptr};
+    DSMOE_TRY(launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, ws + L.acc, dev_status, s, x, row_token, &gated, &core));
+    return launch_combine(p, ws + L.acc, nullptr, token_rows, k_t, out, s, true);
+}
+
 dsmoe_status dsmoe_timing_enable(int n_pairs) {
     if (n_pairs < 0 || n_pairs > (1 << 20)) return DSMOE_ERR_INVALID_ARG;
     return timing_enable(n_pairs);

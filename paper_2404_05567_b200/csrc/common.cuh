@@ -129,9 +129,26 @@ struct CombineArgs {
     int* tile_done;      // E * ceil(d / 256) ints
     void* out;
 };
+// With moa, the layer is the mixture of attention heads (Eq. 7-8): the up-projection is the experts' query projection
+// (no activation) and every grouped row attends to its sequence's keys and values before the down-projection.
+struct MoaCore {
+    int n_head, n_seq, L;
+    float scale;
+    const void* Kc;
+    const void* Vc;          // [n_seq][n_head][L][d_head]
+    const int32_t* tok_seq;  // [T] or NULL (one sequence)
+    const int32_t* pos;      // [T]: token t sees keys 0..pos[t]
+};
 dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,
                              void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s, const void* x = nullptr,
-                             const int32_t* row_token = nullptr, const CombineArgs* cmb = nullptr);
+                             const int32_t* row_token = nullptr, const CombineArgs* cmb = nullptr,
+                             const MoaCore* moa = nullptr);
+
+// ---- moa.cu : the attention step of the mixture-of-attention-heads layer
+bool moa_supported(const dsmoe_layer_desc& p, int n_head, int L);
+// qa [Amax, H] bf16: the grouped rows' queries on entry, their attention outputs on return
+dsmoe_status launch_moa_attention(const dsmoe_layer_desc& p, const MoaCore& c, void* qa, const int32_t* row_token,
+                                  const int32_t* offsets, int32_t* dev_status, cudaStream_t s);
 // Whole-layer paths that need no grouping (all experts selected, or few tokens).  *done = false
 // means "not taken": the caller continues with the grouped path.
 // Whole layer for few tokens (T <= 128) in one cooperative launch, router included.

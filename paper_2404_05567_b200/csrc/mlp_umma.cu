@@ -1948,7 +1948,7 @@ bool umma_supported(const dsmoe_layer_desc& p) {
 
 dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,
                              void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s, const void* x,
-                             const int32_t* row_token, const CombineArgs* cmb) {
+                             const int32_t* row_token, const CombineArgs* cmb, const MoaCore* moa) {
     if (p.T == 0) return DSMOE_OK;
     if (!umma_supported(p)) return DSMOE_ERR_UNSUPPORTED;
     const size_t amax = amax_of(p);
@@ -1968,6 +1968,7 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
     up.gather = row_token;
     up.gather_src = x;
     up.gather_rows = p.T;
+    if (moa) up.epi = EPI_STORE;      // query projection: no activation (Eq. 7)
     GemmParams down{};
     down.mode = GEMM_GROUPED; down.epi = EPI_STORE; down.E = p.E; down.n_per_expert = p.d; down.k_per_expert = p.H;
     down.rows = (int)amax; down.offsets = offsets; down.out = yp; down.ld_out = p.d; down.dev_status = dev_status;
@@ -1991,7 +1992,8 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
     // top-K selection alone (an upper bound otherwise), so only there may the launches pair on their own
     const long long known = p.mode == DSMOE_SELECT_TOPK ? (long long)p.T * (p.K < p.E ? p.K : p.E) : 0;
     const int pair_tiles = known >= 1024ll * p.E ? INT_MAX : (pair_override() == 1 ? INT_MAX : 0);
-    DSMOE_TRY(launch_gemm(*mA1, *mB1, up, sm_count(), s, true, pair_tiles));
+    DSMOE_TRY(launch_gemm(*mA1, *mB1, up, sm_count(), s, true, moa ? 0 : pair_tiles));
+    if (moa) DSMOE_TRY(launch_moa_attention(p, *moa, hbuf, row_token, offsets, dev_status, s));
     DSMOE_TRY(launch_gemm(*mA2, *mB2, down, sm_count(), s, true, pair_tiles));
     return DSMOE_OK;
 }
