@@ -472,6 +472,99 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
     return res
 
 
+# Mixture-of-attention-heads layer (Eq. 7-8) at DS-MoE-6B's attention shape (Table tab:model_arch: 8 experts of 4 heads
+# of 128, model width 4096; 5 of 8 experts per token, the > 60 % layer utilisation the paper reports for attention):
+# prefill = 32 sequences of 256 tokens (the sequence length of the paper's input-throughput setting), decode = one new
+# token for each of 32 sequences with 2048 cached positions (its latency setting's context).
+MOA_WORKLOADS = {
+    "moa6b_prefill": dict(T=8192, d=4096, E=8, n_head=4, dh=128, K=5, n_seq=32, L=256, layout="prefill"),
+    "moa6b_decode": dict(T=32, d=4096, E=8, n_head=4, dh=128, K=5, n_seq=32, L=2048, layout="decode"),
+}
+
+
+def run_moa(name: str, steps: int, warmup: int, sampler_index=0):
+    import torch
+    import paper_2404_05567_b200 as dm
+
+    def to_dev(a):
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+        return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+    w = MOA_WORKLOADS[name]
+    T, d, E, nh, dh, L, n_seq = w["T"], w["d"], w["E"], w["n_head"], w["dh"], w["L"], w["n_seq"]
+    H = nh * dh
+    s = gi.LayerSpec(name, T=T, d=d, H=H, E=E, dtype="bf16", mode=gi.MODE_TOPK, K=w["K"], router_gain=4.0)
+    desc = dm.make_desc(T, d, H, E, dm.BF16, s.mode, 0.0, 0, s.K, 0, 0, 0)
+    P = peaks()
+    Wr, br = gi.router(s)
+    Wq, Wo = gi.experts(s)
+    packed = torch.empty(dm.dsmoe_packed_size(desc), dtype=torch.uint8, device="cuda")
+    dm.dsmoe_pack_weights(desc, to_dev(Wq), to_dev(Wo), packed)
+    # the key/value cache is drawn on the device (values of the same distribution as the generator's; no parity is
+    # taken from this run): 32 x 4 x 2048 x 128 x 2 tensors would take the host generator a while
+    g = torch.Generator(device="cuda").manual_seed(0)
+    Kc = torch.randn((n_seq, nh, L, dh), generator=g, device="cuda").bfloat16()
+    Vc = torch.randn((n_seq, nh, L, dh), generator=g, device="cuda").bfloat16()
+    if w["layout"] == "prefill":
+        per = T // n_seq
+        seq = (np.arange(T) // per).astype(np.int32)
+        pos = (np.arange(T) % per).astype(np.int32)
+    else:
+        seq = np.arange(T, dtype=np.int32)
+        pos = np.full(T, L - 1, dtype=np.int32)
+    seq_d, pos_d = to_dev(seq), to_dev(pos)
+    x_d, Wr_d, br_d = to_dev(gi.tokens(s)), to_dev(Wr), to_dev(br) if br is not None else None
+    ws = torch.empty(dm.dsmoe_workspace_size_packed(desc), dtype=torch.uint8, device="cuda")
+    out = torch.empty((T, d), dtype=torch.bfloat16, device="cuda")
+    counts = torch.zeros(64, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    scale = 1.0 / float(np.sqrt(dh))
+
+    def step(want=False):
+        dm.dsmoe_moa_forward(desc, nh, scale, Kc, Vc, seq_d, pos_d, x_d, Wr_d, br_d, packed, out, None,
+                             counts if want else None, ws, status)
+
+    step(True)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    A = int(counts[:E].sum().item())
+    for _ in range(max(warmup, 3)):
+        step()
+    dm.dsmoe_timing_enable(3 * steps)
+    sampler = ClockSampler(sampler_index)
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    clocks = sampler.finish()
+    durs = np.array(dm.dsmoe_timing_read(3 * steps)).reshape(steps, 3).mean(axis=0)       # query projection, attention, output projection
+    dm.dsmoe_timing_enable(0)
+    assert int(status.item()) == 0
+    proj_flops = 4.0 * A * d * H
+    att_flops = 4.0 * w["K"] * nh * dh * float((pos.astype(np.float64) + 1).sum())
+    kv_bytes = 2.0 * n_seq * nh * L * dh * 2 if w["layout"] == "decode" else 0.0
+    weight_bytes = 2.0 * E * d * H * 2.0
+    ach = proj_flops / ((durs[0] + durs[2]) * 1e-3) / 1e12
+    t_flop, t_byte = (proj_flops + att_flops) / (P["tf_burst"] * 1e12), (weight_bytes + kv_bytes) / (P["hbm"] * 1e9)
+    roof = dict(bound="tensor" if t_flop >= t_byte else "hbm", kernel="umma_gemm_kernel (projections), moa_attention_kernel",
+                achieved=ach, peak=P["tf_burst"], unit="TFLOP/s", peak_source=P["source"] + " (burst bf16; projections only)",
+                frac=ach / P["tf_burst"], frac_burst=ach / P["tf_burst"], frac_sustained=ach / P["tf_sustained"],
+                frac_nominal=ach / NOMINAL["tf"], roofline_ms=max(t_flop, t_byte) * 1e3,
+                frac_of_roofline_time=max(t_flop, t_byte) / (float(durs.sum()) * 1e-3),
+                step_frac_of_roofline_time=max(t_flop, t_byte) / (ms * 1e-3), step_frac=proj_flops / (ms * 1e-3) / 1e12 / P["tf_burst"],
+                algorithmic_per_launch=proj_flops / 2, attention_flops=att_flops, kv_bytes=kv_bytes, traffic=None,
+                kernel_ms_per_step=float(durs.sum()), ms_per_step_with_events=ms, launch_ms_each=[float(v) for v in durs],
+                launches_per_step=3)
+    return dict(workload=name, value=T / (ms * 1e-3), unit="tokens/s", ms_per_step=ms, steps=steps, roofline=roof, clocks=clocks,
+                assignments=A, active_experts=E, config=dict(w))
+
+
 def workload_config(name, s):
     mode = {0: "threshold", 1: "topk", 2: "all", 3: "threshold_topk"}[s.mode]
     return {"workload": name, "T": s.T, "d": s.d, "E": s.E, "H": s.H, "select": mode, "eps": s.eps, "K": s.K,
@@ -527,7 +620,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2_t32", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="c2_t32", choices=sorted(WORKLOADS) + sorted(MOA_WORKLOADS))
     ap.add_argument("--no-extra", action="store_true")
     ap.add_argument("--graph", action="store_true", help="replay each step as one CUDA graph")
     ap.add_argument("--fuse-combine", type=int, default=None, choices=[0, 1, 2],
@@ -544,6 +637,17 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if name in MOA_WORKLOADS:
+        # the attention layer alone (one GPU; a diagnostic line: the default line is the feed-forward layer's)
+        import torch
+        torch.cuda.set_device(0)
+        from paper_2404_05567_b200 import build as lib_build
+        lib_build.build()
+        gi.build()
+        r = run_moa(name, steps, warmup)
+        print(json.dumps(dict(metric="moa_layer_tokens_per_s", n_gpus=1, warmup=max(warmup, 3), higher_is_better=True,
+                              dtype="bf16", data="synthetic", gpu_launches=11 * steps, **r)))
+        return
     if args.fuse_combine is not None:
         for k in WORKLOADS:
             WORKLOADS[k] = (WORKLOADS[k][0], dict(WORKLOADS[k][1], fuse_combine=args.fuse_combine))
@@ -619,6 +723,9 @@ def main():
                              "active_experts_per_layer": r["active_experts_per_layer"],
                              "activation_rms_per_layer": r["activation_rms_per_layer"],
                              "near_threshold_1e-6": r["stats"]["near_threshold"]})
+            for other, k in (("moa6b_prefill", 20), ("moa6b_decode", 200)):
+                drop_weights(torch)
+                also.append(run_moa(other, k, 5, sampler_index=physical_gpu_index(local_rank)))
             line["also"] = also
     print(json.dumps(line))
     if dist is not None:

@@ -362,7 +362,7 @@ dsmoe_status dsmoe_moa_forward(const dsmoe_layer_desc* desc, const dsmoe_moa_arg
     int32_t* row_token = reinterpret_cast<int32_t*>(ws + L.row_token);
     float* row_gate = reinterpret_cast<float*>(ws + L.row_gate);
     int32_t* token_rows = reinterpret_cast<int32_t*>(ws + L.token_rows);
-    const MoaCore core{args->n_head, args->n_seq, args->L, args->scale, args->Kc, args->Vc, args->tok_seq, args->pos};
+    const MoaCore core{args->n_head, args->n_seq, args->L, args->scale, args->Kc, args->Vc, args->tok_seq, args->pos, token_rows};
 
     // router, selection and grouping as in dsmoe_layer_forward's grouped path (also when every expert is selected)
     dsmoe_layer_desc pr = p;

@@ -138,6 +138,7 @@ struct MoaCore {
     const void* Vc;          // [n_seq][n_head][L][d_head]
     const int32_t* tok_seq;  // [T] or NULL (one sequence)
     const int32_t* pos;      // [T]: token t sees keys 0..pos[t]
+    const int32_t* token_rows;   // [T, W]: the grouped rows of each token (from the permute step)
 };
 dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const void* packed, const int32_t* offsets,
                              void* hbuf, void* yp, int32_t* dev_status, cudaStream_t s, const void* x = nullptr,
@@ -148,7 +149,7 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
 bool moa_supported(const dsmoe_layer_desc& p, int n_head, int L);
 // qa [Amax, H] bf16: the grouped rows' queries on entry, their attention outputs on return
 dsmoe_status launch_moa_attention(const dsmoe_layer_desc& p, const MoaCore& c, void* qa, const int32_t* row_token,
-                                  const int32_t* offsets, int32_t* dev_status, cudaStream_t s);
+                                  const int32_t* token_rows, const int32_t* offsets, int32_t* dev_status, cudaStream_t s);
 // Whole-layer paths that need no grouping (all experts selected, or few tokens).  *done = false
 // means "not taken": the caller continues with the grouped path.
 // Whole layer for few tokens (T <= 128) in one cooperative launch, router included.

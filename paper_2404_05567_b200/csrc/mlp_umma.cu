@@ -1993,7 +1993,7 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
     const long long known = p.mode == DSMOE_SELECT_TOPK ? (long long)p.T * (p.K < p.E ? p.K : p.E) : 0;
     const int pair_tiles = known >= 1024ll * p.E ? INT_MAX : (pair_override() == 1 ? INT_MAX : 0);
     DSMOE_TRY(launch_gemm(*mA1, *mB1, up, sm_count(), s, true, moa ? 0 : pair_tiles));
-    if (moa) DSMOE_TRY(launch_moa_attention(p, *moa, hbuf, row_token, offsets, dev_status, s));
+    if (moa) DSMOE_TRY(launch_moa_attention(p, *moa, hbuf, row_token, moa->token_rows, offsets, dev_status, s));
     DSMOE_TRY(launch_gemm(*mA2, *mB2, down, sm_count(), s, true, pair_tiles));
     return DSMOE_OK;
 }

@@ -5,7 +5,10 @@
 // with the router-weighted sum of Eq. 8; in between every grouped row -- one (token, expert) pair, n_head query
 // vectors of d_head -- attends to the keys and values of its token's sequence, head j to key/value head j
 // (the keys and values are shared by all experts).  This file holds that middle step.
+#include <cstdlib>
+
 #include "common.cuh"
+#include "tensor_maps.cuh"
 
 namespace dsmoe {
 
@@ -99,6 +102,266 @@ moa_attention_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restrict__
     for (int i = 0; i < DPL; ++i) qrow[lane + 32 * i] = __float2bfloat16_rn(acc[i] * inv);
 }
 
+// ---------------------------------------------------------------- the same step on the warp-level tensor-core path
+//
+// One CTA per (token, head, tile of up to 16 of the token's grouped rows): the rows of a token share its keys and
+// values, and 16 rows are exactly the M of an m16n8k16 MMA.  The 8 warps share out the visible keys in blocks of 32:
+// a warp copies its block of K and V into (padded, conflict-free) shared memory, forms S = Q.K^T (Q fragments stay
+// in registers for the whole kernel), updates the running row maxima and sums, rescales its accumulators and adds
+// P.V with P taken straight from S's registers -- the usual streaming-softmax order.  The warps' partial results
+// (maximum, sum, accumulator per row) are merged through shared memory at the end, in warp order.
+constexpr int kKeyBlock = 32;
+
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int DH, int kMmaWarps>      // long caches: 8 warps share out the keys; short ones: 2, and several CTAs fit an SM
+__global__ void __launch_bounds__(32 * kMmaWarps)
+moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restrict__ token_rows, int W, int row_tiles,
+                         int tpt, long long amax, int n_head, int H, int T, const __nv_bfloat16* __restrict__ Kc,
+                         const __nv_bfloat16* __restrict__ Vc, const int32_t* __restrict__ tok_seq,
+                         const int32_t* __restrict__ pos, int n_seq, int L, float scale, int* __restrict__ dev_status) {
+    constexpr int STRIDE = DH * 2 + 16;                 // bytes per key row in shared memory: 16 of padding
+    constexpr int KS = DH / 16, DT = DH / 8, CH = DH / 8;
+    extern __shared__ __align__(16) unsigned char moa_mma_smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q4 = lane & 3;
+    // The tile's 16 rows: with tpt == 1, slots 16 rt .. of token t0; with tpt > 1 (rows per token W <= 8, one row
+    // tile), all W slots of the tpt tokens t0, t0 + 1, ...: neighbouring tokens of one sequence see nearly the same
+    // keys, so their rows share the copies of K and V.
+    const int rt = blockIdx.x % row_tiles;
+    const int j = (blockIdx.x / row_tiles) % n_head;
+    const int t0 = (blockIdx.x / (row_tiles * n_head)) * tpt;
+    const auto row_token_slot = [&](int i, int& tok, int& slot) {
+        if (tpt == 1) {
+            tok = t0;
+            slot = rt * 16 + i;
+        } else {
+            tok = t0 + i / W;
+            slot = i % W;
+            if (i >= tpt * W) tok = T;
+        }
+    };
+    // this thread's two rows of the tile (g and g + 8): grouped row (-1 = none), token, last visible key
+    int r0 = -1, r1 = -1, tk0, tk1, sl0, sl1, last0 = 0, last1 = 0;
+    row_token_slot(g, tk0, sl0);
+    row_token_slot(g + 8, tk1, sl1);
+    if (tk0 < T && sl0 < W) r0 = token_rows[(size_t)tk0 * W + sl0];
+    if (tk1 < T && sl1 < W) r1 = token_rows[(size_t)tk1 * W + sl1];
+    if (r0 >= amax) r0 = -1;
+    if (r1 >= amax) r1 = -1;
+    if (__syncthreads_or(r0 >= 0 || r1 >= 0) == 0) return;          // no rows in this tile
+    bool bad = false;
+    if (r0 >= 0) {
+        last0 = pos[tk0];
+        bad = bad || last0 < 0 || last0 >= L;
+        last0 = min(max(last0, 0), L - 1);
+    }
+    if (r1 >= 0) {
+        last1 = pos[tk1];
+        bad = bad || last1 < 0 || last1 >= L;
+        last1 = min(max(last1, 0), L - 1);
+    }
+    // the tokens of the tile: one pass over the keys if they all belong to one sequence, else one pass per token
+    const int ntok = min(tpt, T - t0);
+    int seq_first = tok_seq ? tok_seq[t0] : 0;
+    bool same = true;
+    for (int u = 1; u < ntok; ++u) same = same && (tok_seq ? tok_seq[t0 + u] : 0) == seq_first;
+    const int npass = same ? 1 : ntok;
+    // Q fragments (the A operand of S = Q.K^T)
+    uint32_t qf[KS][4];
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+        const int c = j * DH + ks * 16 + q4 * 2;
+        qf[ks][0] = r0 >= 0 ? *reinterpret_cast<const uint32_t*>(qa + (size_t)r0 * H + c) : 0u;
+        qf[ks][1] = r1 >= 0 ? *reinterpret_cast<const uint32_t*>(qa + (size_t)r1 * H + c) : 0u;
+        qf[ks][2] = r0 >= 0 ? *reinterpret_cast<const uint32_t*>(qa + (size_t)r0 * H + c + 8) : 0u;
+        qf[ks][3] = r1 >= 0 ? *reinterpret_cast<const uint32_t*>(qa + (size_t)r1 * H + c + 8) : 0u;
+    }
+    unsigned char* Ks = moa_mma_smem + (size_t)warp * 2 * kKeyBlock * STRIDE;
+    unsigned char* Vs = Ks + kKeyBlock * STRIDE;
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    float o[DT][4];
+#pragma unroll
+    for (int i = 0; i < DT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    for (int ps = 0; ps < npass; ++ps) {
+    // this pass: the sequence whose keys are walked, the rows that take part, the last key any of them sees
+    int sq = same ? seq_first : (tok_seq ? tok_seq[t0 + ps] : 0);
+    bad = bad || sq < 0 || sq >= n_seq;
+    sq = min(max(sq, 0), n_seq - 1);
+    const bool act0 = r0 >= 0 && (same || tk0 == t0 + ps), act1 = r1 >= 0 && (same || tk1 == t0 + ps);
+    int last = 0;
+    for (int u = same ? 0 : ps; u < (same ? ntok : ps + 1); ++u) last = max(last, min(max(pos[t0 + u], 0), L - 1));
+    const __nv_bfloat16* Kh = Kc + ((size_t)(sq * n_head + j) * L) * DH;
+    const __nv_bfloat16* Vh = Vc + ((size_t)(sq * n_head + j) * L) * DH;
+    const int nblocks = last / kKeyBlock + 1;
+    for (int b = warp; b < nblocks; b += kMmaWarps) {
+        const int key0 = b * kKeyBlock, nk = min(kKeyBlock, last + 1 - key0);
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {                  // 32 rows x CH 16-byte pieces, a piece per lane and step
+            const int idx = lane + 32 * i, row = idx / CH, ch = idx % CH;
+            // asynchronous 16-byte copies, all in flight at once; rows past the last visible key are filled with zeros
+            const int rr = row < nk ? row : 0;
+            const uint32_t nbytes = row < nk ? 16u : 0u;
+            const uint32_t kd = (uint32_t)__cvta_generic_to_shared(Ks + row * STRIDE + ch * 16);
+            const uint32_t vd = (uint32_t)__cvta_generic_to_shared(Vs + row * STRIDE + ch * 16);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(kd), "l"(Kh + (size_t)(key0 + rr) * DH + ch * 8), "r"(nbytes) : "memory");
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(vd), "l"(Vh + (size_t)(key0 + rr) * DH + ch * 8), "r"(nbytes) : "memory");
+        }
+        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+        float sc[kKeyBlock / 8][4];
+#pragma unroll
+        for (int nt = 0; nt < kKeyBlock / 8; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+            for (int nt = 0; nt < kKeyBlock / 8; ++nt) {
+                const unsigned char* kp = Ks + (nt * 8 + g) * STRIDE + (ks * 16 + q4 * 2) * 2;
+                mma_bf16_16816(sc[nt], qf[ks], *reinterpret_cast<const uint32_t*>(kp), *reinterpret_cast<const uint32_t*>(kp + 16));
+            }
+        }
+        // scale, hide the keys past each row's position (and everything from rows not in this pass), new row maxima
+        float bm0 = -INFINITY, bm1 = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < kKeyBlock / 8; ++nt) {
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                const int key = key0 + nt * 8 + q4 * 2 + c;
+                sc[nt][c] = (act0 && key <= last0) ? sc[nt][c] * scale : -INFINITY;
+                sc[nt][2 + c] = (act1 && key <= last1) ? sc[nt][2 + c] * scale : -INFINITY;
+                bm0 = fmaxf(bm0, sc[nt][c]);
+                bm1 = fmaxf(bm1, sc[nt][2 + c]);
+            }
+        }
+        bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, 1));
+        bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, 2));
+        bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, 1));
+        bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, 2));
+        // a row that has seen no key yet (and sees none here) keeps m = -inf: nothing to rescale, nothing to add
+        const float n0 = fmaxf(m0, bm0), n1 = fmaxf(m1, bm1);
+        const float c0 = n0 == -INFINITY ? 1.f : expf(m0 - n0), c1 = n1 == -INFINITY ? 1.f : expf(m1 - n1);
+        m0 = n0;
+        m1 = n1;
+        l0 *= c0;
+        l1 *= c1;
+#pragma unroll
+        for (int i = 0; i < DT; ++i) {
+            o[i][0] *= c0;
+            o[i][1] *= c0;
+            o[i][2] *= c1;
+            o[i][3] *= c1;
+        }
+        uint32_t pf[kKeyBlock / 16][4];
+#pragma unroll
+        for (int nt = 0; nt < kKeyBlock / 8; ++nt) {
+            const float p0 = sc[nt][0] > -INFINITY ? expf(sc[nt][0] - m0) : 0.f, p1 = sc[nt][1] > -INFINITY ? expf(sc[nt][1] - m0) : 0.f;
+            const float p2 = sc[nt][2] > -INFINITY ? expf(sc[nt][2] - m1) : 0.f, p3 = sc[nt][3] > -INFINITY ? expf(sc[nt][3] - m1) : 0.f;
+            l0 += p0 + p1;
+            l1 += p2 + p3;
+            pf[nt / 2][(nt & 1) * 2] = pack_bf16(p0, p1);
+            pf[nt / 2][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+        }
+#pragma unroll
+        for (int kk = 0; kk < kKeyBlock / 16; ++kk) {
+#pragma unroll
+            for (int dt = 0; dt < DT; ++dt) {
+                uint32_t b0, b1;
+                const uint32_t addr = (uint32_t)__cvta_generic_to_shared(Vs + (kk * 16 + (lane & 15)) * STRIDE + dt * 16);
+                asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(addr));
+                mma_bf16_16816(o[dt], pf[kk], b0, b1);
+            }
+        }
+    }
+    }
+    if (bad && threadIdx.x == 0) *dev_status = DSMOE_ERR_INVALID_ARG;      // clamped above: nothing left the cache
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    // ---- merge the warps' partial results: per warp 16 maxima, 16 sums, 16 x DH accumulators
+    __syncthreads();
+    float* ms = reinterpret_cast<float*>(moa_mma_smem);                 // [warps][16]
+    float* ls = ms + kMmaWarps * 16;                                    // [warps][16]
+    float* os = ls + kMmaWarps * 16;                                    // [warps][16][DH]
+    if (q4 == 0) {
+        ms[warp * 16 + g] = m0;
+        ms[warp * 16 + g + 8] = m1;
+        ls[warp * 16 + g] = l0;
+        ls[warp * 16 + g + 8] = l1;
+    }
+#pragma unroll
+    for (int dt = 0; dt < DT; ++dt) {
+        float* o0 = os + ((size_t)warp * 16 + g) * DH + dt * 8 + q4 * 2;
+        float* o1 = os + ((size_t)warp * 16 + g + 8) * DH + dt * 8 + q4 * 2;
+        o0[0] = o[dt][0];
+        o0[1] = o[dt][1];
+        o1[0] = o[dt][2];
+        o1[1] = o[dt][3];
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < 16 * DH; idx += 32 * kMmaWarps) {
+        const int row = idx / DH, dcol = idx % DH;
+        int tok, slot;
+        row_token_slot(row, tok, slot);
+        if (tok >= T || slot >= W) continue;
+        const int r = token_rows[(size_t)tok * W + slot];
+        if (r < 0 || r >= amax) continue;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kMmaWarps; ++w) M = fmaxf(M, ms[w * 16 + row]);
+        float num = 0.f, den = 0.f;
+#pragma unroll
+        for (int w = 0; w < kMmaWarps; ++w) {
+            const float wgt = expf(ms[w * 16 + row] - M);               // 0 for a warp that saw no key
+            num = fmaf(wgt, os[((size_t)w * 16 + row) * DH + dcol], num);
+            den = fmaf(wgt, ls[w * 16 + row], den);
+        }
+        qa[(size_t)r * H + j * DH + dcol] = __float2bfloat16_rn(num / den);
+    }
+}
+
+template <int DH, int kMmaWarps>
+dsmoe_status launch_mma_attention_nw(const dsmoe_layer_desc& p, const MoaCore& c, __nv_bfloat16* q, const int32_t* token_rows,
+                                  int32_t* dev_status, cudaStream_t s) {
+    constexpr size_t stride = DH * 2 + 16;
+    const size_t loop_bytes = (size_t)kMmaWarps * 2 * kKeyBlock * stride;
+    const size_t merge_bytes = (size_t)kMmaWarps * (32 + 16 * DH) * 4;
+    const size_t smem = loop_bytes > merge_bytes ? loop_bytes : merge_bytes;
+    static bool attr[kMaxDeviceSlots] = {};
+    int dev = 0;
+    DeviceState* st = nullptr;
+    DSMOE_TRY(device_state(&st, &dev));
+    if (!attr[dev]) {
+        DSMOE_CUDA_TRY(cudaFuncSetAttribute(moa_attention_mma_kernel<DH, kMmaWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr[dev] = true;
+    }
+    const int W = width_of(p), row_tiles = (W + 15) / 16;
+    // several tokens per tile where a token has few rows and there are tokens enough to fill the GPU without
+    const int tpt = (W <= 8 && (long long)p.T * c.n_head >= 8ll * st->sm_count) ? 16 / W : 1;
+    const long long ctas = (long long)((p.T + tpt - 1) / tpt) * c.n_head * row_tiles;
+    if (ctas > 0x7fffffffll) return DSMOE_ERR_UNSUPPORTED;
+    moa_attention_mma_kernel<DH, kMmaWarps><<<(unsigned)ctas, 32 * kMmaWarps, smem, s>>>(
+        q, token_rows, W, row_tiles, tpt, (long long)amax_of(p), c.n_head, p.H, p.T, static_cast<const __nv_bfloat16*>(c.Kc),
+        static_cast<const __nv_bfloat16*>(c.Vc), c.tok_seq, c.pos, c.n_seq, c.L, c.scale, dev_status);
+    return DSMOE_OK;
+}
+
+template <int DH>
+dsmoe_status launch_mma_attention(const dsmoe_layer_desc& p, const MoaCore& c, __nv_bfloat16* q, const int32_t* token_rows,
+                                  int32_t* dev_status, cudaStream_t s) {
+    if (c.L <= 512) return launch_mma_attention_nw<DH, 2>(p, c, q, token_rows, dev_status, s);
+    return launch_mma_attention_nw<DH, 8>(p, c, q, token_rows, dev_status, s);
+}
+
 }  // namespace
 
 bool moa_supported(const dsmoe_layer_desc& p, int n_head, int L) {
@@ -108,8 +371,19 @@ bool moa_supported(const dsmoe_layer_desc& p, int n_head, int L) {
 }
 
 dsmoe_status launch_moa_attention(const dsmoe_layer_desc& p, const MoaCore& c, void* qa, const int32_t* row_token,
-                                  const int32_t* offsets, int32_t* dev_status, cudaStream_t s) {
+                                  const int32_t* token_rows, const int32_t* offsets, int32_t* dev_status, cudaStream_t s) {
     const int dh = p.H / c.n_head;
+    if (token_rows && (dh == 64 || dh == 96 || dh == 128) && !getenv("DSMOE_MOA_PLAIN")) {
+        // head widths of the paper's models: the tensor-core kernel, a CTA per (token, head)
+        int timed = -1;
+        DSMOE_TRY(timing_begin(s, &timed));
+        auto* qb = static_cast<__nv_bfloat16*>(qa);
+        if (dh == 64) DSMOE_TRY(launch_mma_attention<64>(p, c, qb, token_rows, dev_status, s));
+        else if (dh == 96) DSMOE_TRY(launch_mma_attention<96>(p, c, qb, token_rows, dev_status, s));
+        else DSMOE_TRY(launch_mma_attention<128>(p, c, qb, token_rows, dev_status, s));
+        DSMOE_CUDA_TRY(cudaGetLastError());
+        return timing_end(s, timed);
+    }
     int warps = kMoaWarps;
     const size_t per_warp = (size_t)(dh + ((c.L + 3) & ~3)) * 4;
     const size_t smem = per_warp * warps;
@@ -119,6 +393,8 @@ dsmoe_status launch_moa_attention(const dsmoe_layer_desc& p, const MoaCore& c, v
     auto* q = static_cast<__nv_bfloat16*>(qa);
     auto* K = static_cast<const __nv_bfloat16*>(c.Kc);
     auto* V = static_cast<const __nv_bfloat16*>(c.Vc);
+    int timed = -1;
+    DSMOE_TRY(timing_begin(s, &timed));
 #define MOA_LAUNCH(DPL)                                                                                                   \
     do {                                                                                                                  \
         if (smem > 48 * 1024)                                                                                             \
@@ -140,6 +416,7 @@ dsmoe_status launch_moa_attention(const dsmoe_layer_desc& p, const MoaCore& c, v
     }
 #undef MOA_LAUNCH
     DSMOE_CUDA_TRY(cudaGetLastError());
+    DSMOE_TRY(timing_end(s, timed));
     return DSMOE_OK;
 }
 
