@@ -53,7 +53,7 @@ for _n, (_d, _H, _K) in PAPER_SHAPES.items():
     WORKLOADS[f"paper{_n}_prefill"] = ("c3", dict(T=8192, d=_d, H=_H, K=_K))
     WORKLOADS[f"paper{_n}_t32"] = ("c2", dict(T=32, d=_d, H=_H))
 # dram bytes per launch of the dominant kernel from the ncu captures under profiles/ (c3: mean of the up- and down-projection)
-NCU_TRAFFIC_BYTES = {"c2_t32": 274.4e6, "c3": 1541.3e6}
+NCU_TRAFFIC_BYTES = {"c2_t32": 274.4e6, "c3": 1522.9e6, "c4": 2581.4e6}
 DEFAULT_STEPS = {"c3": 100, "c3_separate": 100, "c4": 50}
 ALSO = [("c2_t1", 500), ("c2_t8", 500), ("c3", 30), ("c3_separate", 30), ("c4", 15)] + [(f"c5_eps{e}", 15) for e in (0.0, 0.01, 0.05, 0.1, 0.2)] + \
        [(f"paper{n}_prefill", 30) for n in PAPER_SHAPES] + [(f"paper{n}_t32", 300) for n in ("1b", "3b", "6b", "19b")] + \
@@ -552,12 +552,20 @@ def run_moa(name: str, steps: int, warmup: int, sampler_index=0):
     weight_bytes = 2.0 * E * d * H * 2.0
     ach = proj_flops / ((durs[0] + durs[2]) * 1e-3) / 1e12
     t_flop, t_byte = (proj_flops + att_flops) / (P["tf_burst"] * 1e12), (weight_bytes + kv_bytes) / (P["hbm"] * 1e9)
-    roof = dict(bound="tensor" if t_flop >= t_byte else "hbm", kernel="umma_gemm_kernel (projections), moa_attention_kernel",
-                achieved=ach, peak=P["tf_burst"], unit="TFLOP/s", peak_source=P["source"] + " (burst bf16; projections only)",
-                frac=ach / P["tf_burst"], frac_burst=ach / P["tf_burst"], frac_sustained=ach / P["tf_sustained"],
-                frac_nominal=ach / NOMINAL["tf"], roofline_ms=max(t_flop, t_byte) * 1e3,
+    if t_flop >= t_byte:
+        # many tokens: the two projections' flops against the measured GEMM rate (their two launches' time)
+        head = dict(bound="tensor", achieved=ach, peak=P["tf_burst"], unit="TFLOP/s",
+                    peak_source=P["source"] + " (burst bf16; the two projections)", frac=ach / P["tf_burst"],
+                    frac_burst=ach / P["tf_burst"], frac_sustained=ach / P["tf_sustained"], frac_nominal=ach / NOMINAL["tf"])
+    else:
+        # few tokens: every expert's projection weights and the visible keys and values, read once, against the
+        # measured copy bandwidth (all three launches' time)
+        gbs = (weight_bytes + kv_bytes) / (float(durs.sum()) * 1e-3) / 1e9
+        head = dict(bound="hbm", achieved=gbs, peak=P["hbm"], unit="GB/s", peak_source=P["source"] + " (copy bandwidth)",
+                    frac=gbs / P["hbm"], frac_nominal=gbs / NOMINAL["hbm"])
+    roof = dict(head, kernel="umma_gemm_kernel (projections) + moa_attention_mma_kernel", roofline_ms=max(t_flop, t_byte) * 1e3,
                 frac_of_roofline_time=max(t_flop, t_byte) / (float(durs.sum()) * 1e-3),
-                step_frac_of_roofline_time=max(t_flop, t_byte) / (ms * 1e-3), step_frac=proj_flops / (ms * 1e-3) / 1e12 / P["tf_burst"],
+                step_frac_of_roofline_time=max(t_flop, t_byte) / (ms * 1e-3), step_frac=max(t_flop, t_byte) / (ms * 1e-3),
                 algorithmic_per_launch=proj_flops / 2, attention_flops=att_flops, kv_bytes=kv_bytes, traffic=None,
                 kernel_ms_per_step=float(durs.sum()), ms_per_step_with_events=ms, launch_ms_each=[float(v) for v in durs],
                 launches_per_step=3)
