@@ -111,6 +111,9 @@ moa_attention_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restrict__
 // P.V with P taken straight from S's registers -- the usual streaming-softmax order.  The warps' partial results
 // (maximum, sum, accumulator per row) are merged through shared memory at the end, in warp order.
 constexpr int kKeyBlock = 32;
+#ifndef DSMOE_MOA_MINBLOCKS
+#define DSMOE_MOA_MINBLOCKS 6
+#endif
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -124,7 +127,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 template <int DH, int kMmaWarps>      // long caches: 8 warps share out the keys; short ones: 2, and several CTAs fit an SM
-__global__ void __launch_bounds__(32 * kMmaWarps)
+__global__ void __launch_bounds__(32 * kMmaWarps, kMmaWarps == 2 ? DSMOE_MOA_MINBLOCKS : 1)
 moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restrict__ token_rows, int W, int row_tiles,
                          int tpt, long long amax, int n_head, int H, int T, const __nv_bfloat16* __restrict__ Kc,
                          const __nv_bfloat16* __restrict__ Vc, const int32_t* __restrict__ tok_seq,
