@@ -121,6 +121,7 @@ struct GemmParams {
     // dot_part[(token * E + e) * column_tiles + column_tile] (Eq. 3's <e_j(X), dO>, see launch_dense_backward)
     const __nv_bfloat16* act;   // [rows, E * n_per_expert] hidden activations GeLU(x.W1[e])
     float* dot_part;
+    int stage_f32;              // EPI_GELU, EPI_STORE: rows go out through a shared-memory tile (set by launch_gemm)
 };
 
 struct Tile {
@@ -750,6 +751,86 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (valid) {
                     const int ntn = (P.n_per_expert + BN - 1) / BN;
                     P.dot_part[(grow * P.E + t.e) * ntn + t.n0 / BN] = active ? dot : 0.f;
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) release_acc(acc);
+                if (++acc == 2) {
+                    acc = 0;
+                    aph ^= 1u;
+                }
+                continue;
+            }
+            if (P.out_f32 && P.stage_f32) {
+                // fp32 rows through a shared-memory tile: out of TMEM a lane holds 32 columns of ONE row (128 bytes that
+                // it would store as eight scattered 16-byte pieces); turned through the tile, 8 lanes store one row's 128
+                // bytes together, four whole rows per instruction
+                constexpr int LD = 36;                  // floats per staged row: 16-byte aligned, conflict-free in quarter warps
+                float* tp = reinterpret_cast<float*>(smem_raw + (base - raw) + RING_BYTES + SHARED_BYTES) + q * 32 * LD;
+                const int rr = lane >> 3, cc = lane & 7;
+                float* const out_f = static_cast<float*>(P.out);
+                for (int c = 0; warp_has_rows && c < t.bn; c += 32) {
+                    uint32_t r[32];
+                    ptx::tmem_ld32(taddr + (uint32_t)c, r);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<float4*>(tp + lane * LD + 4 * j) =
+                            make_float4(g * __uint_as_float(r[4 * j]), g * __uint_as_float(r[4 * j + 1]),
+                                        g * __uint_as_float(r[4 * j + 2]), g * __uint_as_float(r[4 * j + 3]));
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int rl = i * 4 + rr;      // row of this warp's 32
+                        if (q * 32 + rl < t.rows_valid)
+                            *reinterpret_cast<float4*>(out_f + ((long long)t.row0 + q * 32 + rl) * P.ld_out + t.out_col0 + c + cc * 4) =
+                                *reinterpret_cast<const float4*>(tp + rl * LD + cc * 4);
+                    }
+                    __syncwarp();
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) release_acc(acc);
+                if (++acc == 2) {
+                    acc = 0;
+                    aph ^= 1u;
+                }
+                continue;
+            }
+            if (P.stage_f32 && !P.out_f32) {
+                // bf16 rows (hidden activations, bf16 outputs) the same way: a lane's 64 bytes of one row go through the
+                // tile, 4 lanes store a row's 64 bytes together, eight rows per instruction
+                constexpr int LDB = 80;                 // bytes per staged row
+                unsigned char* tb = smem_raw + (base - raw) + RING_BYTES + SHARED_BYTES + q * 32 * LDB;
+                const int rr = lane >> 2, cc = lane & 3;
+                __nv_bfloat16* const out_h = static_cast<__nv_bfloat16*>(P.out);
+                for (int c = 0; warp_has_rows && c < t.bn; c += 32) {
+                    uint32_t r[32];
+                    ptx::tmem_ld32(taddr + (uint32_t)c, r);
+                    ptx::tmem_ld_wait();
+                    uint4 pk[4];
+                    __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
+                    if (P.epi == EPI_GELU) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            hv[j] = __floats2bfloat162_rn(g * gelu_erf(__uint_as_float(r[2 * j])),
+                                                          g * gelu_erf(__uint_as_float(r[2 * j + 1])));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            hv[j] = __floats2bfloat162_rn(g * __uint_as_float(r[2 * j]), g * __uint_as_float(r[2 * j + 1]));
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(tb + lane * LDB + 16 * j) = pk[j];
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int rl = i * 8 + rr;
+                        if (q * 32 + rl < t.rows_valid)
+                            *reinterpret_cast<uint4*>(out_h + ((long long)t.row0 + q * 32 + rl) * P.ld_out + t.out_col0 + c + cc * 8) =
+                                *reinterpret_cast<const uint4*>(tb + rl * LDB + 16 * cc);
+                    }
+                    __syncwarp();
                 }
                 ptx::tc_fence_before();
                 __syncwarp();
@@ -1792,7 +1873,7 @@ int pair_override() {
 
 // pair_tiles: an upper bound of the number of 256-row tiles (INT_MAX where only the device knows, as in the grouped
 // modes); 0 = never pair (the caller's shapes do not allow it).
-dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams& P, int grid, cudaStream_t s,
+dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams& P_in, int grid, cudaStream_t s,
                          bool may_time = true, int pair_tiles = 0) {
     DeviceState* st = nullptr;
     DSMOE_TRY(device_state(&st));
@@ -1801,8 +1882,12 @@ dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams&
         DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_CMB_BYTES));
         st->attr_gemm = true;
     }
+    GemmParams Pl = P_in;
+    // EPI_GELU and EPI_STORE send their rows out through a shared-memory tile (whole rows per store instruction)
+    Pl.stage_f32 = ((P_in.epi == EPI_STORE || P_in.epi == EPI_GELU) && !getenv("DSMOE_NO_STAGE")) ? 1 : 0;
+    const GemmParams& P = Pl;
     int threads = (P.gather || P.epi == EPI_COMBINE) ? GATHER_THREADS : NUM_THREADS;
-    const size_t smem = P.epi == EPI_COMBINE ? SMEM_GEMM_CMB_BYTES : SMEM_GEMM_BYTES;
+    const size_t smem = (P.epi == EPI_COMBINE || P.stage_f32) ? SMEM_GEMM_CMB_BYTES : SMEM_GEMM_BYTES;
     if (st->max_pairs < 0) {
         // how many clusters of two CTAs fit the device at once (the persistent kernel launches no more)
         cudaLaunchConfig_t q{};
