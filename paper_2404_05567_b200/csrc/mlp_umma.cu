@@ -121,7 +121,6 @@ struct GemmParams {
     // dot_part[(token * E + e) * column_tiles + column_tile] (Eq. 3's <e_j(X), dO>, see launch_dense_backward)
     const __nv_bfloat16* act;   // [rows, E * n_per_expert] hidden activations GeLU(x.W1[e])
     float* dot_part;
-    int stage_f32;              // EPI_GELU, EPI_STORE: rows go out through a shared-memory tile (set by launch_gemm)
 };
 
 struct Tile {
@@ -761,8 +760,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
                 continue;
             }
-            if (P.out_f32 && P.stage_f32) {
-                // fp32 rows through a shared-memory tile: out of TMEM a lane holds 32 columns of ONE row (128 bytes that
+            // EPI_GELU and EPI_STORE.  The rows go out through a shared-memory tile.
+            if (P.out_f32) {
+                // fp32 rows: out of TMEM a lane holds 32 columns of ONE row (128 bytes that
                 // it would store as eight scattered 16-byte pieces); turned through the tile, 8 lanes store one row's 128
                 // bytes together, four whole rows per instruction
                 constexpr int LD = 36;                  // floats per staged row: 16-byte aligned, conflict-free in quarter warps
@@ -788,16 +788,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                     __syncwarp();
                 }
-                ptx::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) release_acc(acc);
-                if (++acc == 2) {
-                    acc = 0;
-                    aph ^= 1u;
-                }
-                continue;
-            }
-            if (P.stage_f32 && !P.out_f32) {
+            } else {
                 // bf16 rows (hidden activations, bf16 outputs) the same way: a lane's 64 bytes of one row go through the
                 // tile, 4 lanes store a row's 64 bytes together, eight rows per instruction
                 constexpr int LDB = 80;                 // bytes per staged row
@@ -831,47 +822,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                 *reinterpret_cast<const uint4*>(tb + rl * LDB + 16 * cc);
                     }
                     __syncwarp();
-                }
-                ptx::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) release_acc(acc);
-                if (++acc == 2) {
-                    acc = 0;
-                    aph ^= 1u;
-                }
-                continue;
-            }
-            for (int c = 0; warp_has_rows && c < t.bn; c += 32) {
-                uint32_t r[32];
-                ptx::tmem_ld32(taddr + (uint32_t)c, r);
-                ptx::tmem_ld_wait();
-                if (!valid) continue;
-                const long long o = grow * P.ld_out + t.out_col0 + c;
-                if (P.epi == EPI_GELU) {
-                    uint4 pk[4];
-                    __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
-#pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        hv[j] = __floats2bfloat162_rn(g * gelu_erf(__uint_as_float(r[2 * j])),
-                                                      g * gelu_erf(__uint_as_float(r[2 * j + 1])));
-                    uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) + o);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) dst[j] = pk[j];
-                } else if (P.out_f32) {
-                    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(P.out) + o);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        dst[j] = make_float4(g * __uint_as_float(r[4 * j]), g * __uint_as_float(r[4 * j + 1]),
-                                             g * __uint_as_float(r[4 * j + 2]), g * __uint_as_float(r[4 * j + 3]));
-                } else {
-                    uint4 pk[4];
-                    __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
-#pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        hv[j] = __floats2bfloat162_rn(g * __uint_as_float(r[2 * j]), g * __uint_as_float(r[2 * j + 1]));
-                    uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) + o);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) dst[j] = pk[j];
                 }
             }
             ptx::tc_fence_before();
@@ -1882,12 +1832,10 @@ dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams&
         DSMOE_CUDA_TRY(cudaFuncSetAttribute(umma_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_GEMM_CMB_BYTES));
         st->attr_gemm = true;
     }
-    GemmParams Pl = P_in;
-    // EPI_GELU and EPI_STORE send their rows out through a shared-memory tile (whole rows per store instruction)
-    Pl.stage_f32 = ((P_in.epi == EPI_STORE || P_in.epi == EPI_GELU) && !getenv("DSMOE_NO_STAGE")) ? 1 : 0;
-    const GemmParams& P = Pl;
+    const GemmParams& P = P_in;
     int threads = (P.gather || P.epi == EPI_COMBINE) ? GATHER_THREADS : NUM_THREADS;
-    const size_t smem = (P.epi == EPI_COMBINE || P.stage_f32) ? SMEM_GEMM_CMB_BYTES : SMEM_GEMM_BYTES;
+    // the ring, the barriers, and the tile the epilogues send their rows through (EPI_BWD needs none)
+    const size_t smem = P.epi == EPI_BWD ? SMEM_GEMM_BYTES : SMEM_GEMM_CMB_BYTES;
     if (st->max_pairs < 0) {
         // how many clusters of two CTAs fit the device at once (the persistent kernel launches no more)
         cudaLaunchConfig_t q{};

@@ -376,6 +376,7 @@ bool moa_supported(const dsmoe_layer_desc& p, int n_head, int L) {
 dsmoe_status launch_moa_attention(const dsmoe_layer_desc& p, const MoaCore& c, void* qa, const int32_t* row_token,
                                   const int32_t* token_rows, const int32_t* offsets, int32_t* dev_status, cudaStream_t s) {
     const int dh = p.H / c.n_head;
+    // DSMOE_MOA_PLAIN in the environment sends every head width to the plain kernel (a testing aid)
     if (token_rows && (dh == 64 || dh == 96 || dh == 128) && !getenv("DSMOE_MOA_PLAIN")) {
         // head widths of the paper's models: the tensor-core kernel, a CTA per (token, head)
         int timed = -1;

@@ -136,3 +136,12 @@ def test_moa_rejects_what_it_does_not_support():
     with pytest.raises(dm.DsmoeError) as ei:
         dm.dsmoe_moa_forward(desc, 2, 1.0, K, K, None, z, z, z, None, z, z, None, None, z)
     assert ei.value.code in (1, 2)
+
+
+def test_moa_plain_attention_kernel_on_a_common_head_width(monkeypatch):
+    """Head widths 64, 96 and 128 normally take the tensor-core attention kernel; the plain one (other widths) is run on
+    such a shape too, through the library's switch for it."""
+    monkeypatch.setenv("DSMOE_MOA_PLAIN", "1")
+    s, *rest = _moa_case("moa_plain", 200, 512, 8, 2, 64, 3, 77, "mixed", gi.MODE_TOPK, K=3)
+    e, er = _run(s, *rest, 2, 0.125)
+    assert er <= TOL_BF16, (e, er)
