@@ -109,7 +109,8 @@ moa_attention_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restrict__
 // a warp copies its block of K and V into (padded, conflict-free) shared memory, forms S = Q.K^T (Q fragments stay
 // in registers for the whole kernel), updates the running row maxima and sums, rescales its accumulators and adds
 // P.V with P taken straight from S's registers -- the usual streaming-softmax order.  The warps' partial results
-// (maximum, sum, accumulator per row) are merged through shared memory at the end, in warp order.
+// (maximum, sum, accumulator per row) are merged through shared memory at the end, in warp order.  Exponentials are
+// the fast ones (ex2.approx of the argument times log2 e): the weights are rounded to bf16 before P.V anyway.
 constexpr int kKeyBlock = 32;
 #ifndef DSMOE_MOA_MINBLOCKS
 #define DSMOE_MOA_MINBLOCKS 6
@@ -131,7 +132,8 @@ __global__ void __launch_bounds__(32 * kMmaWarps, kMmaWarps == 2 ? DSMOE_MOA_MIN
 moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restrict__ token_rows, int W, int row_tiles,
                          int tpt, long long amax, int n_head, int H, int T, const __nv_bfloat16* __restrict__ Kc,
                          const __nv_bfloat16* __restrict__ Vc, const int32_t* __restrict__ tok_seq,
-                         const int32_t* __restrict__ pos, int n_seq, int L, float scale, int* __restrict__ dev_status) {
+                         const int32_t* __restrict__ pos, int n_seq, int L, float scale, long long n_tiles,
+                         int* __restrict__ dev_status) {
     constexpr int STRIDE = DH * 2 + 16;                 // bytes per key row in shared memory: 16 of padding
     constexpr int KS = DH / 16, DT = DH / 8, CH = DH / 8;
     extern __shared__ __align__(16) unsigned char moa_mma_smem[];
@@ -139,9 +141,13 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
     // The tile's 16 rows: with tpt == 1, slots 16 rt .. of token t0; with tpt > 1 (rows per token W <= 8, one row
     // tile), all W slots of the tpt tokens t0, t0 + 1, ...: neighbouring tokens of one sequence see nearly the same
     // keys, so their rows share the copies of K and V.
-    const int rt = blockIdx.x % row_tiles;
-    const int j = (blockIdx.x / row_tiles) % n_head;
-    const int t0 = (blockIdx.x / (row_tiles * n_head)) * tpt;
+    // The CTAs are persistent (as many as fit the GPU at once) and walk the tiles: a tile is short, and starting a CTA per
+    // tile cost more than the tile's work.
+    for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    __syncthreads();                                    // the previous tile's merge has read shared memory
+    const int rt = (int)(tile % row_tiles);
+    const int j = (int)((tile / row_tiles) % n_head);
+    const int t0 = (int)(tile / ((long long)row_tiles * n_head)) * tpt;
     const auto row_token_slot = [&](int i, int& tok, int& slot) {
         if (tpt == 1) {
             tok = t0;
@@ -160,7 +166,7 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
     if (tk1 < T && sl1 < W) r1 = token_rows[(size_t)tk1 * W + sl1];
     if (r0 >= amax) r0 = -1;
     if (r1 >= amax) r1 = -1;
-    if (__syncthreads_or(r0 >= 0 || r1 >= 0) == 0) return;          // no rows in this tile
+    if (__syncthreads_or(r0 >= 0 || r1 >= 0) == 0) continue;        // no rows in this tile
     bool bad = false;
     if (r0 >= 0) {
         last0 = pos[tk0];
@@ -251,7 +257,7 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
         bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, 2));
         // a row that has seen no key yet (and sees none here) keeps m = -inf: nothing to rescale, nothing to add
         const float n0 = fmaxf(m0, bm0), n1 = fmaxf(m1, bm1);
-        const float c0 = n0 == -INFINITY ? 1.f : expf(m0 - n0), c1 = n1 == -INFINITY ? 1.f : expf(m1 - n1);
+        const float c0 = n0 == -INFINITY ? 1.f : __expf(m0 - n0), c1 = n1 == -INFINITY ? 1.f : __expf(m1 - n1);
         m0 = n0;
         m1 = n1;
         l0 *= c0;
@@ -266,8 +272,8 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
         uint32_t pf[kKeyBlock / 16][4];
 #pragma unroll
         for (int nt = 0; nt < kKeyBlock / 8; ++nt) {
-            const float p0 = sc[nt][0] > -INFINITY ? expf(sc[nt][0] - m0) : 0.f, p1 = sc[nt][1] > -INFINITY ? expf(sc[nt][1] - m0) : 0.f;
-            const float p2 = sc[nt][2] > -INFINITY ? expf(sc[nt][2] - m1) : 0.f, p3 = sc[nt][3] > -INFINITY ? expf(sc[nt][3] - m1) : 0.f;
+            const float p0 = sc[nt][0] > -INFINITY ? __expf(sc[nt][0] - m0) : 0.f, p1 = sc[nt][1] > -INFINITY ? __expf(sc[nt][1] - m0) : 0.f;
+            const float p2 = sc[nt][2] > -INFINITY ? __expf(sc[nt][2] - m1) : 0.f, p3 = sc[nt][3] > -INFINITY ? __expf(sc[nt][3] - m1) : 0.f;
             l0 += p0 + p1;
             l1 += p2 + p3;
             pf[nt / 2][(nt & 1) * 2] = pack_bf16(p0, p1);
@@ -324,11 +330,12 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
         float num = 0.f, den = 0.f;
 #pragma unroll
         for (int w = 0; w < kMmaWarps; ++w) {
-            const float wgt = expf(ms[w * 16 + row] - M);               // 0 for a warp that saw no key
+            const float wgt = __expf(ms[w * 16 + row] - M);               // 0 for a warp that saw no key
             num = fmaf(wgt, os[((size_t)w * 16 + row) * DH + dcol], num);
             den = fmaf(wgt, ls[w * 16 + row], den);
         }
         qa[(size_t)r * H + j * DH + dcol] = __float2bfloat16_rn(num / den);
+    }
     }
 }
 
@@ -350,11 +357,17 @@ dsmoe_status launch_mma_attention_nw(const dsmoe_layer_desc& p, const MoaCore& c
     const int W = width_of(p), row_tiles = (W + 15) / 16;
     // several tokens per tile where a token has few rows and there are tokens enough to fill the GPU without
     const int tpt = (W <= 8 && (long long)p.T * c.n_head >= 8ll * st->sm_count) ? 16 / W : 1;
-    const long long ctas = (long long)((p.T + tpt - 1) / tpt) * c.n_head * row_tiles;
-    if (ctas > 0x7fffffffll) return DSMOE_ERR_UNSUPPORTED;
+    const long long n_tiles = (long long)((p.T + tpt - 1) / tpt) * c.n_head * row_tiles;
+    static int per_sm_of[kMaxDeviceSlots] = {};      // CTAs of this kernel that fit an SM, asked once per device
+    if (!per_sm_of[dev])
+        DSMOE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm_of[dev], moa_attention_mma_kernel<DH, kMmaWarps>,
+                                                                     32 * kMmaWarps, smem));
+    const int per_sm = per_sm_of[dev];
+    const long long resident = (long long)st->sm_count * (per_sm > 0 ? per_sm : 1);
+    const long long ctas = n_tiles < resident ? n_tiles : resident;
     moa_attention_mma_kernel<DH, kMmaWarps><<<(unsigned)ctas, 32 * kMmaWarps, smem, s>>>(
         q, token_rows, W, row_tiles, tpt, (long long)amax_of(p), c.n_head, p.H, p.T, static_cast<const __nv_bfloat16*>(c.Kc),
-        static_cast<const __nv_bfloat16*>(c.Vc), c.tok_seq, c.pos, c.n_seq, c.L, c.scale, dev_status);
+        static_cast<const __nv_bfloat16*>(c.Vc), c.tok_seq, c.pos, c.n_seq, c.L, c.scale, n_tiles, dev_status);
     return DSMOE_OK;
 }
 
