@@ -54,7 +54,7 @@ for _n, (_d, _H, _K) in PAPER_SHAPES.items():
     WORKLOADS[f"paper{_n}_t32"] = ("c2", dict(T=32, d=_d, H=_H))
 # dram bytes per launch of the dominant kernel from the ncu captures under profiles/ (c3: mean of the up- and down-projection)
 NCU_TRAFFIC_BYTES = {"c2_t32": 272.8e6, "c3": 1532.5e6, "c4": 3175.4e6}
-DEFAULT_STEPS = {"c3": 100, "c3_separate": 100, "c4": 50}
+DEFAULT_STEPS = {"c3": 100, "c3_separate": 100, "c4": 50, "c4_backward": 20}
 ALSO = [("c2_t1", 500), ("c2_t8", 500), ("c3", 30), ("c3_separate", 30), ("c4", 15)] + [(f"c5_eps{e}", 15) for e in (0.0, 0.01, 0.05, 0.1, 0.2)] + \
        [(f"paper{n}_prefill", 30) for n in PAPER_SHAPES] + [(f"paper{n}_t32", 300) for n in ("1b", "3b", "6b", "19b")] + \
        [("decode_loop_t8", 20), ("decode_loop_t32", 20)]
@@ -573,6 +573,82 @@ def run_moa(name: str, steps: int, warmup: int, sampler_index=0):
                 assignments=A, active_experts=E, config=dict(w))
 
 
+def run_training_side(steps: int, warmup: int, sampler_index=0):
+    """The training side of the layer at the dense forward's shape (C4): the gradients of dense training (Eq. 3) for a
+    given output gradient -- two tensor-core launches, the recomputed activations and dO.W2^T with the gradients in its
+    epilogue -- and the router's mutual-information loss with its gradient (Eq. 4-6)."""
+    import torch
+    import paper_2404_05567_b200 as dm
+
+    def to_dev(a):
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+        return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+    s = gi.spec("c4")
+    desc = dm.make_desc(s.T, s.d, s.H, s.E, dm.BF16, s.mode, s.eps, s.eps_normalized, s.K, s.min_k, 0, 0)
+    P = peaks()
+    Wr, br = gi.router(s)
+    W1, W2 = gi.experts(s)
+    W2_d = to_dev(W2)
+    packed = packed_weights(dm, torch, s, desc, 0)
+    x_d, Wr_d = to_dev(gi.tokens(s)), to_dev(Wr)
+    br_d = to_dev(br) if br is not None else None
+    scores = torch.empty((s.T, s.E), dtype=torch.float32, device="cuda")
+    dm.dsmoe_router(desc, x_d, Wr_d, br_d, scores)
+    g = torch.Generator(device="cuda").manual_seed(0)
+    dO = torch.randn((s.T, s.d), generator=g, device="cuda").bfloat16()
+    dS = torch.empty((s.T, s.E), dtype=torch.float32, device="cuda")
+    dA = torch.empty((s.T, s.E * s.H), dtype=torch.bfloat16, device="cuda")
+    loss3 = torch.zeros(3, dtype=torch.float32, device="cuda")
+    grad = torch.empty((s.T, s.E), dtype=torch.float32, device="cuda")
+    ws = torch.empty(dm.dsmoe_workspace_size_packed(desc), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def step():
+        dm.dsmoe_dense_backward(desc, x_d, None, W2_d, packed, scores, None, dO, dS, dA, ws, status)
+
+    for _ in range(max(warmup, 3)):
+        step()
+    dm.dsmoe_timing_enable(2 * steps)
+    sampler = ClockSampler(sampler_index)
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    clocks = sampler.finish()
+    durs = np.array(dm.dsmoe_timing_read(2 * steps)).reshape(steps, 2).mean(axis=0)
+    dm.dsmoe_timing_enable(0)
+    assert int(status.item()) == 0
+    n_mi = 200
+    for _ in range(5):
+        dm.dsmoe_mi_loss(desc, scores, loss3, grad, ws)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(n_mi):
+        dm.dsmoe_mi_loss(desc, scores, loss3, grad, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    mi_us = e0.elapsed_time(e1) / n_mi * 1e3
+    flops = 4.0 * s.T * s.E * s.d * s.H
+    ach = flops / (float(durs.sum()) * 1e-3) / 1e12
+    roof = dict(bound="tensor", kernel="umma_gemm_kernel", achieved=ach, peak=P["tf_burst"], unit="TFLOP/s",
+                peak_source=P["source"] + " (burst bf16)", frac=ach / P["tf_burst"], frac_burst=ach / P["tf_burst"],
+                frac_sustained=ach / P["tf_sustained"], frac_nominal=ach / NOMINAL["tf"],
+                step_frac=flops / (ms * 1e-3) / 1e12 / P["tf_burst"], algorithmic_per_launch=flops / 2, traffic=None,
+                kernel_ms_per_step=float(durs.sum()), ms_per_step_with_events=ms, launch_ms_each=[float(v) for v in durs],
+                launches_per_step=2)
+    return dict(workload="c4_backward", value=s.T / (ms * 1e-3), unit="tokens/s", ms_per_step=ms, steps=steps, roofline=roof,
+                clocks=clocks, assignments=s.T * s.E, active_experts=s.E,
+                mi_loss={"us_per_call": mi_us, "tokens": s.T, "experts": s.E, "with_gradient": True,
+                         "bytes": 2.0 * s.T * s.E * 4, "L_MI": float(loss3[0].item())})
+
+
 def workload_config(name, s):
     mode = {0: "threshold", 1: "topk", 2: "all", 3: "threshold_topk"}[s.mode]
     return {"workload": name, "T": s.T, "d": s.d, "E": s.E, "H": s.H, "select": mode, "eps": s.eps, "K": s.K,
@@ -628,7 +704,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2_t32", choices=sorted(WORKLOADS) + sorted(MOA_WORKLOADS))
+    ap.add_argument("--workload", default="c2_t32", choices=sorted(WORKLOADS) + sorted(MOA_WORKLOADS) + ["c4_backward"])
     ap.add_argument("--no-extra", action="store_true")
     ap.add_argument("--graph", action="store_true", help="replay each step as one CUDA graph")
     ap.add_argument("--fuse-combine", type=int, default=None, choices=[0, 1, 2],
@@ -645,16 +721,18 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if name in MOA_WORKLOADS:
-        # the attention layer alone (one GPU; a diagnostic line: the default line is the feed-forward layer's)
+    if name in MOA_WORKLOADS or name == "c4_backward":
+        # the attention layer, or the training side, alone (one GPU; a diagnostic line: the default line is the
+        # feed-forward layer's)
         import torch
         torch.cuda.set_device(0)
         from paper_2404_05567_b200 import build as lib_build
         lib_build.build()
         gi.build()
-        r = run_moa(name, steps, warmup)
-        print(json.dumps(dict(metric="moa_layer_tokens_per_s", n_gpus=1, warmup=max(warmup, 3), higher_is_better=True,
-                              dtype="bf16", data="synthetic", gpu_launches=11 * steps, **r)))
+        r = run_training_side(steps, warmup) if name == "c4_backward" else run_moa(name, steps, warmup)
+        print(json.dumps(dict(metric="dense_backward_tokens_per_s" if name == "c4_backward" else "moa_layer_tokens_per_s",
+                              n_gpus=1, warmup=max(warmup, 3), higher_is_better=True, dtype="bf16", data="synthetic",
+                              gpu_launches=(3 if name == "c4_backward" else 11) * steps, **r)))
         return
     if args.fuse_combine is not None:
         for k in WORKLOADS:
@@ -731,6 +809,8 @@ def main():
                              "active_experts_per_layer": r["active_experts_per_layer"],
                              "activation_rms_per_layer": r["activation_rms_per_layer"],
                              "near_threshold_1e-6": r["stats"]["near_threshold"]})
+            drop_weights(torch)
+            also.append(run_training_side(10, 3, sampler_index=physical_gpu_index(local_rank)))
             for other, k in (("moa6b_prefill", 20), ("moa6b_decode", 200)):
                 drop_weights(torch)
                 also.append(run_moa(other, k, 5, sampler_index=physical_gpu_index(local_rank)))

@@ -719,18 +719,30 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const bool active = valid && (!P.sel_mask || ((P.sel_mask[grow] >> t.e) & 1ull));   // Eq. 2's mask M
                 const float gs = active ? g : 0.f;
                 float dot = 0.f;
+                // the activations come in and the gradients go out through two shared-memory tiles, whole rows per
+                // load / store instruction (4 lanes a row's 64 bytes, eight rows at a time)
+                constexpr int LDB = 80;                 // bytes per staged row
+                unsigned char* ta = smem_raw + (base - raw) + RING_BYTES + SHARED_BYTES + q * 2 * 32 * LDB;
+                unsigned char* tb = ta + 32 * LDB;
+                const int rr = lane >> 2, cc = lane & 3;
+                const __nv_bfloat16* const act = P.act;
+                __nv_bfloat16* const out_h = static_cast<__nv_bfloat16*>(P.out);
                 for (int c = 0; warp_has_rows && c < t.bn; c += 32) {
-                    const long long o = grow * P.ld_out + t.out_col0 + c;
-                    uint4 av[4];
-                    if (active) {
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) av[j] = __ldg(reinterpret_cast<const uint4*>(P.act + o) + j);
+                    for (int i = 0; i < 4; ++i) {
+                        const int rl = i * 8 + rr;
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (q * 32 + rl < t.rows_valid)
+                            v = __ldg(reinterpret_cast<const uint4*>(act + ((long long)t.row0 + q * 32 + rl) * P.ld_out + t.out_col0 + c + cc * 8));
+                        *reinterpret_cast<uint4*>(ta + rl * LDB + 16 * cc) = v;
                     }
                     uint32_t r[32];
                     ptx::tmem_ld32(taddr + (uint32_t)c, r);
                     ptx::tmem_ld_wait();
-                    if (!valid) continue;
-                    uint4 pk[4];
+                    __syncwarp();
+                    uint4 av[4], pk[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) av[j] = *reinterpret_cast<const uint4*>(ta + lane * LDB + 16 * j);
                     __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(pk);
                     const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(av);
 #pragma unroll
@@ -743,9 +755,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                         hv[j] = __floats2bfloat162_rn(gs * g0, gs * g1);
                     }
-                    uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) + o);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) dst[j] = pk[j];
+                    for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(tb + lane * LDB + 16 * j) = pk[j];
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int rl = i * 8 + rr;
+                        if (q * 32 + rl < t.rows_valid)
+                            *reinterpret_cast<uint4*>(out_h + ((long long)t.row0 + q * 32 + rl) * P.ld_out + t.out_col0 + c + cc * 8) =
+                                *reinterpret_cast<const uint4*>(tb + rl * LDB + 16 * cc);
+                    }
+                    __syncwarp();
                 }
                 if (valid) {
                     const int ntn = (P.n_per_expert + BN - 1) / BN;
@@ -1834,8 +1854,8 @@ dsmoe_status launch_gemm(const CUtensorMap& a, const BMaps& b, const GemmParams&
     }
     const GemmParams& P = P_in;
     int threads = (P.gather || P.epi == EPI_COMBINE) ? GATHER_THREADS : NUM_THREADS;
-    // the ring, the barriers, and the tile the epilogues send their rows through (EPI_BWD needs none)
-    const size_t smem = P.epi == EPI_BWD ? SMEM_GEMM_BYTES : SMEM_GEMM_CMB_BYTES;
+    // the ring, the barriers, and the tiles the epilogues send their rows through
+    const size_t smem = SMEM_GEMM_CMB_BYTES;
     if (st->max_pairs < 0) {
         // how many clusters of two CTAs fit the device at once (the persistent kernel launches no more)
         cudaLaunchConfig_t q{};
