@@ -121,6 +121,9 @@ struct GemmParams {
     // dot_part[(token * E + e) * column_tiles + column_tile] (Eq. 3's <e_j(X), dO>, see launch_dense_backward)
     const __nv_bfloat16* act;   // [rows, E * n_per_expert] hidden activations GeLU(x.W1[e])
     float* dot_part;
+    // GEMM_DENSE_UP: "expert" e reads A's columns from e * a_expert_stride on (0: every expert reads the same columns;
+    // the router's logits use it to cut their reduction into pieces with an output block each)
+    int a_expert_stride;
 };
 
 struct Tile {
@@ -415,7 +418,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     } else {
                         b_e = t.e;
                         b_k = i * BK;
-                        a_col = b_k;
+                        a_col = t.e * P.a_expert_stride + b_k;
                     }
                     if (!P.gather) {
                         if (PAIR) ptx::tma_load_2d_pair(smA + s * A_STAGE_BYTES, &tmA, bar, a_col, t.row0);
@@ -1936,27 +1939,36 @@ __global__ void __launch_bounds__(256) router_split_kernel(const float* __restri
 }
 
 // logits = (s1 + s2) + s3 + bias per expert, then softmax and selection: one warp per token
+// (the reduction over d may come in `pieces` blocks of 3 EP sums each, added in ascending order)
 __global__ void __launch_bounds__(256) router_finish_kernel(const float* __restrict__ sums, const float* __restrict__ br,
                                                             float* __restrict__ scores, uint64_t* __restrict__ mask,
-                                                            int32_t* __restrict__ k_t, int T, int EP, SelParams q) {
+                                                            int32_t* __restrict__ k_t, int T, int EP, int pieces, SelParams q) {
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (t >= T) return;
-    const float* row = sums + (size_t)t * 3 * EP;
+    const float* row = sums + (size_t)t * 3 * EP * pieces;
     const bool v_lo = lane < q.E, v_hi = lane + 32 < q.E;
     float l_lo = 0.f, l_hi = 0.f;
-    if (v_lo) l_lo = ((row[lane] + row[EP + lane]) + row[2 * EP + lane]) + (br ? br[lane] : 0.f);
-    if (v_hi) l_hi = ((row[lane + 32] + row[EP + lane + 32]) + row[2 * EP + lane + 32]) + (br ? br[lane + 32] : 0.f);
+    for (int pc = 0; pc < pieces; ++pc, row += 3 * EP) {
+        if (v_lo) l_lo += (row[lane] + row[EP + lane]) + row[2 * EP + lane];
+        if (v_hi) l_hi += (row[lane + 32] + row[EP + lane + 32]) + row[2 * EP + lane + 32];
+    }
+    if (v_lo && br) l_lo += br[lane];
+    if (v_hi && br) l_hi += br[lane + 32];
     softmax_select_store(l_lo, l_hi, t, q, lane, scores, mask, k_t);
 }
 
 }  // namespace
 
+// With few row tiles the logits' reduction over d is cut into 2 or 4 pieces, each a tile with its own block of sums,
+// so that the launch covers most SMs instead of T / 128 of them.
+constexpr int kRouterMaxPieces = 4;
+
 size_t router_umma_scratch(const dsmoe_layer_desc& p, size_t* split_bytes) {
     const size_t EP = p.E <= 32 ? 32 : 64;
     const size_t a = align_up(3 * EP * (size_t)p.d * 2, 256);
     if (split_bytes) *split_bytes = a;
-    return a + align_up((size_t)p.T * 3 * EP * 4, 256);
+    return a + align_up((size_t)p.T * kRouterMaxPieces * 3 * EP * 4, 256);
 }
 
 bool router_umma_supported(const dsmoe_layer_desc& p) { return umma_supported(p) && p.T > 256; }
@@ -1974,13 +1986,17 @@ dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const 
     const CUtensorMap* mA;
     const BMaps* mB;
     DSMOE_TRY(cached_map_2d(&mA, x, p.T, p.d, BM));
-    DSMOE_TRY(cached_bmaps(&mB, wsplit, 1, 3 * EP, p.d));
+    const int row_tiles = ceil_div(p.T, BM);
+    int pieces = kRouterMaxPieces;
+    while (pieces > 1 && (row_tiles * pieces > sm_count() || (p.d / BK) % pieces)) pieces /= 2;
+    DSMOE_TRY(cached_bmaps(&mB, wsplit, pieces, 3 * EP, p.d / pieces));
     GemmParams g{};
-    g.mode = GEMM_DENSE_DOWN; g.epi = EPI_STORE; g.E = 1; g.n_per_expert = 3 * EP; g.k_per_expert = p.d; g.rows = p.T;
-    g.out = sums; g.ld_out = 3 * EP; g.out_f32 = 1; g.dev_status = dev_status;
-    const int tiles = ceil_div(p.T, BM);
+    g.mode = GEMM_DENSE_UP; g.epi = EPI_STORE; g.E = pieces; g.n_per_expert = 3 * EP; g.k_per_expert = p.d / pieces;
+    g.a_expert_stride = p.d / pieces; g.rows = p.T;
+    g.out = sums; g.ld_out = (long long)pieces * 3 * EP; g.out_f32 = 1; g.dev_status = dev_status;
+    const int tiles = row_tiles * pieces;
     DSMOE_TRY(launch_gemm(*mA, *mB, g, tiles < sm_count() ? tiles : sm_count(), s, false));
-    router_finish_kernel<<<ceil_div(p.T, 8), 256, 0, s>>>(sums, br, scores, mask, k_t, p.T, EP,
+    router_finish_kernel<<<ceil_div(p.T, 8), 256, 0, s>>>(sums, br, scores, mask, k_t, p.T, EP, pieces,
                                                          SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k, nullptr});
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
