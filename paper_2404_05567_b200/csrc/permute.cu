@@ -8,7 +8,7 @@ namespace dsmoe {
 // Row indices.  A warp owns a chunk of 32 consecutive tokens; for expert e the ballot of "selected"
 // gives each token its rank inside the chunk, and chunk_prefix gives the number of earlier tokens,
 // so rows inside an expert segment ascend by token without any atomic.
-__global__ void __launch_bounds__(256) permute_index_kernel(const uint64_t* __restrict__ mask,
+__global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __restrict__ mask,
                                                             const float* __restrict__ scores,
                                                             const int32_t* __restrict__ offsets,
                                                             const int32_t* __restrict__ chunk_prefix,
@@ -16,19 +16,24 @@ __global__ void __launch_bounds__(256) permute_index_kernel(const uint64_t* __re
                                                             int32_t* __restrict__ token_rows, int T, int E, int W,
                                                             int64_t amax, uint4* __restrict__ zero_out, int row_vecs) {
     const int lane = threadIdx.x & 31;
-    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int c = blockIdx.x * 4 + (threadIdx.x >> 5);
     if (c * kChunk >= T) return;
     const int t = c * kChunk + lane;
     const uint64_t m = t < T ? mask[t] : 0;
+    // every load the loop below needs is issued before it: lane l holds the first row of this chunk in experts l and
+    // l + 32 (passed around by shuffles), and a token's scores are fetched right after its mask
+    const int base_lo = lane < E ? offsets[lane] + chunk_prefix[(size_t)c * E + lane] : 0;
+    const int base_hi = lane + 32 < E ? offsets[lane + 32] + chunk_prefix[(size_t)c * E + lane + 32] : 0;
     int slot = 0;
     for (int e = 0; e < E; ++e) {
         const bool bit = (m >> e) & 1;
         const unsigned b = __ballot_sync(0xffffffffu, bit);
+        const int base = __shfl_sync(0xffffffffu, e < 32 ? base_lo : base_hi, e & 31);
         if (bit) {
-            const int r = offsets[e] + chunk_prefix[(size_t)c * E + e] + __popc(b & ((1u << lane) - 1u));
+            const int r = base + __popc(b & ((1u << lane) - 1u));
             if (r >= 0 && r < amax) {   // inconsistent caller-supplied offsets must not become a wild store
                 row_token[r] = t;
-                row_gate[r] = scores[(size_t)t * E + e];
+                row_gate[r] = __ldg(scores + (size_t)t * E + e);
             }
             if (slot < W) token_rows[(size_t)t * W + slot] = r;
             ++slot;
@@ -192,7 +197,7 @@ dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const floa
     const int nchunks = ceil_div(p.T, kChunk);
     const int64_t amax = (int64_t)amax_of(p);
     const int row_vecs = (int)((size_t)p.d * (p.out_fp32 ? 4 : elem_size(p.dtype)) / 16);
-    permute_index_kernel<<<ceil_div(nchunks, 8), 256, 0, s>>>(mask, scores, offsets, chunk_prefix, row_token, row_gate,
+    permute_index_kernel<<<ceil_div(nchunks, 4), 128, 0, s>>>(mask, scores, offsets, chunk_prefix, row_token, row_gate,
                                                              token_rows, p.T, p.E, width_of(p), amax,
                                                              static_cast<uint4*>(zero_out), row_vecs);
     DSMOE_CUDA_TRY(cudaGetLastError());
