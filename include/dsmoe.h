@@ -303,8 +303,8 @@ dsmoe_status dsmoe_dense_backward(const dsmoe_layer_desc* desc, const void* x, c
  * the sequence of each token, or NULL (all 0); pos  device int32 [T], 0 <= pos[t] < L.
  * packed   device: dsmoe_pack_weights(desc, Wq, Wo, packed) with Wq [E][d][H], Wo [E][H][d].
  * x, Wr, br, out, mask_out, counts_out, workspace (dsmoe_workspace_size_packed(desc) bytes), dev_status: as for
- * dsmoe_layer_forward.  Supported: bf16, d and H multiples of 64, d_head a multiple of 32 up to 256, L up to
- * 12000; DSMOE_ERR_UNSUPPORTED otherwise.  A tok_seq or pos entry out of range is clamped and reported as
+ * dsmoe_layer_forward.  Supported: bf16, d and H multiples of 64, d_head 64, 96 or 128 (any L), or another
+ * multiple of 32 up to 256 with L up to 12000; DSMOE_ERR_UNSUPPORTED otherwise.  A tok_seq or pos entry out of range is clamped and reported as
  * DSMOE_ERR_INVALID_ARG in *dev_status.
  */
 typedef struct dsmoe_moa_args {

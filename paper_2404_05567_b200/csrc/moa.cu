@@ -383,7 +383,9 @@ dsmoe_status launch_mma_attention(const dsmoe_layer_desc& p, const MoaCore& c, _
 bool moa_supported(const dsmoe_layer_desc& p, int n_head, int L) {
     if (!umma_supported(p) || n_head <= 0 || p.H % n_head) return false;
     const int dh = p.H / n_head;
-    return dh % 32 == 0 && dh <= 256 && L > 0 && (size_t)(dh + L + 3) * 4 * kMoaWarps <= 200 * 1024;
+    if (L <= 0 || dh % 32 || dh > 256) return false;
+    if (dh == 64 || dh == 96 || dh == 128) return true;                       // tensor-core kernel: any cache length
+    return (size_t)(dh + L + 3) * 4 * kMoaWarps <= 200 * 1024;                // plain kernel: a warp's logits sit in shared memory
 }
 
 dsmoe_status launch_moa_attention(const dsmoe_layer_desc& p, const MoaCore& c, void* qa, const int32_t* row_token,
