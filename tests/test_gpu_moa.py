@@ -89,6 +89,8 @@ MOA = [
     ("moa_empty_rows", 260, 256, 16, 2, 64, 3, 50, "mixed", gi.MODE_THRESHOLD, dict(eps=0.3)),  # tokens that select nothing
     ("moa_wide_head", 200, 512, 4, 1, 256, 2, 90, "mixed", gi.MODE_TOPK, dict(K=2)),
     ("moa_ttk", 513, 256, 8, 4, 32, 4, 140, "mixed", gi.MODE_THRESHOLD_TOPK, dict(eps=0.03)),
+    ("moa_many_experts", 70, 256, 40, 2, 64, 2, 50, "mixed", gi.MODE_ALL, dict()),               # 40 rows per token: three row tiles
+    ("moa_many_experts_topk", 600, 256, 24, 2, 64, 3, 90, "mixed", gi.MODE_TOPK, dict(K=20)),      # 20 rows per token: two row tiles
     ("moa_full_cache", 300, 1024, 8, 4, 64, 6, 200, "full", gi.MODE_TOPK, dict(K=4)),
     ("moa_full_cache_6b", 64, 4096, 8, 4, 128, 8, 1000, "full", gi.MODE_TOPK, dict(K=5)),
 ]
