@@ -143,8 +143,13 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
     // keys, so their rows share the copies of K and V.
     // The CTAs are persistent (as many as fit the GPU at once) and walk the tiles: a tile is short, and starting a CTA per
     // tile cost more than the tile's work.
-    for (long long tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-    __syncthreads();                                    // the previous tile's merge has read shared memory
+    // With 8 warps (long caches, few tiles) the warps of a CTA share out the KEYS of one tile and merge their partial
+    // results at the end; with 2 warps (short caches, many tiles) each warp takes a tile of its OWN, walks all its
+    // keys and writes its result straight from registers: no merge, no CTA-wide barrier.
+    constexpr bool SPLIT = kMmaWarps > 2;
+    constexpr int TW = SPLIT ? 1 : kMmaWarps;           // tiles a CTA works on at a time
+    for (long long tile = (long long)blockIdx.x * TW + (SPLIT ? 0 : warp); tile < n_tiles; tile += (long long)gridDim.x * TW) {
+    if (SPLIT) __syncthreads();                         // the previous tile's merge has read shared memory
     const int rt = (int)(tile % row_tiles);
     const int j = (int)((tile / row_tiles) % n_head);
     const int t0 = (int)(tile / ((long long)row_tiles * n_head)) * tpt;
@@ -166,7 +171,7 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
     if (tk1 < T && sl1 < W) r1 = token_rows[(size_t)tk1 * W + sl1];
     if (r0 >= amax) r0 = -1;
     if (r1 >= amax) r1 = -1;
-    if (__syncthreads_or(r0 >= 0 || r1 >= 0) == 0) continue;        // no rows in this tile
+    if ((SPLIT ? __syncthreads_or(r0 >= 0 || r1 >= 0) : (int)__any_sync(0xffffffffu, r0 >= 0 || r1 >= 0)) == 0) continue;   // no rows in this tile
     bool bad = false;
     if (r0 >= 0) {
         last0 = pos[tk0];
@@ -211,7 +216,7 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
     const __nv_bfloat16* Kh = Kc + ((size_t)(sq * n_head + j) * L) * DH;
     const __nv_bfloat16* Vh = Vc + ((size_t)(sq * n_head + j) * L) * DH;
     const int nblocks = last / kKeyBlock + 1;
-    for (int b = warp; b < nblocks; b += kMmaWarps) {
+    for (int b = SPLIT ? warp : 0; b < nblocks; b += SPLIT ? kMmaWarps : 1) {
         const int key0 = b * kKeyBlock, nk = min(kKeyBlock, last + 1 - key0);
         __syncwarp();
 #pragma unroll
@@ -291,11 +296,22 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
         }
     }
     }
-    if (bad && threadIdx.x == 0) *dev_status = DSMOE_ERR_INVALID_ARG;      // clamped above: nothing left the cache
+    if (bad && lane == 0) *dev_status = DSMOE_ERR_INVALID_ARG;             // clamped above: nothing left the cache
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
     l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    if (!SPLIT) {
+        // the warp has seen every key of its rows: normalise and write (the queries it replaces are in its registers)
+        const float i0 = 1.f / l0, i1 = 1.f / l1;
+#pragma unroll
+        for (int dt = 0; dt < DT; ++dt) {
+            const int c = j * DH + dt * 8 + q4 * 2;
+            if (r0 >= 0) *reinterpret_cast<uint32_t*>(qa + (size_t)r0 * H + c) = pack_bf16(o[dt][0] * i0, o[dt][1] * i0);
+            if (r1 >= 0) *reinterpret_cast<uint32_t*>(qa + (size_t)r1 * H + c) = pack_bf16(o[dt][2] * i1, o[dt][3] * i1);
+        }
+        continue;
+    }
     // ---- merge the warps' partial results: per warp 16 maxima, 16 sums, 16 x DH accumulators
     __syncthreads();
     float* ms = reinterpret_cast<float*>(moa_mma_smem);                 // [warps][16]
@@ -364,7 +380,8 @@ dsmoe_status launch_mma_attention_nw(const dsmoe_layer_desc& p, const MoaCore& c
                                                                      32 * kMmaWarps, smem));
     const int per_sm = per_sm_of[dev];
     const long long resident = (long long)st->sm_count * (per_sm > 0 ? per_sm : 1);
-    const long long ctas = n_tiles < resident ? n_tiles : resident;
+    const long long want = kMmaWarps > 2 ? n_tiles : (n_tiles + kMmaWarps - 1) / kMmaWarps;     // 2 warps: a tile per warp
+    const long long ctas = want < resident ? want : resident;
     moa_attention_mma_kernel<DH, kMmaWarps><<<(unsigned)ctas, 32 * kMmaWarps, smem, s>>>(
         q, token_rows, W, row_tiles, tpt, (long long)amax_of(p), c.n_head, p.H, p.T, static_cast<const __nv_bfloat16*>(c.Kc),
         static_cast<const __nv_bfloat16*>(c.Vc), c.tok_seq, c.pos, c.n_seq, c.L, c.scale, n_tiles, dev_status);
