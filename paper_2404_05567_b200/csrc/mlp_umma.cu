@@ -1113,14 +1113,11 @@ __device__ __noinline__ void small_router_pass(const RouterArgs P, Shared& sh, i
     for (int i = 0; i < ntok; ++i) {
         const int tt = w + i * NW;
         float l_lo = b_lo, l_hi = b_hi;
-#pragma unroll 1
-        for (int sl = 0; sl < KS; ++sl) {
-            l_lo += vlo[0];
-            l_hi += vhi[0];
 #pragma unroll
-            for (int j = 0; j < 15; ++j) {      // the next slice sum moves to the front
-                vlo[j] = vlo[j + 1];
-                vhi[j] = vhi[j + 1];
+        for (int j = 0; j < 16; ++j) {          // this token's slice sums are v[i KS .. i KS + KS): added in ascending order
+            if ((j >> lg) == i) {
+                l_lo += vlo[j];
+                l_hi += vhi[j];
             }
         }
         float s_lo, s_hi;
