@@ -248,8 +248,11 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     // with the threshold rule, then the selection is redone with the batch's K
     dsmoe_layer_desc pr = p;
     if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK) pr.mode = DSMOE_SELECT_THRESHOLD;
+    // the tensor-core router leaves the per-chunk counts of its own selection behind (not Threshold-TopK's: that one
+    // selects again)
+    const bool counted = fast && router_umma_supported(p) && p.mode != DSMOE_SELECT_THRESHOLD_TOPK;
     if (fast && router_umma_supported(p))
-        DSMOE_TRY(launch_router_umma(pr, x, Wr, br, scores, mask, k_t, ws + L.router, dev_status, s));
+        DSMOE_TRY(launch_router_umma(pr, x, Wr, br, scores, mask, k_t, ws + L.router, dev_status, s, counted ? chunk_prefix : nullptr));
     else
         DSMOE_TRY(launch_router(pr, x, Wr, br, scores, mask, k_t, s));
     if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK)
@@ -261,23 +264,23 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     }
 
     // grouped path: duplicate tokens per selected expert, run the experts, aggregate
-    DSMOE_TRY(launch_finalize(p, mask, counts, offsets, chunk_prefix, counts_out, s));
     if (fast && fuses_combine(p)) {
         // no grouped copy of the tokens (the up-projection gathers rows of x by row_token), no buffer of expert
         // outputs and no aggregation pass: the down-projection's epilogue adds each expert's gate-weighted output
         // to the token's fp32 sum, in ascending expert order, and writes the final rounding
-        DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, nullptr, s, out));
+        DSMOE_TRY(launch_group(p, scores, mask, counts, offsets, chunk_prefix, counts_out, row_token, row_gate, token_rows, s, out, counted));
         const CombineArgs cmb{row_token, row_gate, mask, reinterpret_cast<float*>(ws + L.acc),
                               reinterpret_cast<int*>(ws + L.tile_done), out};
         return launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, nullptr, dev_status, s, x, row_token, &cmb);
     }
     if (fast) {
         // the down-projection's epilogue multiplies by the gate and stores fp32 rows; the aggregation only adds
-        DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, nullptr, s));
+        DSMOE_TRY(launch_group(p, scores, mask, counts, offsets, chunk_prefix, counts_out, row_token, row_gate, token_rows, s, nullptr, counted));
         const CombineArgs gated{row_token, row_gate, nullptr, nullptr, nullptr, nullptr};
         DSMOE_TRY(launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, ws + L.acc, dev_status, s, x, row_token, &gated));
         return launch_combine(p, ws + L.acc, nullptr, token_rows, k_t, out, s, true);
     }
+    DSMOE_TRY(launch_finalize(p, mask, counts, offsets, chunk_prefix, counts_out, s));
     DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, ws + L.xp, s));
     DSMOE_TRY(launch_mlp_generic(p, ws + L.xp, W1, W2, offsets, reinterpret_cast<float*>(ws + L.h_plain), ws + L.yp, s));
     return launch_combine(p, ws + L.yp, row_gate, token_rows, k_t, out, s);
@@ -367,20 +370,22 @@ dsmoe_status dsmoe_moa_forward(const dsmoe_layer_desc* desc, const dsmoe_moa_arg
     // router, selection and grouping as in dsmoe_layer_forward's grouped path (also when every expert is selected)
     dsmoe_layer_desc pr = p;
     if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK) pr.mode = DSMOE_SELECT_THRESHOLD;
+    // the tensor-core router leaves the per-chunk counts of its own selection behind (not Threshold-TopK's: that one
+    // selects again)
+    const bool counted = router_umma_supported(p) && p.mode != DSMOE_SELECT_THRESHOLD_TOPK;
     if (router_umma_supported(p))
-        DSMOE_TRY(launch_router_umma(pr, x, Wr, br, scores, mask, k_t, ws + L.router, dev_status, s));
+        DSMOE_TRY(launch_router_umma(pr, x, Wr, br, scores, mask, k_t, ws + L.router, dev_status, s, counted ? chunk_prefix : nullptr));
     else
         DSMOE_TRY(launch_router(pr, x, Wr, br, scores, mask, k_t, s));
     if (p.mode == DSMOE_SELECT_THRESHOLD_TOPK)
         DSMOE_TRY(launch_select(p, scores, mask, k_t, s, reinterpret_cast<int*>(ws + L.batch_k)));
-    DSMOE_TRY(launch_finalize(p, mask, counts, offsets, chunk_prefix, counts_out, s));
     if (fuses_combine(p)) {
-        DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, nullptr, s, out));
+        DSMOE_TRY(launch_group(p, scores, mask, counts, offsets, chunk_prefix, counts_out, row_token, row_gate, token_rows, s, out, counted));
         const CombineArgs cmb{row_token, row_gate, mask, reinterpret_cast<float*>(ws + L.acc),
                               reinterpret_cast<int*>(ws + L.tile_done), out};
         return launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, nullptr, dev_status, s, x, row_token, &cmb, &core);
     }
-    DSMOE_TRY(launch_permute(p, x, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, nullptr, s));
+    DSMOE_TRY(launch_group(p, scores, mask, counts, offsets, chunk_prefix, counts_out, row_token, row_gate, token_rows, s, nullptr, counted));
     const CombineArgs gated{row_token, row_gate, nullptr, nullptr, nullptr, nullptr};
     DSMOE_TRY(launch_mlp_umma(p, nullptr, packed, offsets, ws + L.h, ws + L.acc, dev_status, s, x, row_token, &gated, &core));
     return launch_combine(p, ws + L.acc, nullptr, token_rows, k_t, out, s, true);

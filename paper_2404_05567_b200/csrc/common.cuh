@@ -72,6 +72,11 @@ dsmoe_status launch_router(const dsmoe_layer_desc& p, const void* x, const float
 // k_scratch: one int of device memory, needed by DSMOE_SELECT_THRESHOLD_TOPK only (the batch's K)
 dsmoe_status launch_select(const dsmoe_layer_desc& p, const float* scores, uint64_t* mask, int32_t* k_t,
                            cudaStream_t s, int* k_scratch = nullptr);
+// launch_finalize = launch_chunk_counts (per chunk of 32 tokens, how many selected each expert) + launch_chunk_scan
+// (prefixes over the chunks, counts, offsets)
+dsmoe_status launch_chunk_counts(const dsmoe_layer_desc& p, const uint64_t* mask, int32_t* chunk_prefix, cudaStream_t s);
+dsmoe_status launch_chunk_scan(const dsmoe_layer_desc& p, int32_t* counts, int32_t* offsets, int32_t* chunk_prefix,
+                               int32_t* counts_out, cudaStream_t s);
 dsmoe_status launch_finalize(const dsmoe_layer_desc& p, const uint64_t* mask, int32_t* counts,
                              int32_t* offsets, int32_t* chunk_prefix, int32_t* counts_out, cudaStream_t s);
 
@@ -81,6 +86,11 @@ dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const floa
                             const uint64_t* mask, const int32_t* offsets, const int32_t* chunk_prefix,
                             int32_t* row_token, float* row_gate, int32_t* token_rows, void* xp,
                             cudaStream_t s, void* zero_out = nullptr);
+// Grouping for the fused layers: counts, offsets and the row indices of launch_finalize + launch_permute (without a
+// grouped copy of x).  chunk_counts_ready: chunk_prefix already holds the chunks' counts (the router wrote them).
+dsmoe_status launch_group(const dsmoe_layer_desc& p, const float* scores, const uint64_t* mask, int32_t* counts,
+                          int32_t* offsets, int32_t* chunk_prefix, int32_t* counts_out, int32_t* row_token,
+                          float* row_gate, int32_t* token_rows, cudaStream_t s, void* zero_out, bool chunk_counts_ready);
 // Selection statistics (see dsmoe_stats)
 dsmoe_status launch_stats(const dsmoe_layer_desc& p, const float* scores, const uint64_t* mask,
                           dsmoe_selection_stats* stats, cudaStream_t s);
@@ -115,7 +125,7 @@ bool router_umma_supported(const dsmoe_layer_desc& p);
 size_t router_umma_scratch(const dsmoe_layer_desc& p, size_t* split_bytes = nullptr);
 dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
                                 float* scores, uint64_t* mask, int32_t* k_t, char* scratch, int32_t* dev_status,
-                                cudaStream_t s);
+                                cudaStream_t s, int32_t* chunk_counts = nullptr);   // chunk_counts: see launch_group
 // Grouped expert MLPs on expert-sorted rows: h = GeLU(xp.W1[e]) (bf16, in `hbuf`), yp = h.W2[e].
 // With row_token (and x), the up-projection gathers its rows from x by index and xp is not read.
 // With cmb->out, the down-projection's epilogue also aggregates (Eq. 1's weighted sum, ascending expert order per

@@ -1953,23 +1953,44 @@ __global__ void __launch_bounds__(256) router_split_kernel(const float* __restri
 }
 
 // logits = (s1 + s2) + s3 + bias per expert, then softmax and selection: one warp per token
-// (the reduction over d may come in `pieces` blocks of 3 EP sums each, added in ascending order)
-__global__ void __launch_bounds__(256) router_finish_kernel(const float* __restrict__ sums, const float* __restrict__ br,
-                                                            float* __restrict__ scores, uint64_t* __restrict__ mask,
-                                                            int32_t* __restrict__ k_t, int T, int EP, int pieces, SelParams q) {
-    const int lane = threadIdx.x & 31;
-    const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (t >= T) return;
-    const float* row = sums + (size_t)t * 3 * EP * pieces;
-    const bool v_lo = lane < q.E, v_hi = lane + 32 < q.E;
-    float l_lo = 0.f, l_hi = 0.f;
-    for (int pc = 0; pc < pieces; ++pc, row += 3 * EP) {
-        if (v_lo) l_lo += (row[lane] + row[EP + lane]) + row[2 * EP + lane];
-        if (v_hi) l_hi += (row[lane + 32] + row[EP + lane + 32]) + row[2 * EP + lane + 32];
+// (the reduction over d may come in `pieces` blocks of 3 EP sums each, added in ascending order).  A block is one
+// chunk of 32 tokens; with chunk_counts its first warp then counts, per expert, the chunk's tokens that selected it
+// (what chunk_count_kernel would write to chunk_prefix[chunk,:]).
+__global__ void __launch_bounds__(32 * kChunk) router_finish_kernel(const float* __restrict__ sums, const float* __restrict__ br,
+                                                                    float* __restrict__ scores, uint64_t* __restrict__ mask,
+                                                                    int32_t* __restrict__ k_t, int32_t* __restrict__ chunk_counts,
+                                                                    int T, int EP, int pieces, SelParams q) {
+    __shared__ uint64_t mask_s[kChunk];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = blockIdx.x * kChunk + warp;
+    uint64_t m = 0;
+    if (t < T) {
+        const float* row = sums + (size_t)t * 3 * EP * pieces;
+        const bool v_lo = lane < q.E, v_hi = lane + 32 < q.E;
+        float l_lo = 0.f, l_hi = 0.f;
+        for (int pc = 0; pc < pieces; ++pc, row += 3 * EP) {
+            if (v_lo) l_lo += (row[lane] + row[EP + lane]) + row[2 * EP + lane];
+            if (v_hi) l_hi += (row[lane + 32] + row[EP + lane + 32]) + row[2 * EP + lane + 32];
+        }
+        if (v_lo && br) l_lo += br[lane];
+        if (v_hi && br) l_hi += br[lane + 32];
+        m = softmax_select_store(l_lo, l_hi, t, q, lane, scores, mask, k_t);
     }
-    if (v_lo && br) l_lo += br[lane];
-    if (v_hi && br) l_hi += br[lane + 32];
-    softmax_select_store(l_lo, l_hi, t, q, lane, scores, mask, k_t);
+    if (!chunk_counts) return;
+    if (lane == 0) mask_s[warp] = m;
+    __syncthreads();
+    if (warp == 0) {
+        const uint64_t mt = mask_s[lane];
+        int c_lo = 0, c_hi = 0;
+        for (int e = 0; e < q.E; ++e) {
+            const int n = __popc(__ballot_sync(0xffffffffu, (mt >> e) & 1));
+            if (lane == (e & 31)) {
+                if (e < 32) c_lo = n; else c_hi = n;
+            }
+        }
+        if (lane < q.E) chunk_counts[(size_t)blockIdx.x * q.E + lane] = c_lo;
+        if (lane + 32 < q.E) chunk_counts[(size_t)blockIdx.x * q.E + lane + 32] = c_hi;
+    }
 }
 
 }  // namespace
@@ -1989,7 +2010,7 @@ bool router_umma_supported(const dsmoe_layer_desc& p) { return umma_supported(p)
 
 dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const float* Wr, const float* br,
                                 float* scores, uint64_t* mask, int32_t* k_t, char* scratch, int32_t* dev_status,
-                                cudaStream_t s) {
+                                cudaStream_t s, int32_t* chunk_counts) {
     const int EP = p.E <= 32 ? 32 : 64;
     size_t split_bytes = 0;
     router_umma_scratch(p, &split_bytes);
@@ -2010,7 +2031,7 @@ dsmoe_status launch_router_umma(const dsmoe_layer_desc& p, const void* x, const 
     g.out = sums; g.ld_out = (long long)pieces * 3 * EP; g.out_f32 = 1; g.dev_status = dev_status;
     const int tiles = row_tiles * pieces;
     DSMOE_TRY(launch_gemm(*mA, *mB, g, tiles < sm_count() ? tiles : sm_count(), s, false));
-    router_finish_kernel<<<ceil_div(p.T, 8), 256, 0, s>>>(sums, br, scores, mask, k_t, p.T, EP, pieces,
+    router_finish_kernel<<<ceil_div(p.T, kChunk), 32 * kChunk, 0, s>>>(sums, br, scores, mask, k_t, chunk_counts, p.T, EP, pieces,
                                                          SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k, nullptr});
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;

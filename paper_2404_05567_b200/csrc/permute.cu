@@ -8,22 +8,110 @@ namespace dsmoe {
 // Row indices.  A warp owns a chunk of 32 consecutive tokens; for expert e the ballot of "selected"
 // gives each token its rank inside the chunk, and chunk_prefix gives the number of earlier tokens,
 // so rows inside an expert segment ascend by token without any atomic.
+// SCAN: chunk_prefix holds the chunks' own counts (chunk_count_kernel's output, not yet the prefixes over the
+// chunks): every block adds up the chunks before its own and all chunks itself -- a few thousand integers out of
+// L2 -- instead of waiting for a one-block scan kernel in between; block 0 writes counts, offsets (and counts_out).
+// The integers are the same either way.
+template <bool SCAN>
 __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __restrict__ mask,
                                                             const float* __restrict__ scores,
-                                                            const int32_t* __restrict__ offsets,
+                                                            int32_t* __restrict__ offsets,
                                                             const int32_t* __restrict__ chunk_prefix,
+                                                            int32_t* __restrict__ counts, int32_t* __restrict__ counts_out,
                                                             int32_t* __restrict__ row_token, float* __restrict__ row_gate,
                                                             int32_t* __restrict__ token_rows, int T, int E, int W,
                                                             int64_t amax, uint4* __restrict__ zero_out, int row_vecs) {
-    const int lane = threadIdx.x & 31;
-    const int c = blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (c * kChunk >= T) return;
+    // a chunk's scores, staged so that the loop over the experts below waits for no load: [token][E + 1]
+    __shared__ float sc_s[4][kChunk * (kMaxExperts + 1)];
+    __shared__ int before_s[4][kMaxExperts], total_s[4][kMaxExperts], base_s[4][kMaxExperts];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c0 = blockIdx.x * 4, c = c0 + warp;
+    const int nchunks = (T + kChunk - 1) / kChunk;
+    const bool live = c < nchunks;
     const int t = c * kChunk + lane;
-    const uint64_t m = t < T ? mask[t] : 0;
-    // every load the loop below needs is issued before it: lane l holds the first row of this chunk in experts l and
-    // l + 32 (passed around by shuffles), and a token's scores are fetched right after its mask
-    const int base_lo = lane < E ? offsets[lane] + chunk_prefix[(size_t)c * E + lane] : 0;
-    const int base_hi = lane + 32 < E ? offsets[lane + 32] + chunk_prefix[(size_t)c * E + lane + 32] : 0;
+    const uint64_t m = live && t < T ? mask[t] : 0;
+    if (live) {
+        float* sc = sc_s[warp];
+        const float* src = scores + (size_t)c * kChunk * E;
+        const int n = min(kChunk, T - c * kChunk) * E;
+        for (int i = lane; i < n; i += 32) sc[(i / E) * (E + 1) + i % E] = __ldg(src + i);
+    }
+    if (SCAN) {
+        // thread (e, part) adds every `parts`-th chunk's count of expert e: coalesced rows of E integers
+        const int EP = E <= 32 ? 32 : 64, parts = 128 / EP;
+        const int e = threadIdx.x % EP, part = threadIdx.x / EP;
+        int before = 0, total = 0;
+        if (e < E) {
+            for (int k = part; k < nchunks; k += parts) {
+                const int v = chunk_prefix[(size_t)k * E + e];
+                total += v;
+                if (k < c0) before += v;
+            }
+        }
+        before_s[part][e] = before;
+        total_s[part][e] = total;
+        __syncthreads();
+        if (warp == 0) {
+            int b_lo = 0, b_hi = 0, c_lo = 0, c_hi = 0;
+            for (int k = 0; k < parts; ++k) {
+                b_lo += before_s[k][lane];
+                c_lo += total_s[k][lane];
+                if (EP == 64) {
+                    b_hi += before_s[k][lane + 32];
+                    c_hi += total_s[k][lane + 32];
+                }
+            }
+            if (lane >= E) c_lo = 0;
+            if (lane + 32 >= E) c_hi = 0;
+            int i_lo = c_lo, i_hi = c_hi;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int a = __shfl_up_sync(0xffffffffu, i_lo, o);
+                const int b = __shfl_up_sync(0xffffffffu, i_hi, o);
+                if (lane >= o) {
+                    i_lo += a;
+                    i_hi += b;
+                }
+            }
+            const int tot_lo = __shfl_sync(0xffffffffu, i_lo, 31);
+            const int tot = tot_lo + __shfl_sync(0xffffffffu, i_hi, 31);
+            int run_lo = i_lo - c_lo + b_lo, run_hi = tot_lo + i_hi - c_hi + b_hi;   // first row of chunk c0 in the expert
+            for (int w = 0; w < 4; ++w) {
+                base_s[w][lane] = run_lo;
+                base_s[w][lane + 32] = run_hi;
+                if (c0 + w < nchunks) {
+                    if (lane < E) run_lo += chunk_prefix[(size_t)(c0 + w) * E + lane];
+                    if (lane + 32 < E) run_hi += chunk_prefix[(size_t)(c0 + w) * E + lane + 32];
+                }
+            }
+            if (blockIdx.x == 0) {
+                if (lane < E) {
+                    counts[lane] = c_lo;
+                    offsets[lane] = i_lo - c_lo;
+                    if (counts_out) counts_out[lane] = c_lo;
+                }
+                if (lane + 32 < E) {
+                    counts[lane + 32] = c_hi;
+                    offsets[lane + 32] = tot_lo + i_hi - c_hi;
+                    if (counts_out) counts_out[lane + 32] = c_hi;
+                }
+                if (lane == 0) offsets[E] = tot;
+            }
+        }
+        __syncthreads();
+    }
+    if (!live) return;
+    __syncwarp();
+    // lane l holds the first row of this chunk in experts l and l + 32 (passed around by shuffles)
+    int base_lo, base_hi;
+    if (SCAN) {
+        base_lo = base_s[warp][lane];
+        base_hi = base_s[warp][lane + 32];
+    } else {
+        base_lo = lane < E ? offsets[lane] + chunk_prefix[(size_t)c * E + lane] : 0;
+        base_hi = lane + 32 < E ? offsets[lane + 32] + chunk_prefix[(size_t)c * E + lane + 32] : 0;
+    }
+    const float* my = sc_s[warp] + lane * (E + 1);
     int slot = 0;
     for (int e = 0; e < E; ++e) {
         const bool bit = (m >> e) & 1;
@@ -33,7 +121,7 @@ __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __re
             const int r = base + __popc(b & ((1u << lane) - 1u));
             if (r >= 0 && r < amax) {   // inconsistent caller-supplied offsets must not become a wild store
                 row_token[r] = t;
-                row_gate[r] = __ldg(scores + (size_t)t * E + e);
+                row_gate[r] = my[e];
             }
             if (slot < W) token_rows[(size_t)t * W + slot] = r;
             ++slot;
@@ -197,9 +285,10 @@ dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const floa
     const int nchunks = ceil_div(p.T, kChunk);
     const int64_t amax = (int64_t)amax_of(p);
     const int row_vecs = (int)((size_t)p.d * (p.out_fp32 ? 4 : elem_size(p.dtype)) / 16);
-    permute_index_kernel<<<ceil_div(nchunks, 4), 128, 0, s>>>(mask, scores, offsets, chunk_prefix, row_token, row_gate,
-                                                             token_rows, p.T, p.E, width_of(p), amax,
-                                                             static_cast<uint4*>(zero_out), row_vecs);
+    permute_index_kernel<false><<<ceil_div(nchunks, 4), 128, 0, s>>>(mask, scores, const_cast<int32_t*>(offsets), chunk_prefix,
+                                                                    nullptr, nullptr, row_token, row_gate, token_rows, p.T,
+                                                                    p.E, width_of(p), amax, static_cast<uint4*>(zero_out),
+                                                                    row_vecs);
     DSMOE_CUDA_TRY(cudaGetLastError());
     if (xp) {
         const int vec_per_row = (int)((size_t)p.d * elem_size(p.dtype) / 16);
@@ -208,6 +297,28 @@ dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const floa
                                                 static_cast<uint4*>(xp), p.E, p.T, vec_per_row, amax);
         DSMOE_CUDA_TRY(cudaGetLastError());
     }
+    return DSMOE_OK;
+}
+
+// Up to this many chunks every block of permute_index_kernel adds up the chunks' counts itself (no scan kernel)
+constexpr int kScanInBlockChunks = 512;
+
+dsmoe_status launch_group(const dsmoe_layer_desc& p, const float* scores, const uint64_t* mask, int32_t* counts,
+                          int32_t* offsets, int32_t* chunk_prefix, int32_t* counts_out, int32_t* row_token,
+                          float* row_gate, int32_t* token_rows, cudaStream_t s, void* zero_out, bool chunk_counts_ready) {
+    if (!chunk_counts_ready) DSMOE_TRY(launch_chunk_counts(p, mask, chunk_prefix, s));
+    const int nchunks = ceil_div(p.T, kChunk);
+    if (nchunks == 0 || nchunks > kScanInBlockChunks) {
+        DSMOE_TRY(launch_chunk_scan(p, counts, offsets, chunk_prefix, counts_out, s));
+        return launch_permute(p, nullptr, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, nullptr, s,
+                              zero_out);
+    }
+    const int row_vecs = (int)((size_t)p.d * (p.out_fp32 ? 4 : elem_size(p.dtype)) / 16);
+    permute_index_kernel<true><<<ceil_div(nchunks, 4), 128, 0, s>>>(mask, scores, offsets, chunk_prefix, counts, counts_out,
+                                                                   row_token, row_gate, token_rows, p.T, p.E, width_of(p),
+                                                                   (int64_t)amax_of(p), static_cast<uint4*>(zero_out),
+                                                                   row_vecs);
+    DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
 }
 

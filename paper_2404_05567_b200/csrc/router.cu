@@ -405,16 +405,26 @@ dsmoe_status launch_select(const dsmoe_layer_desc& p, const float* scores, uint6
     return DSMOE_OK;
 }
 
-dsmoe_status launch_finalize(const dsmoe_layer_desc& p, const uint64_t* mask, int32_t* counts, int32_t* offsets,
-                             int32_t* chunk_prefix, int32_t* counts_out, cudaStream_t s) {
+dsmoe_status launch_chunk_counts(const dsmoe_layer_desc& p, const uint64_t* mask, int32_t* chunk_prefix, cudaStream_t s) {
     const int nchunks = ceil_div(p.T, kChunk);
     if (nchunks > 0) {
         chunk_count_kernel<<<ceil_div(nchunks, 8), 256, 0, s>>>(mask, chunk_prefix, p.T, p.E);
         DSMOE_CUDA_TRY(cudaGetLastError());
     }
+    return DSMOE_OK;
+}
+
+dsmoe_status launch_chunk_scan(const dsmoe_layer_desc& p, int32_t* counts, int32_t* offsets, int32_t* chunk_prefix,
+                               int32_t* counts_out, cudaStream_t s) {
     finalize_kernel<<<1, 1024, 0, s>>>(counts, offsets, chunk_prefix, counts_out, p.T, p.E);
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
+}
+
+dsmoe_status launch_finalize(const dsmoe_layer_desc& p, const uint64_t* mask, int32_t* counts, int32_t* offsets,
+                             int32_t* chunk_prefix, int32_t* counts_out, cudaStream_t s) {
+    DSMOE_TRY(launch_chunk_counts(p, mask, chunk_prefix, s));
+    return launch_chunk_scan(p, counts, offsets, chunk_prefix, counts_out, s);
 }
 
 }  // namespace dsmoe

@@ -88,10 +88,11 @@ __device__ __forceinline__ void softmax_warp(float l_lo, float l_hi, int E, int 
     s_hi = __fdiv_rn(p_hi, den);
 }
 
-// Softmax, then selection; the warp writes scores[t,:], mask[t], k_t[t] (each optional).
-__device__ __forceinline__ void softmax_select_store(float l_lo, float l_hi, int t, const SelParams& q, int lane,
-                                                     float* __restrict__ scores, uint64_t* __restrict__ mask,
-                                                     int32_t* __restrict__ k_t) {
+// Softmax, then selection; the warp writes scores[t,:], mask[t], k_t[t] (each optional) and returns the selection word
+// (0 where neither mask nor k_t is asked for).
+__device__ __forceinline__ uint64_t softmax_select_store(float l_lo, float l_hi, int t, const SelParams& q, int lane,
+                                                         float* __restrict__ scores, uint64_t* __restrict__ mask,
+                                                         int32_t* __restrict__ k_t) {
     const bool v_lo = lane < q.E, v_hi = lane + 32 < q.E;
     float s_lo, s_hi;
     softmax_warp(l_lo, l_hi, q.E, lane, s_lo, s_hi);
@@ -99,13 +100,15 @@ __device__ __forceinline__ void softmax_select_store(float l_lo, float l_hi, int
         if (v_lo) scores[(size_t)t * q.E + lane] = s_lo;
         if (v_hi) scores[(size_t)t * q.E + lane + 32] = s_hi;
     }
+    uint64_t m = 0;
     if (mask || k_t) {
-        const uint64_t m = select_warp(s_lo, s_hi, q, lane);
+        m = select_warp(s_lo, s_hi, q, lane);
         if (lane == 0) {
             if (mask) mask[t] = m;
             if (k_t) k_t[t] = __popcll(m);
         }
     }
+    return m;
 }
 
 }  // namespace dsmoe
