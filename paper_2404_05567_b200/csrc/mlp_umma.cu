@@ -14,6 +14,7 @@
 //   DENSE_DOWN  out[t,:] = sum over (e,j) of that h times W2[e][j,:] -- the router-weighted sum of
 //               Eq. 1 folded into the reduction dimension, so no grouping and no aggregation pass
 // small_layer_kernel: the whole layer for a handful of tokens (decode) in one cooperative launch.
+#include <algorithm>
 #include <climits>
 #include <cstdlib>
 
@@ -124,11 +125,15 @@ struct GemmParams {
     // GEMM_DENSE_UP: "expert" e reads A's columns from e * a_expert_stride on (0: every expert reads the same columns;
     // the router's logits use it to cut their reduction into pieces with an output block each)
     int a_expert_stride;
+    // GEMM_GROUPED, EPI_STORE with out_f32, single CTAs: the reduction is cut into k_splits equal runs of 64-wide blocks
+    // (0 or 1: not cut); split s of a tile stores its partial sums to rows split_rows * s + r of `out`
+    int k_splits, split_rows;
 };
 
 struct Tile {
     int row0, rows_valid, e, n0, bn, nk, out_col0;   // rows_valid <= 0: this CTA's half of a pair's tile lies past the rows
     int row_safe;                                    // a row that exists (stands in for rows past the end)
+    int k0, out_row0;                                // first 64-wide block of the reduction; row of `out` that row0 goes to
 };
 
 // small_layer_kernel: the selected experts and the work partition and ring geometry that follow from them
@@ -238,7 +243,7 @@ template <bool PAIR>
 __device__ __forceinline__ int total_tiles(const GemmParams& P, const Shared& sh) {
     constexpr int MT = Geo<PAIR>::MT;
     const int ntn = (P.n_per_expert + BN - 1) / BN;
-    if (P.mode == GEMM_GROUPED) return sh.tile_prefix[P.E];
+    if (P.mode == GEMM_GROUPED) return sh.tile_prefix[P.E] * max(P.k_splits, 1);
     const int mt = (P.rows + MT - 1) / MT;
     return P.mode == GEMM_DENSE_UP ? mt * ntn * P.E : mt * ntn;
 }
@@ -249,7 +254,10 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& P, const Shared& s
     constexpr int MT = Geo<PAIR>::MT;
     Tile t;
     const int kbpe = P.k_per_expert / BK;
+    t.k0 = 0;
     if (P.mode == GEMM_GROUPED) {
+        const int splits = max(P.k_splits, 1), split = id % splits;
+        id /= splits;
         int e = 0;
         while (e + 1 < P.E && id >= sh.tile_prefix[e + 1]) ++e;
         const int local = id - sh.tile_prefix[e];
@@ -261,8 +269,10 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& P, const Shared& s
         t.rows_valid = min(BM, sh.seg1[e] - t.row0);
         t.row_safe = sh.seg0[e];
         t.n0 = nt * BN;
-        t.nk = kbpe;
+        t.nk = kbpe / splits;
+        t.k0 = split * t.nk;
         t.out_col0 = t.n0;
+        t.out_row0 = t.row0 + split * P.split_rows;
     } else {
         const int mtiles = (P.rows + MT - 1) / MT;
         const int ntn = (P.n_per_expert + BN - 1) / BN;
@@ -287,6 +297,7 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& P, const Shared& s
             rest = rem / bm;
         }
         t.row0 = mt * MT + half * BM;
+        t.out_row0 = t.row0;
         t.rows_valid = min(BM, P.rows - t.row0);
         t.row_safe = 0;
         if (P.mode == GEMM_DENSE_UP) {
@@ -434,7 +445,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         a_col = b_e * P.k_per_expert + b_k;
                     } else {
                         b_e = t.e;
-                        b_k = i * BK;
+                        b_k = (t.k0 + i) * BK;
                         a_col = t.e * P.a_expert_stride + b_k;
                     }
                     if (!P.gather) {
@@ -587,7 +598,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     break;
                 }
                 const uint32_t dst0 = smA + s * A_STAGE_BYTES;
-                const char* src0 = static_cast<const char*>(P.gather_src) + (size_t)i * (BK * 2) + lc * 16;
+                const char* src0 = static_cast<const char*>(P.gather_src) + (size_t)(t.k0 + i) * (BK * 2) + lc * 16;
 #pragma unroll
                 for (int jj = 0; jj < ROWS / 4; ++jj) {
                     const int rl = jj * 4 + lr, r = part * ROWS + rl;
@@ -823,7 +834,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     for (int i = 0; i < 8; ++i) {
                         const int rl = i * 4 + rr;      // row of this warp's 32
                         if (q * 32 + rl < t.rows_valid)
-                            *reinterpret_cast<float4*>(out_f + ((long long)t.row0 + q * 32 + rl) * P.ld_out + t.out_col0 + c + cc * 4) =
+                            *reinterpret_cast<float4*>(out_f + ((long long)t.out_row0 + q * 32 + rl) * P.ld_out + t.out_col0 + c + cc * 4) =
                                 *reinterpret_cast<const float4*>(tp + rl * LD + cc * 4);
                     }
                     __syncwarp();
@@ -1993,6 +2004,29 @@ __global__ void __launch_bounds__(32 * kChunk) router_finish_kernel(const float*
     }
 }
 
+// out[r,:] (bf16) = the sum over the splits, in ascending order, of the fp32 partial rows part[s * split_rows + r,:]
+// that a launch with k_splits left behind; rows from offsets[E] on do not exist
+__global__ void __launch_bounds__(256) split_sum_kernel(const float4* __restrict__ part, int splits, int split_rows,
+                                                        const int32_t* __restrict__ offsets, int E, int n,
+                                                        __nv_bfloat16* __restrict__ out) {
+    const int nvec = n / 4;
+    const long long rows = min(max(offsets[E], 0), split_rows);
+    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < rows * nvec; i += (long long)gridDim.x * 256) {
+        float4 a = part[i];
+        for (int sp = 1; sp < splits; ++sp) {
+            const float4 b = part[(long long)sp * split_rows * nvec + i];
+            a.x += b.x;
+            a.y += b.y;
+            a.z += b.z;
+            a.w += b.w;
+        }
+        uint2 pk;
+        *reinterpret_cast<__nv_bfloat162*>(&pk.x) = __floats2bfloat162_rn(a.x, a.y);
+        *reinterpret_cast<__nv_bfloat162*>(&pk.y) = __floats2bfloat162_rn(a.z, a.w);
+        reinterpret_cast<uint2*>(out)[i] = pk;
+    }
+}
+
 }  // namespace
 
 // With few row tiles the logits' reduction over d is cut into 2 or 4 pieces, each a tile with its own block of sums,
@@ -2096,7 +2130,27 @@ dsmoe_status launch_mlp_umma(const dsmoe_layer_desc& p, const void* xp, const vo
     // top-K selection alone (an upper bound otherwise), so only there may the launches pair on their own
     const long long known = p.mode == DSMOE_SELECT_TOPK ? (long long)p.T * (p.K < p.E ? p.K : p.E) : 0;
     const int pair_tiles = known >= 1024ll * p.E ? INT_MAX : (pair_override() == 1 ? INT_MAX : 0);
-    DSMOE_TRY(launch_gemm(*mA1, *mB1, up, sm_count(), s, true, moa ? 0 : pair_tiles));
+    // Few rows and a long reduction (the query projection at decode sizes: a handful of tiles, each a chain of d / 64
+    // reduction blocks): the reduction is cut so that the launch covers the SMs; the partial sums (fp32, in the buffer
+    // of the expert outputs, which is idle until the output projection) are added in order by split_sum_kernel
+    int splits = 1;
+    if (moa && yp && cmb && !cmb->out) {
+        const long long max_tiles = ((long long)(amax / BM) + p.E) * ceil_div(p.H, BN);
+        while (splits < 8 && max_tiles * splits * 2 <= sm_count() && (p.d / BK) % (splits * 2) == 0 &&
+               (p.d / BK) / (splits * 2) >= 4 && (long long)splits * 2 * p.H <= p.d)
+            splits *= 2;
+    }
+    if (splits > 1) {
+        up.k_splits = splits; up.split_rows = (int)amax;
+        up.out = yp; up.out_f32 = 1;
+        DSMOE_TRY(launch_gemm(*mA1, *mB1, up, sm_count(), s, true, 0));
+        const long long vecs = (long long)amax * p.H / 4;
+        split_sum_kernel<<<(int)std::min<long long>((vecs + 255) / 256, 8ll * sm_count()), 256, 0, s>>>(
+            static_cast<const float4*>(yp), splits, (int)amax, offsets, p.E, p.H, static_cast<__nv_bfloat16*>(hbuf));
+        DSMOE_CUDA_TRY(cudaGetLastError());
+    } else {
+        DSMOE_TRY(launch_gemm(*mA1, *mB1, up, sm_count(), s, true, moa ? 0 : pair_tiles));
+    }
     if (moa) DSMOE_TRY(launch_moa_attention(p, *moa, hbuf, row_token, moa->token_rows, offsets, dev_status, s));
     DSMOE_TRY(launch_gemm(*mA2, *mB2, down, sm_count(), s, true, pair_tiles));
     return DSMOE_OK;

@@ -1,6 +1,8 @@
 // Grouping of tokens by expert and the router-weighted aggregation back into token order -- the
 // "duplication of intermediate tokens and the aggregation of outputs" that the paper's GPU
 // Inference Analysis names as the overhead of sparse inference -- plus the one-off weight packer.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace dsmoe {
@@ -8,11 +10,13 @@ namespace dsmoe {
 // Row indices.  A warp owns a chunk of 32 consecutive tokens; for expert e the ballot of "selected"
 // gives each token its rank inside the chunk, and chunk_prefix gives the number of earlier tokens,
 // so rows inside an expert segment ascend by token without any atomic.
-// SCAN: chunk_prefix holds the chunks' own counts (chunk_count_kernel's output, not yet the prefixes over the
+// SCAN 1: chunk_prefix holds the chunks' own counts (chunk_count_kernel's output, not yet the prefixes over the
 // chunks): every block adds up the chunks before its own and all chunks itself -- a few thousand integers out of
 // L2 -- instead of waiting for a one-block scan kernel in between; block 0 writes counts, offsets (and counts_out).
+// SCAN 2 (at most kCountInBlockChunks chunks): every block also counts the chunks itself, from the masks.
 // The integers are the same either way.
-template <bool SCAN>
+constexpr int kCountInBlockChunks = 8;
+template <int SCAN>
 __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __restrict__ mask,
                                                             const float* __restrict__ scores,
                                                             int32_t* __restrict__ offsets,
@@ -36,6 +40,24 @@ __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __re
         const int n = min(kChunk, T - c * kChunk) * E;
         for (int i = lane; i < n; i += 32) sc[(i / E) * (E + 1) + i % E] = __ldg(src + i);
     }
+    __shared__ int cnt_s[SCAN == 2 ? kCountInBlockChunks : 1][kMaxExperts];
+    if (SCAN == 2) {
+        for (int k = warp; k < nchunks; k += 4) {
+            const int tk = k * kChunk + lane;
+            const uint64_t mk = tk < T ? mask[tk] : 0;
+            int n_lo = 0, n_hi = 0;
+            for (int e = 0; e < E; ++e) {
+                const int n = __popc(__ballot_sync(0xffffffffu, (mk >> e) & 1));
+                if (lane == (e & 31)) {
+                    if (e < 32) n_lo = n; else n_hi = n;
+                }
+            }
+            cnt_s[k][lane] = n_lo;
+            cnt_s[k][lane + 32] = n_hi;
+        }
+        __syncthreads();
+    }
+    const auto chunk_count = [&](int k, int e) { return SCAN == 2 ? cnt_s[k][e] : chunk_prefix[(size_t)k * E + e]; };
     if (SCAN) {
         // thread (e, part) adds every `parts`-th chunk's count of expert e: coalesced rows of E integers
         const int EP = E <= 32 ? 32 : 64, parts = 128 / EP;
@@ -43,7 +65,7 @@ __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __re
         int before = 0, total = 0;
         if (e < E) {
             for (int k = part; k < nchunks; k += parts) {
-                const int v = chunk_prefix[(size_t)k * E + e];
+                const int v = chunk_count(k, e);
                 total += v;
                 if (k < c0) before += v;
             }
@@ -80,8 +102,8 @@ __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __re
                 base_s[w][lane] = run_lo;
                 base_s[w][lane + 32] = run_hi;
                 if (c0 + w < nchunks) {
-                    if (lane < E) run_lo += chunk_prefix[(size_t)(c0 + w) * E + lane];
-                    if (lane + 32 < E) run_hi += chunk_prefix[(size_t)(c0 + w) * E + lane + 32];
+                    if (lane < E) run_lo += chunk_count(c0 + w, lane);
+                    if (lane + 32 < E) run_hi += chunk_count(c0 + w, lane + 32);
                 }
             }
             if (blockIdx.x == 0) {
@@ -185,7 +207,7 @@ __global__ void __launch_bounds__(128) combine_bf16_kernel(const uint4* __restri
     }
     __syncthreads();
     const int nvec = d / 8;
-    for (int v = threadIdx.x; v < nvec; v += 128) {
+    for (int v = blockIdx.y * 128 + threadIdx.x; v < nvec; v += 128 * gridDim.y) {
         float acc[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = 0.f;
@@ -231,7 +253,7 @@ __global__ void __launch_bounds__(128) combine_f32_kernel(const float4* __restri
     }
     __syncthreads();
     const int nvec = d / 4;
-    for (int v = threadIdx.x; v < nvec; v += 128) {
+    for (int v = blockIdx.y * 128 + threadIdx.x; v < nvec; v += 128 * gridDim.y) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         // four rows' loads are issued before their first use (past the k-th row, row 0 is fetched again and not used)
         for (int i = 0; i < k; i += 4) {
@@ -285,7 +307,7 @@ dsmoe_status launch_permute(const dsmoe_layer_desc& p, const void* x, const floa
     const int nchunks = ceil_div(p.T, kChunk);
     const int64_t amax = (int64_t)amax_of(p);
     const int row_vecs = (int)((size_t)p.d * (p.out_fp32 ? 4 : elem_size(p.dtype)) / 16);
-    permute_index_kernel<false><<<ceil_div(nchunks, 4), 128, 0, s>>>(mask, scores, const_cast<int32_t*>(offsets), chunk_prefix,
+    permute_index_kernel<0><<<ceil_div(nchunks, 4), 128, 0, s>>>(mask, scores, const_cast<int32_t*>(offsets), chunk_prefix,
                                                                     nullptr, nullptr, row_token, row_gate, token_rows, p.T,
                                                                     p.E, width_of(p), amax, static_cast<uint4*>(zero_out),
                                                                     row_vecs);
@@ -306,15 +328,23 @@ constexpr int kScanInBlockChunks = 512;
 dsmoe_status launch_group(const dsmoe_layer_desc& p, const float* scores, const uint64_t* mask, int32_t* counts,
                           int32_t* offsets, int32_t* chunk_prefix, int32_t* counts_out, int32_t* row_token,
                           float* row_gate, int32_t* token_rows, cudaStream_t s, void* zero_out, bool chunk_counts_ready) {
-    if (!chunk_counts_ready) DSMOE_TRY(launch_chunk_counts(p, mask, chunk_prefix, s));
     const int nchunks = ceil_div(p.T, kChunk);
+    const int row_vecs = (int)((size_t)p.d * (p.out_fp32 ? 4 : elem_size(p.dtype)) / 16);
+    if (nchunks > 0 && nchunks <= kCountInBlockChunks) {
+        permute_index_kernel<2><<<ceil_div(nchunks, 4), 128, 0, s>>>(mask, scores, offsets, nullptr, counts, counts_out,
+                                                                    row_token, row_gate, token_rows, p.T, p.E, width_of(p),
+                                                                    (int64_t)amax_of(p), static_cast<uint4*>(zero_out),
+                                                                    row_vecs);
+        DSMOE_CUDA_TRY(cudaGetLastError());
+        return DSMOE_OK;
+    }
+    if (!chunk_counts_ready) DSMOE_TRY(launch_chunk_counts(p, mask, chunk_prefix, s));
     if (nchunks == 0 || nchunks > kScanInBlockChunks) {
         DSMOE_TRY(launch_chunk_scan(p, counts, offsets, chunk_prefix, counts_out, s));
         return launch_permute(p, nullptr, scores, mask, offsets, chunk_prefix, row_token, row_gate, token_rows, nullptr, s,
                               zero_out);
     }
-    const int row_vecs = (int)((size_t)p.d * (p.out_fp32 ? 4 : elem_size(p.dtype)) / 16);
-    permute_index_kernel<true><<<ceil_div(nchunks, 4), 128, 0, s>>>(mask, scores, offsets, chunk_prefix, counts, counts_out,
+    permute_index_kernel<1><<<ceil_div(nchunks, 4), 128, 0, s>>>(mask, scores, offsets, chunk_prefix, counts, counts_out,
                                                                    row_token, row_gate, token_rows, p.T, p.E, width_of(p),
                                                                    (int64_t)amax_of(p), static_cast<uint4*>(zero_out),
                                                                    row_vecs);
@@ -327,19 +357,22 @@ dsmoe_status launch_combine(const dsmoe_layer_desc& p, const void* yp, const flo
     if (p.T == 0) return DSMOE_OK;
     const int W = width_of(p);
     const int64_t amax = (int64_t)amax_of(p);
+    // with few tokens a row's columns are shared out over several blocks (blockIdx.y), enough to cover the SMs
+    const int col_blocks = ceil_div(p.d / (yp_f32 || p.dtype != DSMOE_BF16 ? 4 : 8), 128);
+    const dim3 grid(p.T, (unsigned)(std::max(1, std::min(col_blocks, 1024 / p.T))));
     if (yp_f32 && p.dtype == DSMOE_BF16 && !p.out_fp32) {
-        combine_f32_kernel<true><<<p.T, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t, out, p.d, W, amax);
+        combine_f32_kernel<true><<<grid, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t, out, p.d, W, amax);
     } else if (yp_f32) {
-        combine_f32_kernel<false><<<p.T, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t, out, p.d, W, amax);
+        combine_f32_kernel<false><<<grid, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t, out, p.d, W, amax);
     } else if (p.dtype == DSMOE_BF16) {
         if (p.out_fp32)
-            combine_bf16_kernel<true><<<p.T, 128, 0, s>>>(static_cast<const uint4*>(yp), row_gate, token_rows, k_t, out,
+            combine_bf16_kernel<true><<<grid, 128, 0, s>>>(static_cast<const uint4*>(yp), row_gate, token_rows, k_t, out,
                                                          p.d, W, amax);
         else
-            combine_bf16_kernel<false><<<p.T, 128, 0, s>>>(static_cast<const uint4*>(yp), row_gate, token_rows, k_t, out,
+            combine_bf16_kernel<false><<<grid, 128, 0, s>>>(static_cast<const uint4*>(yp), row_gate, token_rows, k_t, out,
                                                           p.d, W, amax);
     } else {
-        combine_f32_kernel<false><<<p.T, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t, out, p.d, W, amax);
+        combine_f32_kernel<false><<<grid, 128, 0, s>>>(static_cast<const float4*>(yp), row_gate, token_rows, k_t, out, p.d, W, amax);
     }
     DSMOE_CUDA_TRY(cudaGetLastError());
     return DSMOE_OK;
