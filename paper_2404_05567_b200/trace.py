@@ -55,6 +55,9 @@ def gemm_waits(a):
     if a.gemm == "dense":
         T, d, H, E = 16384, 2048, 1024, 32
         desc = dm.make_desc(T, d, H, E, dm.BF16, dm.SELECT_ALL)
+    elif a.gemm == "paper6b":      # the paper's 6B model: narrow experts, a short reduction in the down-projection
+        T, d, H, E = 8192, 4096, 512, 32
+        desc = dm.make_desc(T, d, H, E, dm.BF16, dm.SELECT_TOPK, K=4, fuse_combine=a.fuse)
     else:
         T, d, H, E = 8192, 3072, 1536, 32
         desc = dm.make_desc(T, d, H, E, dm.BF16, dm.SELECT_TOPK, K=12, fuse_combine=a.fuse)
@@ -96,7 +99,7 @@ def main():
     ap.add_argument("--eps", type=float, default=0.03)
     ap.add_argument("--topk", type=int, default=0, help="select exactly this many experts per token instead of the threshold")
     ap.add_argument("--reps", type=int, default=20)
-    ap.add_argument("--gemm", choices=["prefill", "dense"], default=None, help="wait-time shares of the GEMM kernel's roles instead")
+    ap.add_argument("--gemm", choices=["prefill", "dense", "paper6b"], default=None, help="wait-time shares of the GEMM kernel's roles instead")
     ap.add_argument("--fuse", type=int, default=0, help="--gemm prefill: the layer's fuse_combine (0 library's choice, 1 inside, 2 separate)")
     ap.add_argument("--pairs", type=int, default=None, help="--gemm: 0 single CTAs, 1 CTA pairs wherever the shapes allow")
     a = ap.parse_args()
