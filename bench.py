@@ -464,10 +464,48 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
         e1.record()
         barrier()
         ms_e2e = e0.elapsed_time(e1)
-        e2e_value, ms_e2e, _ = job_throughput(dist, ms_e2e, s.T * steps)
+        serial_value, ms_e2e, _ = job_throughput(dist, ms_e2e, s.T * steps)
+        # The calls as a serving loop would issue them (dsmoe_layer_forward_host_async: no wait inside the call): two
+        # streams, each with its own device buffers, workspace and pinned output, steps alternating between them, so
+        # that a step's copies run beside the other stream's kernel.  Every step still copies its input in and its
+        # output out inside the timed region, which ends when both streams have drained.
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        sets = [(x_d, out, ws, status, out_host),
+                (x_d.clone(), torch.empty_like(out), torch.empty_like(ws), torch.zeros_like(status),
+                 torch.empty((s.T, s.d), dtype=torch.bfloat16).pin_memory())]
+
+        def step_pipe(i):
+            xd, o, w, st, oh = sets[i & 1]
+            dm.dsmoe_layer_forward_host_async(desc, x_host, xd, Wr_d, br_d, None, None, packed[i % n_layers], o, oh, w, st,
+                                              stream=streams[i & 1])
+
+        torch.cuda.synchronize()
+        for i in range(4):
+            step_pipe(i)
+        barrier()
+        cur = torch.cuda.current_stream()
+        e0.record(cur)
+        for st in streams:
+            st.wait_event(e0)
+        t_issue = time.perf_counter()
+        for i in range(steps):
+            step_pipe(i)
+        t_issue = (time.perf_counter() - t_issue) / steps * 1e3
+        for st in streams:
+            ev = torch.cuda.Event()
+            ev.record(st)
+            cur.wait_event(ev)
+        e1.record(cur)
+        barrier()
+        for _, _, _, st, _ in sets:
+            if int(st.item()) != 0:
+                raise RuntimeError(f"device status {int(st.item())} in the end-to-end loop")
+        e2e_value, ms_pipe, _ = job_throughput(dist, e0.elapsed_time(e1), s.T * steps)
         nbytes = s.T * s.d * 2
-        res["e2e"] = {"value": e2e_value, "unit": "tokens/s",
-                      "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes}
+        res["e2e"] = {"value": max(e2e_value, serial_value), "unit": "tokens/s",
+                      "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes,
+                      "streams": 2 if e2e_value >= serial_value else 1, "one_stream_value": serial_value,
+                      "two_stream_value": e2e_value, "host_issue_ms_per_step": t_issue}
     del packed, ws
     return res
 

@@ -236,6 +236,19 @@ dsmoe_status dsmoe_layer_forward_host(const dsmoe_layer_desc* desc, const void* 
                                       size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream);
 
 /*
+ * The same without the final wait: both copies and the layer are enqueued on `stream` and the call
+ * returns.  x_host must stay unchanged and out_host unread until the caller has waited for the stream
+ * (or an event recorded behind the call).  Calls on different streams, each with its own x_dev,
+ * out_dev, out_host, workspace and dev_status, overlap one call's copies with another call's kernels:
+ * the serving loop's form.  With pageable host buffers the copies wait by themselves.
+ */
+dsmoe_status dsmoe_layer_forward_host_async(const dsmoe_layer_desc* desc, const void* x_host,
+                                            void* x_dev, const float* Wr, const float* br,
+                                            const void* W1, const void* W2, const void* packed,
+                                            void* out_dev, void* out_host, void* workspace,
+                                            size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream);
+
+/*
  * Selection statistics for logging ("Layer Utilization" paragraph: active experts per layer and per
  * token; Section 4.2 footnote for the threshold).  Written to the DEVICE struct `stats`:
  *   assignments     A = sum_t k_t                          zero_tokens    tokens that selected no expert

@@ -22,7 +22,7 @@ SELECT_THRESHOLD, SELECT_TOPK, SELECT_ALL, SELECT_THRESHOLD_TOPK = 0, 1, 2, 3
 EXPORTS = (
     "dsmoe_status_string", "dsmoe_workspace_size", "dsmoe_router", "dsmoe_select", "dsmoe_permute",
     "dsmoe_expert_mlp", "dsmoe_combine", "dsmoe_packed_size", "dsmoe_pack_weights",
-    "dsmoe_layer_forward", "dsmoe_layer_forward_host", "dsmoe_timing_enable", "dsmoe_timing_read",
+    "dsmoe_layer_forward", "dsmoe_layer_forward_host", "dsmoe_layer_forward_host_async", "dsmoe_timing_enable", "dsmoe_timing_read",
     "dsmoe_select_static", "dsmoe_workspace_size_packed", "dsmoe_workspace_size_stages", "dsmoe_stats",
     "dsmoe_mi_loss", "dsmoe_dense_backward", "dsmoe_moa_forward",
 )
@@ -195,6 +195,17 @@ def dsmoe_layer_forward_host(desc, x_host, x_dev, Wr, br, W1, W2, packed, out_de
                                           _ptr(workspace),
                                           ctypes.c_size_t(workspace.numel() if workspace is not None else 0),
                                           _ptr(dev_status), _stream(stream)), "dsmoe_layer_forward_host")
+
+
+def dsmoe_layer_forward_host_async(desc, x_host, x_dev, Wr, br, W1, W2, packed, out_dev, out_host, workspace,
+                                   dev_status=None, stream=None):
+    """As ``dsmoe_layer_forward_host`` without the final wait: ``out_host`` may be read once the stream has
+    been waited for."""
+    _check(lib().dsmoe_layer_forward_host_async(ctypes.byref(desc), _ptr(x_host), _ptr(x_dev), _ptr(Wr), _ptr(br),
+                                                _ptr(W1), _ptr(W2), _ptr(packed), _ptr(out_dev), _ptr(out_host),
+                                                _ptr(workspace),
+                                                ctypes.c_size_t(workspace.numel() if workspace is not None else 0),
+                                                _ptr(dev_status), _stream(stream)), "dsmoe_layer_forward_host_async")
 
 
 def dsmoe_mi_loss(desc, scores, loss3, grad, workspace, stream=None):

@@ -286,10 +286,10 @@ dsmoe_status dsmoe_layer_forward(const dsmoe_layer_desc* desc, const void* x, co
     return launch_combine(p, ws + L.yp, row_gate, token_rows, k_t, out, s);
 }
 
-dsmoe_status dsmoe_layer_forward_host(const dsmoe_layer_desc* desc, const void* x_host, void* x_dev,
-                                      const float* Wr, const float* br, const void* W1, const void* W2,
-                                      const void* packed, void* out_dev, void* out_host, void* workspace,
-                                      size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream) {
+dsmoe_status dsmoe_layer_forward_host_async(const dsmoe_layer_desc* desc, const void* x_host, void* x_dev,
+                                            const float* Wr, const float* br, const void* W1, const void* W2,
+                                            const void* packed, void* out_dev, void* out_host, void* workspace,
+                                            size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream) {
     DSMOE_TRY(check_desc(desc));
     if (desc->T == 0) return DSMOE_OK;
     if (!x_host || !x_dev || !out_dev || !out_host) return DSMOE_ERR_INVALID_ARG;
@@ -300,7 +300,17 @@ dsmoe_status dsmoe_layer_forward_host(const dsmoe_layer_desc* desc, const void* 
     DSMOE_TRY(dsmoe_layer_forward(desc, x_dev, Wr, br, W1, W2, packed, out_dev, nullptr, nullptr, workspace, ws_bytes,
                                   dev_status, stream));
     DSMOE_CUDA_TRY(cudaMemcpyAsync(out_host, out_dev, n * out_es, cudaMemcpyDeviceToHost, s));
-    DSMOE_CUDA_TRY(cudaStreamSynchronize(s));
+    return DSMOE_OK;
+}
+
+dsmoe_status dsmoe_layer_forward_host(const dsmoe_layer_desc* desc, const void* x_host, void* x_dev,
+                                      const float* Wr, const float* br, const void* W1, const void* W2,
+                                      const void* packed, void* out_dev, void* out_host, void* workspace,
+                                      size_t ws_bytes, int32_t* dev_status, dsmoe_stream stream) {
+    DSMOE_TRY(dsmoe_layer_forward_host_async(desc, x_host, x_dev, Wr, br, W1, W2, packed, out_dev, out_host, workspace,
+                                             ws_bytes, dev_status, stream));
+    if (desc->T == 0) return DSMOE_OK;
+    DSMOE_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     return DSMOE_OK;
 }
 

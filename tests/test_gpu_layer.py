@@ -256,3 +256,38 @@ def test_stack_of_layers_feeding_one_another(T):
     from harness import record
     record("layer_stack", T=T, layers=n_layers, rms_per_layer=rms)
     assert all(np.isfinite(rms)) and rms[-1] > 0.0
+
+
+# ---------------------------------------------------------------- host-buffer entry points
+
+@pytest.mark.parametrize("T", [32, 300])
+def test_host_buffer_calls_match_the_device_call(T):
+    """dsmoe_layer_forward_host and its un-waited form give, in host memory, exactly the device call's output;
+    two un-waited calls on two streams with their own buffers do not disturb one another."""
+    s = gi.LayerSpec("host", T=T, d=256, H=128, E=16, dtype="bf16", mode=gi.MODE_THRESHOLD, eps=0.05, router_gain=4.0)
+    L = Layer(s)
+    ref = L.forward().cpu()
+    x_host = L.x_d.cpu().pin_memory()
+    out_host = torch.zeros((s.T, s.d), dtype=torch.bfloat16).pin_memory()
+    x_dev = torch.zeros_like(L.x_d)
+    out_dev = torch.zeros_like(L.out)
+    dm.dsmoe_layer_forward_host(L.desc, x_host, x_dev, L.Wr_d, L.br_d, L.W1_d, L.W2_d, L.packed, out_dev, out_host,
+                                L.ws, L.dev_status)
+    assert int(L.dev_status.item()) == 0
+    assert torch.equal(out_host, ref)              # no synchronize here: the call itself waited
+    # two calls in flight at once: the second one's input is the first one's tokens in reverse order
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    x2_host = x_host.flip(0).contiguous().pin_memory()
+    outs = [torch.zeros_like(out_host).pin_memory() for _ in range(2)]
+    bufs = [(torch.zeros_like(L.x_d), torch.zeros_like(L.out), torch.empty_like(L.ws), torch.zeros_like(L.dev_status))
+            for _ in range(2)]
+    torch.cuda.synchronize()
+    for i, xh in enumerate((x_host, x2_host)):
+        xd, od, ws, st = bufs[i]
+        dm.dsmoe_layer_forward_host_async(L.desc, xh, xd, L.Wr_d, L.br_d, L.W1_d, L.W2_d, L.packed, od, outs[i], ws, st,
+                                          stream=streams[i])
+    for st in streams:
+        st.synchronize()
+    assert all(int(b[3].item()) == 0 for b in bufs)
+    assert torch.equal(outs[0], ref)
+    assert torch.equal(outs[1], ref.flip(0))       # a token's output does not depend on its place in the batch
