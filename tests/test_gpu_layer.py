@@ -53,6 +53,30 @@ def test_small_layers(case, pack, dtype):
         assert np.all(out[mask == 0] == 0.0)          # Eq. 1 with an empty selection is the zero vector
 
 
+@pytest.mark.parametrize("T,E,sel", [
+    (16384 + 70, 8, dict(mode=gi.MODE_TOPK, K=2)),            # beyond 512 chunks: the one-block scan kernel between counts and rows
+    (16384, 40, dict(mode=gi.MODE_THRESHOLD, eps=0.04)),      # exactly 512 chunks, 64-wide expert words: every block scans itself
+    (250, 8, dict(mode=gi.MODE_TOPK, K=3)),                   # up to 8 chunks: every block also counts from the masks
+    (257, 24, dict(mode=gi.MODE_THRESHOLD, eps=0.06)),        # 9 chunks, the tensor-core router's counts
+], ids=["scan_kernel", "scan_in_block_512", "count_in_block", "router_counts"])
+def test_grouping_forms_of_the_fused_layer(T, E, sel):
+    """The three ways the fused layer gets from masks to grouped rows (by number of 32-token chunks), each on a ragged
+    token count; selection, counts and the layer output against the oracle on a sample that reaches every expert."""
+    s = gi.LayerSpec(f"group{T}", T=T, d=64, H=64, E=E, dtype="bf16", router_gain=5.0, **sel)
+    r = layer_parity(s, sample=768)
+    assert r["err_rows"] <= TOL_BF16, (r["err_rows"], r["err"])
+    assert r["err"] <= TOL_BF16, r["err"]
+    L = r["layer"]
+    # the tail of the batch is where a wrong prefix over the chunks shows: compare the last tokens one by one
+    ids = np.arange(s.T - 40, s.T)
+    S = L.oracle_scores()
+    mask = to_np(L.mask)[:s.T].view(np.uint64)
+    ref = oracle.layer(L.x, L.W1, L.W2, S, mask, token_ids=ids)
+    got = np_f32(L.forward(out_fp32=True))[ids]
+    rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
+    assert float(np.abs(got - ref).max()) <= TOL_BF16 * rms
+
+
 def test_all_tokens_to_one_expert_and_empty_experts():
     s = gi.LayerSpec("onehot", T=150, d=64, H=64, E=8, dtype="bf16", mode=gi.MODE_TOPK, K=1)
     L = Layer(s)
