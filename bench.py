@@ -356,10 +356,19 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
                 step(i)
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            step(0)
-        run_step = lambda i, want=False: g.replay()     # noqa: E731
+        # a graph holds as many consecutive steps as there are weight sets (they are cycled so that no step finds its
+        # weights in L2), a second one the steps that remain: exactly `steps` steps are replayed
+        per_graph = 1 if loop else n_layers
+        graphs = {}
+        for count in {per_graph, steps % per_graph} - {0}:
+            graphs[count] = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graphs[count]):
+                for i in range(count):
+                    step(i)
+
+        def run_step(i, want=False):
+            if i % per_graph == 0:
+                graphs[min(per_graph, steps - i)].replay()
 
     # ---- device-resident timed region.  The library's event pairs around the dominant kernel's launches cost a few
     # microseconds of stream time per step.  Prefill and dense steps (milliseconds) carry them in the timed loop itself:
@@ -367,8 +376,8 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
     # timed clean, and the same un-synchronised loop runs once more with the event pairs for the kernel times.
     for i in range(max(warmup, 3)):
         run_step(i)
-    n_pairs = 0 if graph else steps * calls_per_step * timed_per_call
-    events_in_value_loop = n_pairs > 0 and not decode
+    n_pairs = steps * calls_per_step * timed_per_call
+    events_in_value_loop = n_pairs > 0 and not decode and not graph
     if events_in_value_loop:
         dm.dsmoe_timing_enable(n_pairs)
     sampler = ClockSampler(sampler_index)
@@ -392,7 +401,7 @@ def run_workload(name: str, steps: int, warmup: int, dist=None, with_e2e=True, s
         barrier()
         e0.record()
         for i in range(steps):
-            run_step(i)
+            step(i)                    # direct calls also where `value` came from graph replays: the events are the library's
         e1.record()
         barrier()
         ms_evented = e0.elapsed_time(e1) / steps
