@@ -199,8 +199,8 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
         qf[ks][2] = r0 >= 0 ? *reinterpret_cast<const uint32_t*>(qa + (size_t)r0 * H + c + 8) : 0u;
         qf[ks][3] = r1 >= 0 ? *reinterpret_cast<const uint32_t*>(qa + (size_t)r1 * H + c + 8) : 0u;
     }
-    unsigned char* Ks = moa_mma_smem + (size_t)warp * 2 * kKeyBlock * STRIDE;
-    unsigned char* Vs = Ks + kKeyBlock * STRIDE;
+    constexpr int KB = SPLIT ? kKeyBlock / 2 : kKeyBlock;     // keys per block (SPLIT: two buffers of half a block each)
+    unsigned char* const Ks0 = moa_mma_smem + (size_t)warp * 2 * kKeyBlock * STRIDE;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
     float o[DT][4];
 #pragma unroll
@@ -215,30 +215,67 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
     for (int u = same ? 0 : ps; u < (same ? ntok : ps + 1); ++u) last = max(last, min(max(pos[t0 + u], 0), L - 1));
     const __nv_bfloat16* Kh = Kc + ((size_t)(sq * n_head + j) * L) * DH;
     const __nv_bfloat16* Vh = Vc + ((size_t)(sq * n_head + j) * L) * DH;
-    const int nblocks = last / kKeyBlock + 1;
-    for (int b = SPLIT ? warp : 0; b < nblocks; b += SPLIT ? kMmaWarps : 1) {
-        const int key0 = b * kKeyBlock, nk = min(kKeyBlock, last + 1 - key0);
-        __syncwarp();
+    // Sharing out one tile's keys (SPLIT), a warp walks blocks of KB = 16 keys through two buffers: the copies of its
+    // next block are under way while it works on this one (with one buffer of 32 keys and a wait right behind the
+    // copies, the decode shape's step took 35 us for 134 MB of keys and values).  A tile per warp: one buffer of 32.
+    const int nblocks = last / KB + 1;
+    const auto fetch = [&](int b, unsigned char* Kb, unsigned char* Vb) {
+        const int key0 = b * KB, nk = min(KB, last + 1 - key0);
 #pragma unroll
-        for (int i = 0; i < CH; ++i) {                  // 32 rows x CH 16-byte pieces, a piece per lane and step
+        for (int i = 0; i < CH * KB / 32; ++i) {        // KB rows x CH 16-byte pieces, a piece per lane and step
             const int idx = lane + 32 * i, row = idx / CH, ch = idx % CH;
             // asynchronous 16-byte copies, all in flight at once; rows past the last visible key are filled with zeros
             const int rr = row < nk ? row : 0;
             const uint32_t nbytes = row < nk ? 16u : 0u;
-            const uint32_t kd = (uint32_t)__cvta_generic_to_shared(Ks + row * STRIDE + ch * 16);
-            const uint32_t vd = (uint32_t)__cvta_generic_to_shared(Vs + row * STRIDE + ch * 16);
+            const uint32_t kd = (uint32_t)__cvta_generic_to_shared(Kb + row * STRIDE + ch * 16);
+            const uint32_t vd = (uint32_t)__cvta_generic_to_shared(Vb + row * STRIDE + ch * 16);
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(kd), "l"(Kh + (size_t)(key0 + rr) * DH + ch * 8), "r"(nbytes) : "memory");
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(vd), "l"(Vh + (size_t)(key0 + rr) * DH + ch * 8), "r"(nbytes) : "memory");
         }
-        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    int buf = 0;
+    if (SPLIT && warp < nblocks) {
         __syncwarp();
-        float sc[kKeyBlock / 8][4];
+        fetch(warp, Ks0, Ks0 + KB * STRIDE);
+    }
+    for (int b = SPLIT ? warp : 0; b < nblocks; b += SPLIT ? kMmaWarps : 1) {
+        const int key0 = b * KB;
+        unsigned char* Ks = Ks0 + buf * 2 * KB * STRIDE;
+        unsigned char* Vs = Ks + KB * STRIDE;
+        if (SPLIT) {
+            __syncwarp();              // the other buffer was last read an iteration ago: every lane is past those reads
+            if (b + kMmaWarps < nblocks) {
+                unsigned char* Kn = Ks0 + (buf ^ 1) * 2 * KB * STRIDE;
+                fetch(b + kMmaWarps, Kn, Kn + KB * STRIDE);
+                asm volatile("cp.async.wait_group 1;" ::: "memory");
+            } else {
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+            }
+            buf ^= 1;
+        } else {
+            const int nk = min(KB, last + 1 - key0);
+            __syncwarp();
 #pragma unroll
-        for (int nt = 0; nt < kKeyBlock / 8; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+            for (int i = 0; i < CH; ++i) {                  // 32 rows x CH 16-byte pieces, a piece per lane and step
+                const int idx = lane + 32 * i, row = idx / CH, ch = idx % CH;
+                const int rr = row < nk ? row : 0;
+                const uint32_t nbytes = row < nk ? 16u : 0u;
+                const uint32_t kd = (uint32_t)__cvta_generic_to_shared(Ks + row * STRIDE + ch * 16);
+                const uint32_t vd = (uint32_t)__cvta_generic_to_shared(Vs + row * STRIDE + ch * 16);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(kd), "l"(Kh + (size_t)(key0 + rr) * DH + ch * 8), "r"(nbytes) : "memory");
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(vd), "l"(Vh + (size_t)(key0 + rr) * DH + ch * 8), "r"(nbytes) : "memory");
+            }
+            asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+        }
+        __syncwarp();
+        float sc[KB / 8][4];
+#pragma unroll
+        for (int nt = 0; nt < KB / 8; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
 #pragma unroll
-            for (int nt = 0; nt < kKeyBlock / 8; ++nt) {
+            for (int nt = 0; nt < KB / 8; ++nt) {
                 const unsigned char* kp = Ks + (nt * 8 + g) * STRIDE + (ks * 16 + q4 * 2) * 2;
                 mma_bf16_16816(sc[nt], qf[ks], *reinterpret_cast<const uint32_t*>(kp), *reinterpret_cast<const uint32_t*>(kp + 16));
             }
@@ -246,7 +283,7 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
         // scale, hide the keys past each row's position (and everything from rows not in this pass), new row maxima
         float bm0 = -INFINITY, bm1 = -INFINITY;
 #pragma unroll
-        for (int nt = 0; nt < kKeyBlock / 8; ++nt) {
+        for (int nt = 0; nt < KB / 8; ++nt) {
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 const int key = key0 + nt * 8 + q4 * 2 + c;
@@ -274,9 +311,9 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
             o[i][2] *= c1;
             o[i][3] *= c1;
         }
-        uint32_t pf[kKeyBlock / 16][4];
+        uint32_t pf[KB / 16][4];
 #pragma unroll
-        for (int nt = 0; nt < kKeyBlock / 8; ++nt) {
+        for (int nt = 0; nt < KB / 8; ++nt) {
             const float p0 = sc[nt][0] > -INFINITY ? __expf(sc[nt][0] - m0) : 0.f, p1 = sc[nt][1] > -INFINITY ? __expf(sc[nt][1] - m0) : 0.f;
             const float p2 = sc[nt][2] > -INFINITY ? __expf(sc[nt][2] - m1) : 0.f, p3 = sc[nt][3] > -INFINITY ? __expf(sc[nt][3] - m1) : 0.f;
             l0 += p0 + p1;
@@ -285,7 +322,7 @@ moa_attention_mma_kernel(__nv_bfloat16* __restrict__ qa, const int32_t* __restri
             pf[nt / 2][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
         }
 #pragma unroll
-        for (int kk = 0; kk < kKeyBlock / 16; ++kk) {
+        for (int kk = 0; kk < KB / 16; ++kk) {
 #pragma unroll
             for (int dt = 0; dt < DT; ++dt) {
                 uint32_t b0, b1;
