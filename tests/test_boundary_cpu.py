@@ -72,6 +72,11 @@ def test_null_pointers_and_short_workspace_are_rejected_before_any_launch():
     assert L.dsmoe_packed_size(ctypes.byref(desc), ctypes.byref(ctypes.c_size_t(0))) == 1
     empty = dm.make_desc(0, 64, 64, 4, dm.F32)
     assert L.dsmoe_layer_forward(ctypes.byref(empty), z, z, z, z, z, z, z, z, z, z, ctypes.c_size_t(0), z, z) == 0
+    # the host-buffer forms: a missing host or staging buffer is rejected before any copy; T = 0 is a no-op
+    for fn in (L.dsmoe_layer_forward_host, L.dsmoe_layer_forward_host_async):
+        assert fn(ctypes.byref(desc), z, fake, z, z, fake, fake, z, fake, fake, fake, ctypes.c_size_t(1 << 30), z, z) == 1
+        assert fn(ctypes.byref(desc), fake, fake, z, z, fake, fake, z, fake, z, fake, ctypes.c_size_t(1 << 30), z, z) == 1
+        assert fn(ctypes.byref(empty), z, z, z, z, z, z, z, z, z, z, ctypes.c_size_t(0), z, z) == 0
 
 
 def test_pack_rejects_shapes_that_are_not_multiples_of_64_and_the_new_selection_mode_is_accepted():
