@@ -38,7 +38,17 @@ __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __re
         float* sc = sc_s[warp];
         const float* src = scores + (size_t)c * kChunk * E;
         const int n = min(kChunk, T - c * kChunk) * E;
-        for (int i = lane; i < n; i += 32) sc[(i / E) * (E + 1) + i % E] = __ldg(src + i);
+#pragma unroll 1
+        for (int i0 = lane; i0 < n; i0 += 32 * 8) {      // eight coalesced loads under way at a time
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = i0 + 32 * j < n ? __ldg(src + i0 + 32 * j) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = i0 + 32 * j;
+                if (i < n) sc[(i / E) * (E + 1) + i % E] = v[j];
+            }
+        }
     }
     __shared__ int cnt_s[SCAN == 2 ? kCountInBlockChunks : 1][kMaxExperts];
     if (SCAN == 2) {
@@ -64,14 +74,35 @@ __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __re
         const int e = threadIdx.x % EP, part = threadIdx.x / EP;
         int before = 0, total = 0;
         if (e < E) {
-            for (int k = part; k < nchunks; k += parts) {
-                const int v = chunk_count(k, e);
-                total += v;
-                if (k < c0) before += v;
+            // sixteen loads are issued before the first one is used
+#pragma unroll 1
+            for (int k0 = part; k0 < nchunks; k0 += parts * 16) {
+                int v[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int k = k0 + j * parts;
+                    v[j] = k < nchunks ? chunk_count(k, e) : 0;
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    total += v[j];
+                    if (k0 + j * parts < c0) before += v[j];
+                }
             }
         }
         before_s[part][e] = before;
         total_s[part][e] = total;
+        // the block's own chunks' counts (warp 0 needs them below): asked for before the barrier
+        int own_lo[4] = {0, 0, 0, 0}, own_hi[4] = {0, 0, 0, 0};
+        if (warp == 0) {
+#pragma unroll
+            for (int w = 0; w < 3; ++w) {
+                if (c0 + w < nchunks) {
+                    if (lane < E) own_lo[w] = chunk_count(c0 + w, lane);
+                    if (lane + 32 < E) own_hi[w] = chunk_count(c0 + w, lane + 32);
+                }
+            }
+        }
         __syncthreads();
         if (warp == 0) {
             int b_lo = 0, b_hi = 0, c_lo = 0, c_hi = 0;
@@ -98,13 +129,12 @@ __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __re
             const int tot_lo = __shfl_sync(0xffffffffu, i_lo, 31);
             const int tot = tot_lo + __shfl_sync(0xffffffffu, i_hi, 31);
             int run_lo = i_lo - c_lo + b_lo, run_hi = tot_lo + i_hi - c_hi + b_hi;   // first row of chunk c0 in the expert
+#pragma unroll
             for (int w = 0; w < 4; ++w) {
                 base_s[w][lane] = run_lo;
                 base_s[w][lane + 32] = run_hi;
-                if (c0 + w < nchunks) {
-                    if (lane < E) run_lo += chunk_count(c0 + w, lane);
-                    if (lane + 32 < E) run_hi += chunk_count(c0 + w, lane + 32);
-                }
+                run_lo += own_lo[w];
+                run_hi += own_hi[w];
             }
             if (blockIdx.x == 0) {
                 if (lane < E) {
