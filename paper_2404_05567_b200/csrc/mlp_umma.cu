@@ -1967,7 +1967,7 @@ __global__ void __launch_bounds__(256) router_split_kernel(const float* __restri
 // (the reduction over d may come in `pieces` blocks of 3 EP sums each, added in ascending order).  A block is one
 // chunk of 32 tokens; with chunk_counts its first warp then counts, per expert, the chunk's tokens that selected it
 // (what chunk_count_kernel would write to chunk_prefix[chunk,:]).
-__global__ void __launch_bounds__(32 * kChunk) router_finish_kernel(const float* __restrict__ sums, const float* __restrict__ br,
+__global__ void __launch_bounds__(32 * kChunk, 2) router_finish_kernel(const float* __restrict__ sums, const float* __restrict__ br,
                                                                     float* __restrict__ scores, uint64_t* __restrict__ mask,
                                                                     int32_t* __restrict__ k_t, int32_t* __restrict__ chunk_counts,
                                                                     int T, int EP, int pieces, SelParams q) {

@@ -38,6 +38,7 @@ __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __re
         float* sc = sc_s[warp];
         const float* src = scores + (size_t)c * kChunk * E;
         const int n = min(kChunk, T - c * kChunk) * E;
+        int row = lane / E, col = lane % E;             // of element i below, kept up without a division per element
 #pragma unroll 1
         for (int i0 = lane; i0 < n; i0 += 32 * 8) {      // eight coalesced loads under way at a time
             float v[8];
@@ -45,8 +46,12 @@ __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __re
             for (int j = 0; j < 8; ++j) v[j] = i0 + 32 * j < n ? __ldg(src + i0 + 32 * j) : 0.f;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const int i = i0 + 32 * j;
-                if (i < n) sc[(i / E) * (E + 1) + i % E] = v[j];
+                if (i0 + 32 * j < n) sc[row * (E + 1) + col] = v[j];
+                col += 32;
+                while (col >= E) {
+                    col -= E;
+                    ++row;
+                }
             }
         }
     }
@@ -163,24 +168,42 @@ __global__ void __launch_bounds__(128) permute_index_kernel(const uint64_t* __re
         base_lo = lane < E ? offsets[lane] + chunk_prefix[(size_t)c * E + lane] : 0;
         base_hi = lane + 32 < E ? offsets[lane + 32] + chunk_prefix[(size_t)c * E + lane + 32] : 0;
     }
-    const float* my = sc_s[warp] + lane * (E + 1);
-    int slot = 0;
-    for (int e = 0; e < E; ++e) {
-        const bool bit = (m >> e) & 1;
-        const unsigned b = __ballot_sync(0xffffffffu, bit);
-        const int base = __shfl_sync(0xffffffffu, e < 32 ? base_lo : base_hi, e & 31);
-        if (bit) {
-            const int r = base + __popc(b & ((1u << lane) - 1u));
+    // From here a lane stands for experts `lane` and `lane + 32` and the warp walks the chunk's tokens in order: an
+    // expert's rows ascend by token, a lane counts its own rows, and nothing is exchanged between lanes but the
+    // token's selection word.  (A lane per token and a ballot per expert cost three times the instructions.)
+    const float* sc = sc_s[warp];
+    const uint32_t m_lo = (uint32_t)m, m_hi = (uint32_t)(m >> 32);
+    const uint32_t below = (1u << lane) - 1u;
+    const bool e_lo = lane < E, e_hi = lane + 32 < E;
+    const int ntok = min(kChunk, T - c * kChunk);
+    int row_lo = base_lo, row_hi = base_hi;
+    for (int tt = 0; tt < ntok; ++tt) {
+        const uint32_t a = __shfl_sync(0xffffffffu, m_lo, tt);
+        const int tok = c * kChunk + tt;
+        if (e_lo && ((a >> lane) & 1u)) {
+            const int r = row_lo++;
+            const int slot = __popc(a & below);
             if (r >= 0 && r < amax) {   // inconsistent caller-supplied offsets must not become a wild store
-                row_token[r] = t;
-                row_gate[r] = my[e];
+                row_token[r] = tok;
+                row_gate[r] = sc[tt * (E + 1) + lane];
             }
-            if (slot < W) token_rows[(size_t)t * W + slot] = r;
-            ++slot;
+            if (slot < W) token_rows[(size_t)tok * W + slot] = r;
+        }
+        if (E > 32) {
+            const uint32_t b = __shfl_sync(0xffffffffu, m_hi, tt);
+            if (e_hi && ((b >> lane) & 1u)) {
+                const int r = row_hi++;
+                const int slot = __popc(a) + __popc(b & below);
+                if (r >= 0 && r < amax) {
+                    row_token[r] = tok;
+                    row_gate[r] = sc[tt * (E + 1) + lane + 32];
+                }
+                if (slot < W) token_rows[(size_t)tok * W + slot] = r;
+            }
         }
     }
     if (t < T)
-        for (; slot < W; ++slot) token_rows[(size_t)t * W + slot] = -1;
+        for (int slot = __popcll(m); slot < W; ++slot) token_rows[(size_t)t * W + slot] = -1;
     if (zero_out) {
         // Eq. 1 with an empty selection is the zero vector: no expert tile will ever write this token's row
         unsigned none = __ballot_sync(0xffffffffu, t < T && m == 0);

@@ -43,10 +43,17 @@ __device__ __forceinline__ uint64_t select_warp(float s_lo, float s_hi, const Se
         // rank = number of experts that beat this one (higher score, or equal score and lower index)
         const int K = q.K_dev ? *q.K_dev : q.K;
         int better_lo = 0, better_hi = 0;
-        for (int j = 0; j < q.E; ++j) {
-            const float o = j < 32 ? __shfl_sync(0xffffffffu, s_lo, j) : __shfl_sync(0xffffffffu, s_hi, j - 32);
-            better_lo += (o > s_lo) || (o == s_lo && j < lane);
-            better_hi += (o > s_hi) || (o == s_hi && j < lane + 32);
+        if (q.E <= 32) {                 // one expert per lane: half the comparisons
+            for (int j = 0; j < q.E; ++j) {
+                const float o = __shfl_sync(0xffffffffu, s_lo, j);
+                better_lo += (o > s_lo) || (o == s_lo && j < lane);
+            }
+        } else {
+            for (int j = 0; j < q.E; ++j) {
+                const float o = j < 32 ? __shfl_sync(0xffffffffu, s_lo, j) : __shfl_sync(0xffffffffu, s_hi, j - 32);
+                better_lo += (o > s_lo) || (o == s_lo && j < lane);
+                better_hi += (o > s_hi) || (o == s_hi && j < lane + 32);
+            }
         }
         sel_lo = v_lo && better_lo < K;
         sel_hi = v_hi && better_hi < K;
