@@ -37,6 +37,7 @@ PAPER_SHAPES = {"1b": (2048, 256, 6), "3b": (3072, 384, 6), "6b": (4096, 512, 4)
                 "10b": (5120, 640, 4), "14b": (6144, 768, 4), "19b": (7168, 896, 4)}
 WORKLOADS = {
     "c2_t1": ("c2", dict(T=1)), "c2_t8": ("c2", dict(T=8)), "c2_t32": ("c2", dict(T=32)),
+    "c2_t64": ("c2", dict(T=64)), "c2_t128": ("c2", dict(T=128)), "c2_t256": ("c2", dict(T=256)), "c2_t512": ("c2", dict(T=512)),   # larger decode batches
     "c3": ("c3", {}), "c4": ("c4", {}),
     "c3_separate": ("c3", dict(fuse_combine=2)),   # aggregation as a second kernel instead of inside the down-projection (see dsmoe.h)
     "c5": ("c5", dict(eps=0.01)),

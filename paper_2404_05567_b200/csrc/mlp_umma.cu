@@ -1124,6 +1124,26 @@ struct RouterArgs {
 __device__ __noinline__ void small_router_pass(const RouterArgs P, Shared& sh, int KS, int w, int lane, int mode, int e,
                                                int e2) {
     constexpr int NW = kEpiThreads / 32;
+    if (KS == 0) {
+        // One CTA per token held the whole reduction (KS = 1 in the kernel) and has written that token's scores and
+        // selection itself before the grid barrier: here they are only read (a thread per token)
+        const int tt = w * 32 + lane;
+        if (mode == 0) {
+            unsigned long long m = 0ull;
+            if (tt < P.T) {
+                m = __ldcg(reinterpret_cast<const unsigned long long*>(P.mask) + tt);
+                sh.mask_s[tt] = m;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) m |= __shfl_xor_sync(0xffffffffu, m, o);
+            if (lane == 0 && m) atomicOr(&sh.active_mask, m);
+        } else if (tt < P.T) {
+            const uint64_t mk = sh.mask_s[tt];
+            sh.gate_s[tt] = ((mk >> e) & 1ull) ? __ldcg(P.scores + (size_t)tt * P.E + e) : 0.f;
+            sh.gate2_s[tt] = ((mk >> e2) & 1ull) ? __ldcg(P.scores + (size_t)tt * P.E + e2) : 0.f;
+        }
+        return;
+    }
     const bool v_lo = lane < P.E, v_hi = lane + 32 < P.E;
     const float b_lo = (P.br && v_lo) ? P.br[lane] : 0.f, b_hi = (P.br && v_hi) ? P.br[lane + 32] : 0.f;
     const int ntok = w < P.T ? (P.T - w + NW - 1) / NW : 0;
@@ -1625,7 +1645,20 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 float v = 0.f;
                 for (int r = 0; r < rpp; ++r) v += stg[(r * quads + (e >> 2)) * 4 + (e & 3)];
                 P.partial[((size_t)t * KS + sl) * kMaxExperts + e] = v;   // the partial-sum buffer is free until the down-projection
+                if (KS == 1) sh.gate_s[e] = v;          // the whole reduction: this CTA finishes its token below
             }
+        }
+        EPI_SYNC();
+        // With one CTA per token (KS = 1: 37 tokens or more) the CTA holds its token's logits: it takes softmax and
+        // selection itself and writes them out, and after the barrier every CTA reads all tokens' results instead of
+        // repeating every token's softmax (at 128 tokens that repetition, once for the selection and once for the
+        // gates, took 18 of the kernel's 76 us).  Same arithmetic as small_router_pass: bias + sum, softmax, selection.
+        const bool direct = KS == 1;
+        if (direct && (int)blockIdx.x < P.T && warp == 2) {
+            const bool v_lo = lane < P.E, v_hi = lane + 32 < P.E;
+            const float l_lo = v_lo ? (P.br ? P.br[lane] : 0.f) + sh.gate_s[lane] : 0.f;
+            const float l_hi = v_hi ? (P.br ? P.br[lane + 32] : 0.f) + sh.gate_s[lane + 32] : 0.f;
+            softmax_select_store(l_lo, l_hi, (int)blockIdx.x, P.sel, lane, P.scores, P.mask, P.k_t);
         }
         EPI_SYNC();
         if (etid == 0) {
@@ -1637,7 +1670,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         EPI_SYNC();
         // ---- router, step 2: softmax and selection of every token, in every CTA (see small_router_pass)
         const RouterArgs RA{P.T, P.E, P.br, P.partial, P.scores, P.mask, P.k_t, P.sel};
-        if (!sh.abort_flag) small_router_pass(RA, sh, KS, warp - 2, lane, 0, 0, 0);
+        if (!sh.abort_flag) small_router_pass(RA, sh, direct ? 0 : KS, warp - 2, lane, 0, 0, 0);
         EPI_SYNC();
         if (etid == 0) {
             unsigned long long m = sh.active_mask;
@@ -1692,7 +1725,7 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             if (!have) break;
             // router gate of every token for this tile's expert(s), recomputed from the slice sums (other CTAs' copies
             // of the scores are not visible yet) while the mainloop is still running
-            if (t.phase == 0 && !dead) small_router_pass(RA, sh, KS, warp - 2, lane, 1, t.e, t.e2);
+            if (t.phase == 0 && !dead) small_router_pass(RA, sh, direct ? 0 : KS, warp - 2, lane, 1, t.e, t.e2);
             if (tmem_warp && !dead && !ptx::mbar_wait(ptx::smem_u32(&sh.tfull[acc]), aph, &sh.abort_flag)) dead = true;
             dead = __any_sync(0xffffffffu, dead);     // the TMEM reads below are warp-collective
 #ifdef DSMOE_TRACE
