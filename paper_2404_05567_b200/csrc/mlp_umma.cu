@@ -42,7 +42,10 @@ constexpr int RING_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);   // operan
 #endif
 constexpr int SMALL_RING_BYTES = DSMOE_SMALL_INFLIGHT;                 // small_layer_kernel's ring
 constexpr int SHARED_BYTES = 6144 + 256;                                     // barriers and small tables (struct Shared)
-constexpr int STG_BYTES = BM * 36 * 4;                                 // epilogue staging tile: T rows x (32..256 + 4) floats
+#ifndef DSMOE_SMALL_STG_COLS
+#define DSMOE_SMALL_STG_COLS 64
+#endif
+constexpr int STG_BYTES = BM * (DSMOE_SMALL_STG_COLS + 4) * 4;         // epilogue staging tile: T rows x (64..256 + 4) floats
 // small_layer_kernel asks only for the ring bytes it keeps in flight: what it leaves stays with the SM's L1, which
 // serves the kernel's many small loads (its parameters' copy, the router's operands)
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)SMALL_RING_BYTES + SHARED_BYTES + STG_BYTES;
@@ -1737,7 +1740,10 @@ small_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 // Few tokens fill only the first TMEM lanes, so one warp would do all the GeLU work.  Instead the
                 // warps that own valid lanes copy the accumulators to shared memory, as many columns per round as the
                 // staging tile holds for T rows, and all 128 epilogue threads share the arithmetic.
-                const int CH = P.T <= 16 ? 256 : P.T <= 32 ? 128 : P.T <= 64 ? 64 : 32;   // columns per round
+                // columns per round: what the staging tile holds for T rows (a power of two, at most a whole tile)
+                constexpr int kStgFloats = STG_BYTES / 4;
+                int CH = 256;
+                while (CH > 32 && P.T * (CH + 4) > kStgFloats) CH >>= 1;
                 const int ld = CH + 4;                                                    // floats per staged row
                 for (int c0 = 0; c0 < t.bn; c0 += CH) {
                     const int cw = min(CH, t.bn - c0);
