@@ -54,7 +54,7 @@ for _n, (_d, _H, _K) in PAPER_SHAPES.items():
     WORKLOADS[f"paper{_n}_prefill"] = ("c3", dict(T=8192, d=_d, H=_H, K=_K))
     WORKLOADS[f"paper{_n}_t32"] = ("c2", dict(T=32, d=_d, H=_H))
 # dram bytes per launch of the dominant kernel from the ncu captures under profiles/ (c3: mean of the up- and down-projection)
-NCU_TRAFFIC_BYTES = {"c2_t32": 272.5e6, "c3": 1529.6e6, "c4": 1910.0e6}
+NCU_TRAFFIC_BYTES = {"c2_t32": 273.3e6, "c3": 1529.6e6, "c4": 1910.0e6}
 DEFAULT_STEPS = {"c3": 100, "c3_separate": 100, "c4": 50, "c4_backward": 20}
 ALSO = [("c2_t1", 500), ("c2_t8", 500), ("c3", 30), ("c3_separate", 30), ("c4", 15)] + [(f"c5_eps{e}", 15) for e in (0.0, 0.01, 0.05, 0.1, 0.2)] + \
        [(f"paper{n}_prefill", 30) for n in PAPER_SHAPES] + [(f"paper{n}_t32", 300) for n in ("1b", "3b", "6b", "19b")] + \
