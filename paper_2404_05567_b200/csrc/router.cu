@@ -14,62 +14,84 @@ static SelParams sel_params(const dsmoe_layer_desc& p) {
     return SelParams{p.E, p.mode, p.eps, p.eps_normalized, p.K, p.min_k, nullptr};
 }
 
-// Small T (decode): one block per token, the reduction over d split across all 256 threads.
-template <typename XT, int EP>
+// Small T (decode): a block per TT tokens (1, or 4 (2 beyond 32 experts) from 64 tokens on: the tokens of a block share its loads of Wr, which
+// every block reads in full out of L2), the reduction over d split across all 256 threads.  A token's sums are formed
+// in the same order whatever TT is.
+template <typename XT, int EP, int TT>
 __global__ void __launch_bounds__(256) router_small_kernel(const XT* __restrict__ x, const float* __restrict__ Wr,
                                                            const float* __restrict__ br, float* __restrict__ scores,
                                                            uint64_t* __restrict__ mask, int32_t* __restrict__ k_t,
-                                                           int d, SelParams q) {
-    __shared__ float red[8][EP];
-    const int t = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+                                                           int T, int d, SelParams q) {
+    __shared__ float red[TT][8][EP];
+    const int t0 = blockIdx.x * TT, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int E = q.E;
-    float acc[EP];
+    float acc[TT][EP];
 #pragma unroll
-    for (int e = 0; e < EP; ++e) acc[e] = 0.f;
-    const XT* xr = x + (size_t)t * d;
+    for (int u = 0; u < TT; ++u)
+#pragma unroll
+        for (int e = 0; e < EP; ++e) acc[u][e] = 0.f;
+    const XT* xr[TT];
+#pragma unroll
+    for (int u = 0; u < TT; ++u) xr[u] = x + (size_t)min(t0 + u, T - 1) * d;     // past the end: the last token again, unused
     if ((E & 3) == 0) {
         for (int k = tid; k < d; k += 256) {
-            const float xv = to_f32(xr[k]);
+            float xv[TT];
+#pragma unroll
+            for (int u = 0; u < TT; ++u) xv[u] = to_f32(xr[u][k]);
             const float4* w = reinterpret_cast<const float4*>(Wr + (size_t)k * E);
 #pragma unroll
             for (int e4 = 0; e4 < EP / 4; ++e4) {
                 if (e4 * 4 < E) {
                     const float4 wv = __ldg(w + e4);
-                    acc[e4 * 4 + 0] = fmaf(xv, wv.x, acc[e4 * 4 + 0]);
-                    acc[e4 * 4 + 1] = fmaf(xv, wv.y, acc[e4 * 4 + 1]);
-                    acc[e4 * 4 + 2] = fmaf(xv, wv.z, acc[e4 * 4 + 2]);
-                    acc[e4 * 4 + 3] = fmaf(xv, wv.w, acc[e4 * 4 + 3]);
+#pragma unroll
+                    for (int u = 0; u < TT; ++u) {
+                        acc[u][e4 * 4 + 0] = fmaf(xv[u], wv.x, acc[u][e4 * 4 + 0]);
+                        acc[u][e4 * 4 + 1] = fmaf(xv[u], wv.y, acc[u][e4 * 4 + 1]);
+                        acc[u][e4 * 4 + 2] = fmaf(xv[u], wv.z, acc[u][e4 * 4 + 2]);
+                        acc[u][e4 * 4 + 3] = fmaf(xv[u], wv.w, acc[u][e4 * 4 + 3]);
+                    }
                 }
             }
         }
     } else {
         for (int k = tid; k < d; k += 256) {
-            const float xv = to_f32(xr[k]);
+            float xv[TT];
+#pragma unroll
+            for (int u = 0; u < TT; ++u) xv[u] = to_f32(xr[u][k]);
             const float* w = Wr + (size_t)k * E;
 #pragma unroll
-            for (int e = 0; e < EP; ++e)
-                if (e < E) acc[e] = fmaf(xv, __ldg(w + e), acc[e]);
+            for (int e = 0; e < EP; ++e) {
+                if (e < E) {
+                    const float wv = __ldg(w + e);
+#pragma unroll
+                    for (int u = 0; u < TT; ++u) acc[u][e] = fmaf(xv[u], wv, acc[u][e]);
+                }
+            }
         }
     }
 #pragma unroll
-    for (int e = 0; e < EP; ++e) {
-        const float v = warp_sum(acc[e]);
-        if (lane == 0) red[warp][e] = v;
+    for (int u = 0; u < TT; ++u) {
+#pragma unroll
+        for (int e = 0; e < EP; ++e) {
+            const float v = warp_sum(acc[u][e]);
+            if (lane == 0) red[u][warp][e] = v;
+        }
     }
     __syncthreads();
-    if (warp == 0) {
+    if (warp < TT && t0 + warp < T) {
+        const int u = warp;
         float l_lo = 0.f, l_hi = 0.f;
         if (lane < E) {
             l_lo = br ? br[lane] : 0.f;
 #pragma unroll
-            for (int w = 0; w < 8; ++w) l_lo += red[w][lane % EP];
+            for (int w = 0; w < 8; ++w) l_lo += red[u][w][lane % EP];
         }
         if (EP > 32 && lane + 32 < E) {
             l_hi = br ? br[lane + 32] : 0.f;
 #pragma unroll
-            for (int w = 0; w < 8; ++w) l_hi += red[w][(lane + 32) % EP];
+            for (int w = 0; w < 8; ++w) l_hi += red[u][w][(lane + 32) % EP];
         }
-        softmax_select_store(l_lo, l_hi, t, q, lane, scores, mask, k_t);
+        softmax_select_store(l_lo, l_hi, t0 + u, q, lane, scores, mask, k_t);
     }
 }
 
@@ -332,10 +354,18 @@ static dsmoe_status launch_router_t(const dsmoe_layer_desc& p, const XT* x, cons
                                     float* scores, uint64_t* mask, int32_t* k_t, cudaStream_t s) {
     const SelParams q = sel_params(p);
     if (p.T <= 256) {
-        if (p.E <= 8) router_small_kernel<XT, 8><<<p.T, 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.d, q);
-        else if (p.E <= 16) router_small_kernel<XT, 16><<<p.T, 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.d, q);
-        else if (p.E <= 32) router_small_kernel<XT, 32><<<p.T, 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.d, q);
-        else router_small_kernel<XT, 64><<<p.T, 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.d, q);
+#define ROUTER_SMALL(EP, TT)                                                                                            \
+    do {                                                                                                                \
+        if (p.T >= 64)                                                                                                  \
+            router_small_kernel<XT, EP, TT><<<ceil_div(p.T, TT), 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.T, p.d, q); \
+        else                                                                                                            \
+            router_small_kernel<XT, EP, 1><<<p.T, 256, 0, s>>>(x, Wr, br, scores, mask, k_t, p.T, p.d, q);             \
+    } while (0)
+        if (p.E <= 8) ROUTER_SMALL(8, 4);
+        else if (p.E <= 16) ROUTER_SMALL(16, 4);
+        else if (p.E <= 32) ROUTER_SMALL(32, 4);
+        else ROUTER_SMALL(64, 2);                 // 2 x 64 sums a thread: four tokens' would not fit the registers
+#undef ROUTER_SMALL
     } else {
         const int grid = ceil_div(p.T, kRtTB);
         DeviceState* st = nullptr;
